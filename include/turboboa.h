@@ -1,0 +1,208 @@
+/*
+ * turboboa.h -- C ABI of the B200 (sm_100a) implementation of the TurboBoA
+ * out-channel-group weight quantizer and of its prerequisites (calibration
+ * Hessians, inverse Cholesky factors, propagated-error operands).
+ *
+ * General conventions
+ *   - Unless a parameter says "host", every tensor pointer is a DEVICE pointer
+ *     owned by the caller.  The library never allocates or frees device
+ *     memory: scratch comes from the caller as a workspace whose size the
+ *     matching *_workspace() function returns (bytes; the pointer must be
+ *     256-byte aligned).
+ *   - Matrices are dense row-major.  A weight W is [d_out][d_in], one row per
+ *     out-channel; attention heads are contiguous blocks of d_head rows
+ *     (Algorithm 1 takes W in R^{H x d_h x d}).
+ *   - `stream` is a cudaStream_t passed as void*.  All work is enqueued on it
+ *     and the call returns without synchronising.  Inputs are never modified.
+ *   - Shape, pointer and alignment errors are found on the host before any
+ *     launch and reported through the return value; nothing is enqueued in
+ *     that case.  Numerical failures (a non-positive pivot) are reported in
+ *     device words described with each call.  No call aborts, traps or throws.
+ *   - One GPU per call: the current device of the calling thread.
+ */
+#ifndef TURBOBOA_H_
+#define TURBOBOA_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  TB_OK = 0,
+  TB_ERR_INVALID_ARG = 1, /* NULL pointer, bad shape, misaligned pointer        */
+  TB_ERR_UNSUPPORTED = 2, /* a valid request outside the implemented range      */
+  TB_ERR_WORKSPACE = 3,   /* workspace NULL, misaligned or too small            */
+  TB_ERR_NOT_SPD = 4,     /* reserved for host-side checks of info words        */
+  TB_ERR_CUDA = 5,        /* a CUDA runtime call failed (launch, attribute)     */
+  TB_ERR_TIMEOUT = 6      /* reserved: a bounded device-side wait ran out       */
+} tb_status;
+
+typedef enum { TB_F32 = 0, TB_BF16 = 1 } tb_dtype;
+
+/* flags of tb_layer_desc */
+enum {
+  TB_F_ADAPTIVE_GRID = 1, /* grid chosen per out-channel group just before it is
+                             quantized (Algorithm 1, line 9; Section 3.3).  Off:
+                             the grid of every row is chosen once from the
+                             original weights (the fixed grid of BoA).         */
+  TB_F_CD_REFINE = 2      /* coordinate-descent scale refinement after the loop
+                             (Algorithm 1, line 12; Proposition 3.3)           */
+};
+
+/* Problem description of one projection (Algorithm 1, inputs). */
+typedef struct {
+  int d_out, d_in;   /* W is [d_out][d_in]; d_in must be a multiple of 128       */
+  int n_heads;       /* H; n_heads * d_head == d_out                             */
+  int d_head;        /* d_h                                                      */
+  int n_hin;         /* 1: one H_in shared by all heads (W_Q, W_K rows of
+                        Table 1); n_heads: one per head (the W_V row)            */
+  int bits;          /* b in 2..8; codes lie in {0 .. 2^b - 1}                   */
+  int quant_group;   /* columns per (scale, zero) pair: 0 = the whole row, else
+                        a multiple of 32 that divides d_in                       */
+  int out_block;     /* N of Algorithm 1: out-channels of a head quantized
+                        jointly; must divide d_head.  1 = BoA's sequential rule  */
+  int n_cand;        /* grid candidates 1..32; candidate k clips the row's
+                        min/max range by p_k = 1 - k/32                          */
+  int cd_iters;      /* passes of Algorithm 3 (the paper uses 1)                 */
+  unsigned flags;    /* TB_F_*                                                   */
+} tb_layer_desc;
+
+/* Counters written by tb_quantize_layer (device memory, 64 bytes). */
+typedef struct {
+  unsigned long long near_tie_codes; /* rounding decisions whose pre-rounding value
+                                        lay within 1e-6 of a boundary between two
+                                        distinct codes                           */
+  unsigned long long clamped_codes;  /* decisions that hit 0 or 2^b - 1 by clamp  */
+  unsigned long long column_steps;   /* dependent column steps executed          */
+  unsigned long long reserved[5];
+} tb_stats;
+
+const char* tb_status_string(tb_status st);
+
+/* --------------------------------------------------------------------------
+ * Calibration Hessians (Table 1; Algorithm 1, lines 4-5).
+ * -------------------------------------------------------------------------- */
+
+/* H += X^T X, the un-normalised running sum of the input Hessian X X^T of
+ * Table 1 (X here is token-major [n_tok][d], the transpose of the paper's X).
+ * H: [d][d] float, fully written (both triangles).  X: bf16 or float.
+ * d must be a multiple of 8.  May be called repeatedly over token chunks. */
+tb_status tb_accumulate_hessian(float* H, const void* X, tb_dtype x_type,
+                                long long n_tok, int d, void* stream);
+
+/* R += alpha * (X - Xfp)^T X, the deviation correlation alpha (X - X~) X^T of
+ * Algorithm 1 line 5 in the same un-normalised form: R[a][b] accumulates
+ * alpha * sum_t (x_t[a] - xfp_t[a]) * x_t[b].  R: [d][d] float, not symmetric. */
+tb_status tb_accumulate_cross(float* R, const void* X, const void* Xfp, tb_dtype x_type,
+                              long long n_tok, int d, float alpha, void* stream);
+
+/* H <- H / n_total + damp * mean(diag(H / n_total)) * I ; R <- R / n_total when
+ * R is not NULL.  The paper does not mention damping; damp = 0 reproduces
+ * Table 1 up to the 1/n_total normalisation, which changes no quantized
+ * weight.  Optionally keeps the undamped H / n_total in Hsum_out (or NULL). */
+tb_status tb_finalize_hessian(float* H, float* R, float* Hsum_out, int d, long long n_total,
+                              float damp, void* stream);
+
+/* Out-channel Hessians of Table 1 from the partner projection G
+ * ([g_heads * d_head][d] float, one block of d_head rows per head):
+ *   Hsum != NULL: block b gives G_b Hsum G_b^T  (= K_h^T K_h when W_Q is
+ *                 quantized and G = W_K, since K_h = (W_K,h X)^T; likewise
+ *                 Q_h^T Q_h with G = W_Q);
+ *   Hsum == NULL: block b gives G_b G_b^T (W_out,h^T W_out,h with G = W_out^T).
+ * If g_heads > n_heads (grouped-query attention, key/value side) head h sums
+ * the blocks of its g_heads / n_heads query heads; if g_heads < n_heads head h
+ * takes block h / (n_heads / g_heads).  Then damp * mean(diag) is added to
+ * the diagonal of each head.  H_out: [n_heads][d_head][d_head] float.
+ * Workspace: tb_build_hout_workspace bytes. */
+size_t tb_build_hout_workspace(int g_heads, int d_head, int d);
+tb_status tb_build_hout(float* H_out, const float* G, const float* Hsum, int n_heads,
+                        int g_heads, int d_head, int d, float damp, void* ws, size_t ws_bytes,
+                        void* stream);
+
+/* --------------------------------------------------------------------------
+ * Factors (Eq. 2): U upper triangular with H^{-1} = U^T U.
+ * -------------------------------------------------------------------------- */
+
+/* H: [n_batch][d][d] float, symmetric positive definite (only read).
+ * U: [n_batch][d][d] float; the strictly lower triangle is written as zeros.
+ * Hinv (optional, may be NULL): [n_batch][d][d] float, U^T U.
+ * info (device, [n_batch] int): 0, or the 1-based index (counted in the
+ * elimination order, which runs from the last row to the first) of the first
+ * pivot that was not positive; U of that matrix is then meaningless. */
+size_t tb_factor_workspace(int n_batch, int d);
+tb_status tb_factor(const float* H, int n_batch, int d, float* U, float* Hinv, int* info,
+                    void* ws, size_t ws_bytes, void* stream);
+
+/* Operands of the propagated-error terms from R and U_in:
+ *   P = ((R U^T) masked to its strictly upper triangle) U   (Algorithm 2, line 2)
+ *   C = R U^T U = R H_in^{-1}                               (Proposition 3.2)
+ * All [n_batch][d][d] float.  U must have a zero strictly-lower triangle. */
+size_t tb_prepare_correction_workspace(int n_batch, int d);
+tb_status tb_prepare_correction(const float* R, const float* U_in, int n_batch, int d, float* P,
+                                float* C, void* ws, size_t ws_bytes, void* stream);
+
+/* --------------------------------------------------------------------------
+ * The quantizer (Algorithm 1, lines 6-13, for one projection W).
+ * -------------------------------------------------------------------------- */
+
+/* For every head, and for every group of out_block rows in turn: choose the
+ * grid of the group's rows (line 9), run the column sweep with in-row error
+ * feedback through U_in (line 10; Algorithm 2; Eq. 2), then update the rows of
+ * the head not yet quantized with the closed-form joint compensation
+ * (line 11; Propositions 3.1 and 3.2).  After the loop optionally refine the
+ * scales by coordinate descent (line 12; Proposition 3.3 / Algorithm 3) and
+ * write Q = diag(s)(W_int - z) (line 13).
+ *
+ * Inputs
+ *   W      [d_out][d_in] float
+ *   H_in   [n_hin][d_in][d_in] float, symmetric
+ *   U_in   [n_hin][d_in][d_in] float, upper factor of H_in^{-1}
+ *   H_out  [n_heads][d_head][d_head] float, or NULL for the identity (the GPTQ /
+ *          GPTAQ row of Table 1: every row of a head is quantized at once and
+ *          there is no compensation); U_out likewise (NULL iff H_out is NULL)
+ *   R, P, C  [n_hin][d_in][d_in] float each, or all three NULL (no propagated
+ *          error: the first block of a model)
+ * Outputs
+ *   codes  [d_out][d_in] unsigned char, W_int
+ *   scales [d_out][n_g] float, n_g = d_in / quant_group (1 if quant_group = 0)
+ *   zeros  [d_out][n_g] int, integer zero-points z (the paper's grid has none;
+ *          every formula holds with W_int replaced by W_int - z)
+ *   cand   [d_out][n_g] unsigned char or NULL: index k of the chosen grid candidate
+ *   W_hat  [d_out][d_in] float or NULL: Q
+ *   loss   [n_heads] double or NULL: tr(dW H_in dW^T H_out) + 2 tr(H_out W R dW^T),
+ *          dW = Q - W (the objective in the proofs of Propositions 3.1 / 3.2)
+ *   stats  tb_stats (device) or NULL
+ * The arithmetic of the loop is IEEE double precision: codes are integer
+ * decisions taken inside an error-feedback chain d_in steps long, and they
+ * only reproduce across implementations when the chain is carried in double. */
+size_t tb_quantize_layer_workspace(const tb_layer_desc* desc, int with_r, int with_loss);
+tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W, const float* H_in,
+                            const float* U_in, const float* H_out, const float* U_out,
+                            const float* R, const float* P, const float* C,
+                            unsigned char* codes, float* scales, int* zeros, unsigned char* cand,
+                            float* W_hat, double* loss, tb_stats* stats, void* ws,
+                            size_t ws_bytes, void* stream);
+
+/* Whole path for one projection from HOST buffers: copies X (and G) to the
+ * device, accumulates and finalises H_in, builds H_out, factors both, runs
+ * tb_quantize_layer and copies codes / scales / zeros / W_hat / loss back.
+ * Every *_host pointer is host memory (pinned memory makes the copies
+ * asynchronous); dev_ws is a DEVICE workspace of
+ * tb_quantize_from_host_workspace bytes.  The call synchronises the stream
+ * before it returns.  X_host is bf16 [n_tok][d_in]; G_host is the partner
+ * projection [g_heads*d_head][d_in] float or NULL (then H_out = identity).
+ * Returns TB_ERR_NOT_SPD if a factorisation met a non-positive pivot. */
+size_t tb_quantize_from_host_workspace(const tb_layer_desc* desc, long long n_tok, int g_heads);
+tb_status tb_quantize_from_host(const tb_layer_desc* desc, const float* W_host,
+                                const void* X_host, long long n_tok, const float* G_host,
+                                int g_heads, float damp_in, float damp_out,
+                                unsigned char* codes_host, float* scales_host, int* zeros_host,
+                                float* W_hat_host, double* loss_host, void* dev_ws,
+                                size_t ws_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TURBOBOA_H_ */

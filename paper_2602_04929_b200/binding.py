@@ -1,0 +1,272 @@
+"""Thin ctypes binding of libturboboa.so: argument marshalling only.
+
+Every function has the name of the C entry point it calls (include/turboboa.h)
+and takes torch CUDA tensors; torch provides device memory and the stream and
+nothing else.  There is no CPU path: a missing library or a missing GPU raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+from . import _build
+
+TB_OK = 0
+TB_F32, TB_BF16 = 0, 1
+TB_F_ADAPTIVE_GRID, TB_F_CD_REFINE = 1, 2
+
+_STATUS_NAMES = {0: "TB_OK", 1: "TB_ERR_INVALID_ARG", 2: "TB_ERR_UNSUPPORTED", 3: "TB_ERR_WORKSPACE",
+                 4: "TB_ERR_NOT_SPD", 5: "TB_ERR_CUDA", 6: "TB_ERR_TIMEOUT"}
+
+
+class TurboBoAError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {_STATUS_NAMES.get(status, status)} ({status_string(status)})")
+
+
+class LayerDesc(ctypes.Structure):
+    """tb_layer_desc"""
+    _fields_ = [("d_out", ctypes.c_int), ("d_in", ctypes.c_int), ("n_heads", ctypes.c_int),
+                ("d_head", ctypes.c_int), ("n_hin", ctypes.c_int), ("bits", ctypes.c_int),
+                ("quant_group", ctypes.c_int), ("out_block", ctypes.c_int), ("n_cand", ctypes.c_int),
+                ("cd_iters", ctypes.c_int), ("flags", ctypes.c_uint)]
+
+    @property
+    def n_groups(self) -> int:
+        return 1 if self.quant_group == 0 else self.d_in // self.quant_group
+
+
+def layer_desc(d_out, d_in, n_heads, d_head, bits, quant_group=0, out_block=1, n_hin=1, n_cand=16,
+               cd_iters=1, flags=0) -> LayerDesc:
+    return LayerDesc(d_out, d_in, n_heads, d_head, n_hin, bits, quant_group, out_block, n_cand,
+                     cd_iters, flags)
+
+
+class Stats(ctypes.Structure):
+    """tb_stats"""
+    _fields_ = [("near_tie_codes", ctypes.c_ulonglong), ("clamped_codes", ctypes.c_ulonglong),
+                ("column_steps", ctypes.c_ulonglong), ("reserved", ctypes.c_ulonglong * 5)]
+
+
+_lib = None
+_vp, _sz, _ll, _int, _f = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_longlong, ctypes.c_int, ctypes.c_float
+_SIGNATURES = {
+    "tb_status_string": (ctypes.c_char_p, [_int]),
+    "tb_accumulate_hessian": (_int, [_vp, _vp, _int, _ll, _int, _vp]),
+    "tb_accumulate_cross": (_int, [_vp, _vp, _vp, _int, _ll, _int, _f, _vp]),
+    "tb_finalize_hessian": (_int, [_vp, _vp, _vp, _int, _ll, _f, _vp]),
+    "tb_build_hout_workspace": (_sz, [_int, _int, _int]),
+    "tb_build_hout": (_int, [_vp, _vp, _vp, _int, _int, _int, _int, _f, _vp, _sz, _vp]),
+    "tb_factor_workspace": (_sz, [_int, _int]),
+    "tb_factor": (_int, [_vp, _int, _int, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "tb_prepare_correction_workspace": (_sz, [_int, _int]),
+    "tb_prepare_correction": (_int, [_vp, _vp, _int, _int, _vp, _vp, _vp, _sz, _vp]),
+    "tb_quantize_layer_workspace": (_sz, [ctypes.POINTER(LayerDesc), _int, _int]),
+    "tb_quantize_layer": (_int, [ctypes.POINTER(LayerDesc)] + [_vp] * 15 + [_vp, _sz, _vp]),
+    "tb_quantize_from_host_workspace": (_sz, [ctypes.POINTER(LayerDesc), _ll, _int]),
+    "tb_quantize_from_host": (_int, [ctypes.POINTER(LayerDesc), _vp, _vp, _ll, _vp, _int, _f, _f,
+                                     _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+}
+
+
+def library_path() -> str:
+    return _build.LIB
+
+
+def load(build_if_missing: bool = True) -> ctypes.CDLL:
+    """Load libturboboa.so (building it in-tree first if it is absent or stale)."""
+    global _lib
+    if _lib is None:
+        if build_if_missing:
+            _build.build()
+        if not os.path.exists(_build.LIB):
+            raise RuntimeError("libturboboa.so is missing; run `python -m paper_2602_04929_b200._build`")
+        lib = ctypes.CDLL(_build.LIB)
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = lib
+    return _lib
+
+
+def exported_symbols() -> list[str]:
+    return sorted(_SIGNATURES)
+
+
+def status_string(status: int) -> str:
+    return load().tb_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != TB_OK:
+        raise TurboBoAError(status, where)
+
+
+def _ptr(t, dtype=None, allow_none=False):
+    if t is None:
+        if allow_none:
+            return None
+        raise ValueError("a required tensor is None")
+    if not t.is_cuda:
+        raise ValueError("tensors must live on a CUDA device (there is no CPU path)")
+    if not t.is_contiguous():
+        raise ValueError("tensors must be contiguous")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError(f"expected {dtype}, got {t.dtype}")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _workspace(nbytes: int, device) -> torch.Tensor:
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def _xtype(X):
+    if X.dtype == torch.bfloat16:
+        return TB_BF16
+    if X.dtype == torch.float32:
+        return TB_F32
+    raise ValueError("activations must be bfloat16 or float32")
+
+
+def tb_accumulate_hessian(H, X) -> None:
+    n_tok, d = X.shape
+    _check(load().tb_accumulate_hessian(_ptr(H, torch.float32), _ptr(X), _xtype(X), n_tok, d, _stream()),
+           "tb_accumulate_hessian")
+
+
+def tb_accumulate_cross(R, X, Xfp, alpha: float) -> None:
+    n_tok, d = X.shape
+    if Xfp.dtype != X.dtype or Xfp.shape != X.shape:
+        raise ValueError("X and Xfp must agree in shape and dtype")
+    _check(load().tb_accumulate_cross(_ptr(R, torch.float32), _ptr(X), _ptr(Xfp), _xtype(X), n_tok, d,
+                                      float(alpha), _stream()), "tb_accumulate_cross")
+
+
+def tb_finalize_hessian(H, R, n_total: int, damp: float, Hsum_out=None) -> None:
+    d = H.shape[-1]
+    _check(load().tb_finalize_hessian(_ptr(H, torch.float32), _ptr(R, torch.float32, True),
+                                      _ptr(Hsum_out, torch.float32, True), d, int(n_total), float(damp),
+                                      _stream()), "tb_finalize_hessian")
+
+
+def tb_build_hout(G, Hsum, n_heads: int, d_head: int, damp: float):
+    rows, d = G.shape
+    g_heads = rows // d_head
+    lib = load()
+    H_out = torch.empty((n_heads, d_head, d_head), dtype=torch.float32, device=G.device)
+    ws = _workspace(lib.tb_build_hout_workspace(g_heads, d_head, d), G.device)
+    _check(lib.tb_build_hout(_ptr(H_out), _ptr(G, torch.float32), _ptr(Hsum, torch.float32, True), n_heads,
+                             g_heads, d_head, d, float(damp), _ptr(ws), ws.numel(), _stream()),
+           "tb_build_hout")
+    return H_out
+
+
+def tb_factor(H, want_inverse: bool = False):
+    """Returns (U, info[, Hinv]) for H of shape [n_batch, d, d] or [d, d]."""
+    squeeze = H.dim() == 2
+    Hb = H.unsqueeze(0) if squeeze else H
+    n_batch, d, _ = Hb.shape
+    lib = load()
+    U = torch.empty_like(Hb)
+    Hinv = torch.empty_like(Hb) if want_inverse else None
+    info = torch.empty(n_batch, dtype=torch.int32, device=H.device)
+    ws = _workspace(lib.tb_factor_workspace(n_batch, d), H.device)
+    _check(lib.tb_factor(_ptr(Hb, torch.float32), n_batch, d, _ptr(U), _ptr(Hinv, None, True), _ptr(info),
+                         _ptr(ws), ws.numel(), _stream()), "tb_factor")
+    if squeeze:
+        U = U[0]
+        Hinv = Hinv[0] if want_inverse else None
+    return (U, info, Hinv) if want_inverse else (U, info)
+
+
+def tb_prepare_correction(R, U_in):
+    squeeze = R.dim() == 2
+    Rb = R.unsqueeze(0) if squeeze else R
+    Ub = U_in.unsqueeze(0) if squeeze else U_in
+    n_batch, d, _ = Rb.shape
+    lib = load()
+    P = torch.empty_like(Rb)
+    C = torch.empty_like(Rb)
+    ws = _workspace(lib.tb_prepare_correction_workspace(n_batch, d), R.device)
+    _check(lib.tb_prepare_correction(_ptr(Rb, torch.float32), _ptr(Ub, torch.float32), n_batch, d, _ptr(P),
+                                     _ptr(C), _ptr(ws), ws.numel(), _stream()), "tb_prepare_correction")
+    return (P[0], C[0]) if squeeze else (P, C)
+
+
+@dataclass
+class QuantizeResult:
+    codes: torch.Tensor
+    scales: torch.Tensor
+    zeros: torch.Tensor
+    cand: torch.Tensor
+    w_hat: torch.Tensor
+    loss: torch.Tensor | None
+    stats: torch.Tensor
+
+    def stats_dict(self) -> dict:
+        v = self.stats.cpu().tolist()
+        return {"near_tie_codes": v[0], "clamped_codes": v[1], "column_steps": v[2]}
+
+
+def tb_quantize_layer_workspace(desc: LayerDesc, with_r: bool, with_loss: bool) -> int:
+    return int(load().tb_quantize_layer_workspace(ctypes.byref(desc), int(with_r), int(with_loss)))
+
+
+def tb_quantize_layer(desc: LayerDesc, W, H_in, U_in, H_out=None, U_out=None, R=None, P=None, C=None,
+                      want_loss: bool = True, ws=None, out: QuantizeResult | None = None) -> QuantizeResult:
+    lib = load()
+    dev = W.device
+    ng = desc.n_groups
+    if out is None:
+        out = QuantizeResult(
+            codes=torch.empty((desc.d_out, desc.d_in), dtype=torch.uint8, device=dev),
+            scales=torch.empty((desc.d_out, ng), dtype=torch.float32, device=dev),
+            zeros=torch.empty((desc.d_out, ng), dtype=torch.int32, device=dev),
+            cand=torch.empty((desc.d_out, ng), dtype=torch.uint8, device=dev),
+            w_hat=torch.empty((desc.d_out, desc.d_in), dtype=torch.float32, device=dev),
+            loss=torch.empty(desc.n_heads, dtype=torch.float64, device=dev) if want_loss else None,
+            stats=torch.zeros(8, dtype=torch.int64, device=dev))
+    if ws is None:
+        ws = _workspace(tb_quantize_layer_workspace(desc, R is not None, out.loss is not None), dev)
+    f32 = torch.float32
+    _check(lib.tb_quantize_layer(
+        ctypes.byref(desc), _ptr(W, f32), _ptr(H_in, f32), _ptr(U_in, f32), _ptr(H_out, f32, True),
+        _ptr(U_out, f32, True), _ptr(R, f32, True), _ptr(P, f32, True), _ptr(C, f32, True),
+        _ptr(out.codes), _ptr(out.scales), _ptr(out.zeros), _ptr(out.cand), _ptr(out.w_hat),
+        _ptr(out.loss, None, True), _ptr(out.stats), _ptr(ws), ws.numel(), _stream()), "tb_quantize_layer")
+    return out
+
+
+def tb_quantize_from_host_workspace(desc: LayerDesc, n_tok: int, g_heads: int) -> int:
+    return int(load().tb_quantize_from_host_workspace(ctypes.byref(desc), int(n_tok), int(g_heads)))
+
+
+def tb_quantize_from_host(desc: LayerDesc, W_host, X_host, G_host, damp_in: float, damp_out: float,
+                          out_host: dict, dev_ws) -> None:
+    """All *_host arguments are CPU tensors (pinned for asynchronous copies);
+    out_host holds preallocated CPU tensors codes, scales, zeros, w_hat, loss."""
+    lib = load()
+
+    def hp(t):
+        if t is None:
+            return None
+        if t.is_cuda or not t.is_contiguous():
+            raise ValueError("host tensors must be contiguous CPU tensors")
+        return ctypes.c_void_p(t.data_ptr())
+
+    n_tok = X_host.shape[0]
+    g_heads = 0 if G_host is None else G_host.shape[0] // desc.d_head
+    _check(lib.tb_quantize_from_host(
+        ctypes.byref(desc), hp(W_host), hp(X_host), n_tok, hp(G_host), g_heads, float(damp_in),
+        float(damp_out), hp(out_host["codes"]), hp(out_host["scales"]), hp(out_host["zeros"]),
+        hp(out_host.get("w_hat")), hp(out_host.get("loss")), _ptr(dev_ws), dev_ws.numel(), _stream()),
+        "tb_quantize_from_host")

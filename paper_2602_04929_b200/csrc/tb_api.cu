@@ -1,0 +1,135 @@
+// Status strings and the host-buffer entry point that chains the whole path:
+// Hessians -> factors -> quantizer (Algorithm 1 for one projection).
+#include "tb_common.cuh"
+
+using namespace tb;
+
+extern "C" const char* tb_status_string(tb_status st) {
+  switch (st) {
+    case TB_OK: return "ok";
+    case TB_ERR_INVALID_ARG: return "invalid argument";
+    case TB_ERR_UNSUPPORTED: return "unsupported configuration";
+    case TB_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case TB_ERR_NOT_SPD: return "matrix not positive definite";
+    case TB_ERR_CUDA: return "CUDA runtime error";
+    case TB_ERR_TIMEOUT: return "bounded device wait ran out";
+  }
+  return "unknown status";
+}
+
+namespace {
+
+struct HostPlan {
+  float *W, *G, *Hsum, *Hin, *Uin, *Hout, *Uout, *scales, *What;
+  __nv_bfloat16* X;
+  int *info, *zeros;
+  unsigned char* codes;
+  double* loss;
+  void* sub;
+  size_t sub_bytes, total;
+};
+
+size_t max_sz(size_t a, size_t b) { return a > b ? a : b; }
+
+HostPlan host_plan(const tb_layer_desc* D, long long n_tok, int g_heads, void* ws) {
+  HostPlan h;
+  Bump b(ws);
+  const size_t d = (size_t)D->d_in, dout = (size_t)D->d_out;
+  const size_t ng = D->quant_group > 0 ? d / (size_t)D->quant_group : 1;
+  h.W = b.take<float>(dout * d);
+  h.X = b.take<__nv_bfloat16>((size_t)n_tok * d);
+  h.G = g_heads > 0 ? b.take<float>((size_t)g_heads * D->d_head * d) : nullptr;
+  h.Hsum = b.take<float>(d * d);
+  h.Hin = b.take<float>(d * d);
+  h.Uin = b.take<float>(d * d);
+  h.Hout = g_heads > 0 ? b.take<float>((size_t)D->n_heads * D->d_head * D->d_head) : nullptr;
+  h.Uout = g_heads > 0 ? b.take<float>((size_t)D->n_heads * D->d_head * D->d_head) : nullptr;
+  h.info = b.take<int>((size_t)D->n_heads + 1);
+  h.codes = b.take<unsigned char>(dout * d);
+  h.scales = b.take<float>(dout * ng);
+  h.zeros = b.take<int>(dout * ng);
+  h.What = b.take<float>(dout * d);
+  h.loss = b.take<double>((size_t)D->n_heads);
+  size_t sub = tb_factor_workspace(1, D->d_in);
+  if (g_heads > 0) {
+    sub = max_sz(sub, tb_factor_workspace(D->n_heads, D->d_head));
+    sub = max_sz(sub, tb_build_hout_workspace(g_heads, D->d_head, D->d_in));
+  }
+  sub = max_sz(sub, tb_quantize_layer_workspace(D, 0, 1));
+  h.sub = b.take<unsigned char>(sub);
+  h.sub_bytes = sub;
+  h.total = b.total();
+  return h;
+}
+
+bool desc_ok(const tb_layer_desc* D, long long n_tok, int g_heads) {
+  if (!D || n_tok <= 0 || g_heads < 0) return false;
+  if (D->d_out <= 0 || D->d_in <= 0 || D->n_heads <= 0 || D->d_head <= 0) return false;
+  if ((long long)D->n_heads * D->d_head != D->d_out) return false;
+  if (D->quant_group < 0 || (D->quant_group > 0 && D->d_in % D->quant_group)) return false;
+  if (g_heads > 0 && (g_heads >= D->n_heads ? g_heads % D->n_heads : D->n_heads % g_heads)) return false;
+  return true;
+}
+
+}  // namespace
+
+extern "C" size_t tb_quantize_from_host_workspace(const tb_layer_desc* desc, long long n_tok,
+                                                  int g_heads) {
+  if (!desc_ok(desc, n_tok, g_heads)) return 0;
+  return host_plan(desc, n_tok, g_heads, nullptr).total;
+}
+
+extern "C" tb_status tb_quantize_from_host(const tb_layer_desc* desc, const float* W_host,
+                                           const void* X_host, long long n_tok,
+                                           const float* G_host, int g_heads, float damp_in,
+                                           float damp_out, unsigned char* codes_host,
+                                           float* scales_host, int* zeros_host, float* W_hat_host,
+                                           double* loss_host, void* dev_ws, size_t ws_bytes,
+                                           void* stream) {
+  if (!desc_ok(desc, n_tok, G_host ? g_heads : 0)) return TB_ERR_INVALID_ARG;
+  if (!W_host || !X_host || !codes_host || !scales_host || !zeros_host) return TB_ERR_INVALID_ARG;
+  if (desc->n_hin != 1) return TB_ERR_UNSUPPORTED;  // one shared H_in on this entry point
+  if (!G_host) g_heads = 0;
+  const HostPlan hs = host_plan(desc, n_tok, g_heads, nullptr);
+  if (!dev_ws || !aligned(dev_ws, 256) || ws_bytes < hs.total) return TB_ERR_WORKSPACE;
+  const HostPlan h = host_plan(desc, n_tok, g_heads, dev_ws);
+  cudaStream_t st = as_stream(stream);
+  const size_t d = (size_t)desc->d_in, dout = (size_t)desc->d_out;
+  const size_t ng = desc->quant_group > 0 ? d / (size_t)desc->quant_group : 1;
+  const int H = desc->n_heads, dh = desc->d_head;
+
+  TB_CUDA_CHECK(cudaMemcpyAsync(h.W, W_host, dout * d * sizeof(float), cudaMemcpyHostToDevice, st));
+  TB_CUDA_CHECK(cudaMemcpyAsync(h.X, X_host, (size_t)n_tok * d * sizeof(__nv_bfloat16),
+                                cudaMemcpyHostToDevice, st));
+  if (g_heads > 0)
+    TB_CUDA_CHECK(cudaMemcpyAsync(h.G, G_host, (size_t)g_heads * dh * d * sizeof(float),
+                                  cudaMemcpyHostToDevice, st));
+  TB_CUDA_CHECK(cudaMemsetAsync(h.Hin, 0, d * d * sizeof(float), st));
+  TB_TRY(tb_accumulate_hessian(h.Hin, h.X, TB_BF16, n_tok, (int)d, stream));
+  TB_TRY(tb_finalize_hessian(h.Hin, nullptr, h.Hsum, (int)d, n_tok, damp_in, stream));
+  TB_TRY(tb_factor(h.Hin, 1, (int)d, h.Uin, nullptr, h.info, h.sub, h.sub_bytes, stream));
+  if (g_heads > 0) {
+    TB_TRY(tb_build_hout(h.Hout, h.G, h.Hsum, H, g_heads, dh, (int)d, damp_out, h.sub, h.sub_bytes,
+                         stream));
+    TB_TRY(tb_factor(h.Hout, H, dh, h.Uout, nullptr, h.info + 1, h.sub, h.sub_bytes, stream));
+  } else {
+    TB_CUDA_CHECK(cudaMemsetAsync(h.info + 1, 0, sizeof(int) * (size_t)H, st));
+  }
+  TB_TRY(tb_quantize_layer(desc, h.W, h.Hin, h.Uin, h.Hout, h.Uout, nullptr, nullptr, nullptr,
+                           h.codes, h.scales, h.zeros, nullptr, W_hat_host ? h.What : nullptr,
+                           loss_host ? h.loss : nullptr, nullptr, h.sub, h.sub_bytes, stream));
+  TB_CUDA_CHECK(cudaMemcpyAsync(codes_host, h.codes, dout * d, cudaMemcpyDeviceToHost, st));
+  TB_CUDA_CHECK(cudaMemcpyAsync(scales_host, h.scales, dout * ng * sizeof(float), cudaMemcpyDeviceToHost, st));
+  TB_CUDA_CHECK(cudaMemcpyAsync(zeros_host, h.zeros, dout * ng * sizeof(int), cudaMemcpyDeviceToHost, st));
+  if (W_hat_host)
+    TB_CUDA_CHECK(cudaMemcpyAsync(W_hat_host, h.What, dout * d * sizeof(float), cudaMemcpyDeviceToHost, st));
+  if (loss_host)
+    TB_CUDA_CHECK(cudaMemcpyAsync(loss_host, h.loss, sizeof(double) * (size_t)H, cudaMemcpyDeviceToHost, st));
+  int info_host[1 + 4096];
+  const int n_info = 1 + (H < 4096 ? H : 4096);
+  TB_CUDA_CHECK(cudaMemcpyAsync(info_host, h.info, sizeof(int) * (size_t)n_info, cudaMemcpyDeviceToHost, st));
+  TB_CUDA_CHECK(cudaStreamSynchronize(st));
+  for (int i = 0; i < n_info; ++i)
+    if (info_host[i] != 0) return TB_ERR_NOT_SPD;
+  return TB_OK;
+}

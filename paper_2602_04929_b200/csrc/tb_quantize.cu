@@ -1,0 +1,1150 @@
+// tb_quantize_layer: the out-channel-group loop of Algorithm 1 (lines 6-13).
+//
+// Per step i (a group of g = out_block rows of every head, M = n_heads * g
+// rows in all, heads being independent):
+//   grid     k_grid           Algorithm 1 line 9    candidate search per (row, column group)
+//   sweep    k_sweep_block    Algorithm 2 / Eq. 2   one launch per 128-column block
+//   residual k_residual       E = W0 - Q_B          (Proposition 3.1)
+//            GEMM             E -= W0 C             (Proposition 3.2, only with R)
+//   update   GEMM             W~[rem] -= T_i E      (Algorithm 1 line 11)
+// then, once: coordinate descent on the scales (Algorithm 3), Q = s (W_int - z),
+// and the loss of the proofs of Propositions 3.1 / 3.2.
+//
+// All of this runs in IEEE double on the CUDA cores.  The codes are integer
+// decisions inside an error-feedback chain d_in steps long; in float the
+// accumulated rounding error of the chain (a few 1e-6 code units) exceeds the
+// 1e-6 band inside which a rounding decision may legitimately differ, and one
+// different decision changes every later code of its row.
+#include "tb_common.cuh"
+#include "tb_gemm.cuh"
+
+namespace tb {
+
+// ---------------------------------------------------------------------------
+// Row bookkeeping.  Active row m of a step maps to head m / g, row i0 + m % g
+// of that head.  "Units" are sets of rows that share one H_in / U_in: the
+// whole step when H_in is shared, one head otherwise.
+// ---------------------------------------------------------------------------
+struct RowMap {
+  int g, d_head, i0;
+  __host__ __device__ long long row(int m) const {
+    return (long long)(m / g) * d_head + i0 + (m % g);
+  }
+};
+
+__global__ void k_widen(const float* __restrict__ W, double* __restrict__ Wt, long long n) {
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n;
+       i += (long long)gridDim.x * blockDim.x)
+    Wt[i] = (double)W[i];
+}
+
+// Wk[m][:] = W~[row(m)][:]  (and a second untouched copy W0c when the
+// propagated-error term needs the snapshot as a contiguous GEMM operand)
+__global__ void k_gather(const double* __restrict__ Wt, double* __restrict__ Wk,
+                         double* __restrict__ W0c, RowMap rm, int M, int d) {
+  const long long n = (long long)M * d;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n;
+       i += (long long)gridDim.x * blockDim.x) {
+    const int m = (int)(i / d), k = (int)(i % d);
+    const double v = Wt[rm.row(m) * d + k];
+    Wk[i] = v;
+    if (W0c) W0c[i] = v;
+  }
+}
+
+// ---------------------------------------------------------------------------
+// Compensation matrices of Propositions 3.1 / 3.2 for every head and step:
+//   T = [U_out^T]_{rem,B} ([U_out^T]_{B,B})^{-1},  B = {i0..i0+g-1}, rem = rows after B.
+// With A = U_out^T lower triangular, T A_BB = A_remB is solved row by row,
+// last column first.  T is stored [head][step][d_head][g] (first rem rows used).
+// ---------------------------------------------------------------------------
+__global__ void k_comp_matrices(const float* __restrict__ Uout, double* __restrict__ T, int dh,
+                                int g, int n_steps) {
+  const int step = blockIdx.x, head = blockIdx.y;
+  const int i0 = step * g, r0 = i0 + g, nrem = dh - r0;
+  const float* Uo = Uout + (long long)head * dh * dh;
+  double* Th = T + ((long long)head * n_steps + step) * dh * g;
+  for (int r = threadIdx.x; r < nrem; r += blockDim.x) {
+    double* Tr = Th + (long long)r * g;
+    for (int c = g - 1; c >= 0; --c) {
+      const float* urow = Uo + (long long)(i0 + c) * dh;
+      double v = (double)urow[r0 + r];
+      for (int c2 = c + 1; c2 < g; ++c2) v -= Tr[c2] * (double)urow[i0 + c2];
+      Tr[c] = v / (double)urow[i0 + c];
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------
+// Grid search (Algorithm 1 line 9).  For every (row, column group): n_cand
+// clipped min-max grids, p_k = 1 - k/32; score e H_in[G,G] e^T with e the
+// round-to-nearest error on that grid; the lowest score wins, lowest k on ties.
+//
+// One CTA takes RT = 128 / NCP rows (NCP = n_cand rounded up to a power of
+// two) of one column group: RT * NCP = 128 "candidate rows".  The scores are
+// the row-wise dots of (E H) with E, where E [128 x seg] holds the candidate
+// errors; E H runs on the GEMM tile engine with E produced on the fly.
+// ---------------------------------------------------------------------------
+struct GridP {
+  const double* Wt;   // [d_out][d]
+  const float* Hin;   // [n_hin][d][d]
+  double* sD;         // [d_out][ng]
+  float* s_out;       // [d_out][ng]
+  int* z_out;         // [d_out][ng]
+  unsigned char* cand_out;  // or nullptr
+  RowMap rm;
+  int M, d, seg, ng, maxq, n_cand, ncp, rt;
+  int units, rows_per_unit, tiles_per_unit;
+};
+
+__global__ void __launch_bounds__(GEMM_THREADS, 1) k_grid(GridP p) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  __shared__ double c_s[128], c_rs[128], c_z[128], c_J[128];
+  __shared__ long long c_row[128];  // global row of a candidate row, or -1
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int grp = blockIdx.x;
+  const int unit = blockIdx.y / p.tiles_per_unit;
+  const int tile = blockIdx.y % p.tiles_per_unit;
+  const int seg0 = grp * p.seg;
+  const double maxq = (double)p.maxq;
+
+  // Phase 1: min / max of every row segment, then the candidates' (s, z).
+  for (int r = warp; r < p.rt; r += GEMM_THREADS / 32) {
+    const int rloc = tile * p.rt + r;
+    const bool valid = rloc < p.rows_per_unit;
+    long long grow = -1;
+    double mn = 0.0, mx = 0.0;
+    if (valid) {
+      grow = p.rm.row(unit * p.rows_per_unit + rloc);
+      const double* w = p.Wt + grow * p.d + seg0;
+      for (int a = lane; a < p.seg; a += 32) {
+        const double v = w[a];
+        mn = fmin(mn, v);
+        mx = fmax(mx, v);
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        mn = fmin(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+        mx = fmax(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      }
+    }
+    if (lane < p.ncp) {
+      const int k = lane, cr = r * p.ncp + k;
+      double s = 1.0, z = 0.0;
+      if (valid && k < p.n_cand) {
+        const double pk = 1.0 - (double)k / 32.0;
+        const double lo = pk * mn, hi = pk * mx;
+        if (hi != lo) {
+          s = (hi - lo) / maxq;
+          z = fmin(fmax(rne(-lo / s), 0.0), maxq);
+        }
+      }
+      c_s[cr] = s;
+      c_rs[cr] = 1.0 / s;
+      c_z[cr] = z;
+      c_row[cr] = (valid && k < p.n_cand) ? grow : -1;
+    }
+  }
+  // candidate rows beyond rt * ncp do not exist when ncp divides 128 (it does)
+  __syncthreads();
+
+  const float* H = p.Hin + (long long)unit * p.d * p.d * (p.units > 1 ? 1 : 0);
+  const double* Wt = p.Wt;
+  const int d = p.d, seg = p.seg;
+
+  // quantization error of candidate row cr at segment column a
+  auto err_at = [&](int cr, int a) -> double {
+    const long long grow = c_row[cr];
+    if (grow < 0 || a >= seg) return 0.0;
+    const double w = Wt[grow * d + seg0 + a];
+    const double s = c_s[cr], z = c_z[cr];
+    double q = rne(fma(w, c_rs[cr], z));
+    q = fmin(fmax(q, 0.0), maxq);
+    return w - s * (q - z);
+  };
+
+  double jpart[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) jpart[i] = 0.0;
+
+  for (int a0 = 0; a0 < seg; a0 += GEMM_BN) {
+    double acc[8][8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+      for (int j = 0; j < 8; ++j) acc[i][j] = 0.0;
+    auto la = [&](int mm, int k) -> double { return err_at(mm, k); };
+    auto lb = [&](int nn, int k) -> double {
+      const int a = a0 + nn;
+      return (a < seg && k < seg) ? (double)H[(long long)(seg0 + k) * d + seg0 + a] : 0.0;
+    };
+    gemm_mainloop<double, true, true>(acc, la, lb, 0, seg, smem_raw);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int cr = gemm_row_of(i);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) jpart[i] = fma(acc[i][j], err_at(cr, a0 + gemm_col_of(j)), jpart[i]);
+    }
+  }
+  // sum over the 16 threads (tx) that share the same candidate rows
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    double v = jpart[i];
+#pragma unroll
+    for (int o = 8; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    if ((tid & 15) == 0) c_J[gemm_row_of(i)] = v;
+  }
+  __syncthreads();
+
+  // Phase 3: argmin per row, strict '<' so that the lowest k wins ties.
+  if (tid < p.rt) {
+    const int r = tid;
+    const long long grow = c_row[r * p.ncp];
+    if (grow >= 0) {
+      int best = 0;
+      double bj = c_J[r * p.ncp];
+      for (int k = 1; k < p.n_cand; ++k) {
+        const double j = c_J[r * p.ncp + k];
+        if (j < bj) {
+          bj = j;
+          best = k;
+        }
+      }
+      const int cr = r * p.ncp + best;
+      const long long o = grow * p.ng + grp;
+      p.sD[o] = c_s[cr];
+      p.s_out[o] = (float)c_s[cr];
+      p.z_out[o] = (int)c_z[cr];
+      if (p.cand_out) p.cand_out[o] = (unsigned char)best;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------
+// Column sweep (Algorithm 2; Eq. 2), one launch per 128-column block `blk`.
+//
+// Panel CTAs (8 warps, one active row per warp) finish block `blk`: they apply
+// the previous block's errors to the block's columns, then walk its 128
+// columns in order -- quantize, form the normalised error, feed it back into
+// the columns to the right -- in four 32-column sub-blocks with one lane per
+// column; after a sub-block its 32 errors update the rest of the block.
+// Trailing CTAs apply the previous block's errors (a rank-128 update, rank-256
+// with the P term) to every column block right of `blk`, as GEMM tiles.  Both
+// read Err(blk-1); the panel writes Err(blk).  Stream order between launches
+// is the only synchronisation.
+// ---------------------------------------------------------------------------
+struct SweepP {
+  double* Wk;            // [M][d] working rows
+  const float* U;        // [n_hin][d][d]
+  const float* P;        // [n_hin][d][d] or nullptr
+  double* Err;           // [2][M][128] normalised errors of a block
+  double* Warr;          // [2][M][128] arrival values of a block (P term) or nullptr
+  unsigned char* codes;  // [d_out][d]
+  const double* sD;      // [d_out][ng]
+  const int* z;          // [d_out][ng]
+  tb_stats* stats;       // or nullptr
+  RowMap rm;
+  int M, d, seg, ng, maxq, blk, nblk;
+  int units, rows_per_unit;
+  int panel_ctas_per_unit, n_panel_ctas;
+  int trail_mtiles_per_unit, trail_ntiles;
+};
+
+__device__ __forceinline__ void sweep_panel(const SweepP& p, int pc, unsigned char* smem_raw) {
+  float* sU = reinterpret_cast<float*>(smem_raw);  // [128][128] diagonal block of U
+  float* sP = sU + 128 * 128;                      // [128][128] diagonal block of P (if any)
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int unit = pc / p.panel_ctas_per_unit;
+  const int rloc = (pc % p.panel_ctas_per_unit) * 8 + warp;
+  const int d = p.d, c0 = p.blk * 128;
+  const bool withP = (p.P != nullptr);
+  const float* U = p.U + (long long)unit * d * d * (p.units > 1 ? 1 : 0);
+  const float* Pm = withP ? p.P + (long long)unit * d * d * (p.units > 1 ? 1 : 0) : nullptr;
+
+  // stage the diagonal blocks (float4; rows c0+j, columns c0..c0+127)
+  for (int idx = tid; idx < 128 * 32; idx += GEMM_THREADS) {
+    const int j = idx >> 5, c4 = (idx & 31) * 4;
+    const float4 v = *reinterpret_cast<const float4*>(U + (long long)(c0 + j) * d + c0 + c4);
+    *reinterpret_cast<float4*>(sU + j * 128 + c4) = v;
+    if (withP) {
+      const float4 q = *reinterpret_cast<const float4*>(Pm + (long long)(c0 + j) * d + c0 + c4);
+      *reinterpret_cast<float4*>(sP + j * 128 + c4) = q;
+    }
+  }
+  __syncthreads();
+  if (rloc >= p.rows_per_unit) return;
+
+  const int m = unit * p.rows_per_unit + rloc;
+  const long long grow = p.rm.row(m);
+  const double maxq = (double)p.maxq;
+
+  double w[4];
+  const double* wrow = p.Wk + (long long)m * d + c0;
+#pragma unroll
+  for (int sb = 0; sb < 4; ++sb) w[sb] = wrow[sb * 32 + lane];
+
+  if (p.blk > 0) {
+    const long long eoff = ((long long)((p.blk - 1) & 1) * p.M + m) * 128;
+    const double* Ep = p.Err + eoff;
+    const float* Up = U + (long long)(c0 - 128) * d + c0 + lane;
+#pragma unroll 4
+    for (int j = 0; j < 128; ++j) {
+      const double ej = Ep[j];
+      const float* ur = Up + (long long)j * d;
+      w[0] = fma(-ej, (double)ur[0], w[0]);
+      w[1] = fma(-ej, (double)ur[32], w[1]);
+      w[2] = fma(-ej, (double)ur[64], w[2]);
+      w[3] = fma(-ej, (double)ur[96], w[3]);
+    }
+    if (withP) {
+      const double* Ap = p.Warr + eoff;
+      const float* Pp = Pm + (long long)(c0 - 128) * d + c0 + lane;
+#pragma unroll 4
+      for (int j = 0; j < 128; ++j) {
+        const double aj = Ap[j];
+        const float* pr = Pp + (long long)j * d;
+        w[0] = fma(-aj, (double)pr[0], w[0]);
+        w[1] = fma(-aj, (double)pr[32], w[1]);
+        w[2] = fma(-aj, (double)pr[64], w[2]);
+        w[3] = fma(-aj, (double)pr[96], w[3]);
+      }
+    }
+  }
+
+  unsigned int n_near = 0, n_clamp = 0;
+  const long long cur = ((long long)(p.blk & 1) * p.M + m) * 128;
+#pragma unroll
+  for (int sb = 0; sb < 4; ++sb) {
+    const int cl = sb * 32 + lane;  // column inside the block
+    const int col = c0 + cl;
+    const long long so = grow * p.ng + col / p.seg;
+    const double s_l = p.sD[so], z_l = (double)p.z[so];
+    const double rs_l = 1.0 / s_l;
+    const double rd_l = 1.0 / (double)sU[cl * 128 + cl];
+    const double srd_l = s_l * rd_l;
+    double u[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) u[j] = (double)sU[(sb * 32 + j) * 128 + cl];
+
+    double v = w[sb];
+    if (!withP) {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        // e = (v - s (q - z)) / U_jj, arranged so that the rounding is the only
+        // long dependency: e = (v + s z) / U_jj - (s / U_jj) q
+        const double ard = fma(s_l, z_l, v) * rd_l;
+        double q = rne(fma(v, rs_l, z_l));
+        q = fmin(fmax(q, 0.0), maxq);
+        const double e = fma(-srd_l, q, ard);
+        const double ej = shfl_d(e, j);
+        if (lane > j) v = fma(-ej, u[j], v);
+      }
+    } else {
+      double pu[32];
+#pragma unroll
+      for (int j = 0; j < 32; ++j) pu[j] = (double)sP[(sb * 32 + j) * 128 + cl];
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        const double ard = fma(s_l, z_l, v) * rd_l;
+        double q = rne(fma(v, rs_l, z_l));
+        q = fmin(fmax(q, 0.0), maxq);
+        const double e = fma(-srd_l, q, ard);
+        const double ej = shfl_d(e, j);
+        const double vj = shfl_d(v, j);  // value of column j on arrival
+        if (lane > j) v = fma(-vj, pu[j], fma(-ej, u[j], v));
+      }
+    }
+    // v is now this lane's value on arrival at its own column
+    const double x = fma(v, rs_l, z_l);
+    const double xr = rne(x);
+    const double q = fmin(fmax(xr, 0.0), maxq);
+    const double e_mine = fma(-srd_l, q, fma(s_l, z_l, v) * rd_l);
+    p.codes[grow * d + col] = (unsigned char)(int)q;
+    p.Err[cur + cl] = e_mine;
+    if (withP) p.Warr[cur + cl] = v;
+    {
+      const double fl = floor(x);
+      const double a0 = fmin(fmax(fl, 0.0), maxq), a1 = fmin(fmax(fl + 1.0, 0.0), maxq);
+      if (fabs(x - (fl + 0.5)) < 1e-6 && a0 != a1) ++n_near;
+      if (xr != q) ++n_clamp;
+    }
+    // the sub-block's errors update the later sub-blocks of this block
+    if (sb < 3) {
+#pragma unroll 8
+      for (int j = 0; j < 32; ++j) {
+        const double ej = shfl_d(e_mine, j);
+        const float* ur = sU + (sb * 32 + j) * 128 + lane;
+#pragma unroll
+        for (int sb2 = sb + 1; sb2 < 4; ++sb2) w[sb2] = fma(-ej, (double)ur[sb2 * 32], w[sb2]);
+        if (withP) {
+          const double vj = shfl_d(v, j);
+          const float* pr = sP + (sb * 32 + j) * 128 + lane;
+#pragma unroll
+          for (int sb2 = sb + 1; sb2 < 4; ++sb2) w[sb2] = fma(-vj, (double)pr[sb2 * 32], w[sb2]);
+        }
+      }
+    }
+  }
+  if (p.stats) {
+    n_near = __reduce_add_sync(0xffffffffu, n_near);
+    n_clamp = __reduce_add_sync(0xffffffffu, n_clamp);
+    if (lane == 0) {
+      if (n_near) atomicAdd(&p.stats->near_tie_codes, (unsigned long long)n_near);
+      if (n_clamp) atomicAdd(&p.stats->clamped_codes, (unsigned long long)n_clamp);
+      if (pc == 0 && warp == 0) atomicAdd(&p.stats->column_steps, 128ull);
+    }
+  }
+}
+
+__global__ void __launch_bounds__(GEMM_THREADS, 1) k_sweep_block(SweepP p) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int bid = blockIdx.x;
+  if (bid < p.n_panel_ctas) {
+    sweep_panel(p, bid, smem_raw);
+    return;
+  }
+  // trailing tile: Wk[:, cols] -= Err(blk-1) U[blk-1 rows, cols]  (- Warr(blk-1) P[...])
+  const int t = bid - p.n_panel_ctas;
+  const int per_unit = p.trail_mtiles_per_unit * p.trail_ntiles;
+  const int unit = t / per_unit;
+  const int mt = (t % per_unit) / p.trail_ntiles, nt = (t % per_unit) % p.trail_ntiles;
+  const int d = p.d, prev = p.blk - 1;
+  const long long uoff = (long long)unit * d * d * (p.units > 1 ? 1 : 0);
+  GemmP g;
+  g.A = p.Err + ((long long)(prev & 1) * p.M + (long long)unit * p.rows_per_unit) * 128;
+  g.a_m = 128;
+  g.a_k = 1;
+  g.B = p.U + uoff + (long long)prev * 128 * d;
+  g.b_k = d;
+  g.b_n = 1;
+  g.C = p.Wk + (long long)unit * p.rows_per_unit * d;
+  g.ldc = d;
+  g.a_batch = g.b_batch = g.c_batch = 0;
+  g.M = p.rows_per_unit;
+  g.N = d;
+  g.K = 128;
+  g.n_batch = 1;
+  g.alpha = -1.0;
+  g.beta = 1.0;
+  g.flags = 0;
+  g.btrim = g.boff = g.atrim = g.aoff = 0;
+  const int m0 = mt * GEMM_BM, n0 = (p.blk + 1 + nt) * GEMM_BN;
+  gemm_tile<double, float, double, double, false, true>(g, m0, n0, 0, smem_raw);
+  if (p.P) {
+    g.A = p.Warr + ((long long)(prev & 1) * p.M + (long long)unit * p.rows_per_unit) * 128;
+    g.B = p.P + uoff + (long long)prev * 128 * d;
+    gemm_tile<double, float, double, double, false, true>(g, m0, n0, 0, smem_raw);
+  }
+}
+
+// E[m][k] = W~[row(m)][k] - s (code - z): the quantization error of the group on
+// the weights it saw (Proposition 3.1's W_B - Q_B).
+__global__ void k_residual(const double* __restrict__ Wt, const unsigned char* __restrict__ codes,
+                           const double* __restrict__ sD, const int* __restrict__ z,
+                           double* __restrict__ E, RowMap rm, int M, int d, int seg, int ng) {
+  const long long n = (long long)M * d;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n;
+       i += (long long)gridDim.x * blockDim.x) {
+    const int m = (int)(i / d), k = (int)(i % d);
+    const long long r = rm.row(m);
+    const long long so = r * ng + k / seg;
+    const double q = (double)codes[r * d + k] - (double)z[so];
+    E[i] = Wt[r * d + k] - sD[so] * q;
+  }
+}
+
+// ---------------------------------------------------------------------------
+// Coordinate descent on the scales (Proposition 3.3 / Algorithm 3), with the
+// codes frozen.  Wbar = W_int - z.  State kept current through the pass:
+//   Dm = (Q - W) H_in + W R      [rows][d]
+// and, so that a scale step costs no product with H_in,
+//   Yw[r][g2][:] = Wbar[r, G_g2] H_in[G_g2, :]      (one row of products per scale)
+// A step on scale (j, g2) by delta adds delta * Yw[j][g2][:] to row j of Dm.
+// Rows of a head are visited in order (Gauss-Seidel); per row:
+//   k_cd_row_stats : n0[g]  = <Wbar[j,G_g], (H_out Dm)[j,G_g]>
+//                    A[g2][g] = <Yw[j][g2][G_g], Wbar[j,G_g]>   (A[g][g] is the denominator's
+//                                                                Wbar H_in[G,G] Wbar^T)
+//   k_cd_row_update: the scalar chain over the row's groups,
+//                    delta_g2 = -num_g2 / (A[g2][g2] H_out[j][j]),  num_g += H_out[j][j] delta_g2 A[g2][g],
+//                    then Dm[j,:] += sum_g2 delta_g2 Yw[j][g2][:] and s += delta.
+// ---------------------------------------------------------------------------
+__global__ void k_cd_prep(const float* __restrict__ W, const unsigned char* __restrict__ codes,
+                          const double* __restrict__ sD, const int* __restrict__ z,
+                          double* __restrict__ Dq, float* __restrict__ Wb, long long rows, int d,
+                          int seg, int ng) {
+  const long long n = rows * d;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n;
+       i += (long long)gridDim.x * blockDim.x) {
+    const long long r = i / d;
+    const int k = (int)(i % d);
+    const long long so = r * ng + k / seg;
+    const double wb = (double)codes[i] - (double)z[so];
+    if (Wb) Wb[i] = (float)wb;
+    Dq[i] = sD[so] * wb - (double)W[i];
+  }
+}
+
+struct CdP {
+  double* Dm;           // [rows][d]            (rows of this batch)
+  const double* Yw;     // [rows][ng][d]
+  const float* Wb;      // [rows][d]
+  const float* Hout;    // [heads][dh][dh] of this batch, or nullptr
+  double* sD;           // [rows][ng]
+  double* n0;           // [lines][ng]
+  double* Amat;         // [lines][ng][ng]
+  int d, seg, ng, dh, j0, lines_per_head;  // lines_per_head = 1 (row j0 of each head) or dh
+  int groups_per_cta;
+  int a_in_smem;
+};
+
+// line = head * lines_per_head + l; its row inside the head is j0 + l.
+// Partial sums are kept per 32-column chunk and added in chunk order, so the
+// result does not depend on warp scheduling.
+__global__ void __launch_bounds__(256) k_cd_row_stats(CdP p) {
+  extern __shared__ double cd_sm[];  // part[chunks][ng + 1], then hrow[dh]
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int line = blockIdx.y, head = line / p.lines_per_head, j = p.j0 + line % p.lines_per_head;
+  const int d = p.d, seg = p.seg, ng = p.ng, dh = p.dh;
+  const int g_first = blockIdx.x * p.groups_per_cta;
+  const int g_count = min(p.groups_per_cta, ng - g_first);
+  const int c_first = g_first * seg, c_count = g_count * seg;
+  const int chunks_per_group = seg / 32;
+  const int max_chunks = p.groups_per_cta * chunks_per_group;
+  const long long row = (long long)head * dh + j;
+  double* part = cd_sm;                           // [max_chunks][ng + 1]
+  double* hrow = cd_sm + (size_t)max_chunks * (ng + 1);  // [dh]
+  if (p.Hout)
+    for (int i = tid; i < dh; i += blockDim.x) hrow[i] = (double)p.Hout[((long long)head * dh + j) * dh + i];
+  __syncthreads();
+  const double* Dh = p.Dm + (long long)head * dh * d;
+  const double* Yr = p.Yw + row * ng * d;
+  const float* wbr = p.Wb + row * d;
+  // every warp walks 32 consecutive columns at a time; they lie in one group
+  for (int cb = (tid >> 5) * 32; cb < c_count; cb += (blockDim.x >> 5) * 32) {
+    const int col = c_first + cb + lane;
+    const int chunk = cb / 32;
+    const int g = g_first + cb / seg;
+    const double wb = (double)wbr[col];
+    double gj;
+    if (p.Hout) {
+      gj = 0.0;
+      for (int i = 0; i < dh; ++i) gj = fma(hrow[i], Dh[(long long)i * d + col], gj);
+    } else {
+      gj = Dh[(long long)j * d + col];
+    }
+    const double v = warp_sum(wb * gj);
+    if (lane == 0) part[chunk * (ng + 1) + ng] = v;
+    for (int g2 = 0; g2 <= g; ++g2) {
+      const double a = warp_sum(Yr[(long long)g2 * d + col] * wb);
+      if (lane == 0) part[chunk * (ng + 1) + g2] = a;
+    }
+  }
+  __syncthreads();
+  for (int i = tid; i < g_count * (ng + 1); i += blockDim.x) {
+    const int gl = i / (ng + 1), g2 = i % (ng + 1), g = g_first + gl;
+    if (g2 != ng && g2 > g) continue;
+    double t = 0.0;
+    for (int c = 0; c < chunks_per_group; ++c) t += part[(gl * chunks_per_group + c) * (ng + 1) + g2];
+    if (g2 == ng)
+      p.n0[(long long)line * ng + g] = t;
+    else
+      p.Amat[((long long)line * ng + g2) * ng + g] = t;
+  }
+}
+
+__global__ void __launch_bounds__(256) k_cd_row_update(CdP p) {
+  extern __shared__ double cd_sm[];  // num[ng], delta[ng], then A[ng][ng] if it fits
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int line = blockIdx.y, head = line / p.lines_per_head, j = p.j0 + line % p.lines_per_head;
+  const int d = p.d, seg = p.seg, ng = p.ng, dh = p.dh;
+  const long long row = (long long)head * dh + j;
+  double* num = cd_sm;
+  double* delta = cd_sm + ng;
+  const double hjj = p.Hout ? (double)p.Hout[((long long)head * dh + j) * dh + j] : 1.0;
+  const double* A = p.Amat + (long long)line * ng * ng;
+  for (int g = tid; g < ng; g += blockDim.x) num[g] = p.n0[(long long)line * ng + g];
+  if (p.a_in_smem) {
+    double* As = cd_sm + 2 * ng;
+    for (int i = tid; i < ng * ng; i += blockDim.x) {
+      const int g2 = i / ng, g = i % ng;
+      As[i] = (g >= g2) ? A[i] : 0.0;
+    }
+    A = As;
+  }
+  __syncthreads();
+  if (tid < 32) {
+    for (int g2 = 0; g2 < ng; ++g2) {
+      const double den = A[(long long)g2 * ng + g2] * hjj;
+      const double dl = (den == 0.0) ? 0.0 : -num[g2] / den;
+      if (lane == 0) delta[g2] = dl;
+      for (int g = g2 + 1 + lane; g < ng; g += 32) num[g] = fma(hjj * dl, A[(long long)g2 * ng + g], num[g]);
+      __syncwarp();
+    }
+  }
+  __syncthreads();
+  const int g_first = blockIdx.x * p.groups_per_cta;
+  const int g_count = min(p.groups_per_cta, ng - g_first);
+  const int c_first = g_first * seg, c_count = g_count * seg;
+  const double* Yr = p.Yw + row * ng * d;
+  double* dm = p.Dm + row * d;
+  for (int c = tid; c < c_count; c += blockDim.x) {
+    const int col = c_first + c;
+    double acc = dm[col];
+    for (int g2 = 0; g2 < ng; ++g2) acc = fma(delta[g2], Yr[(long long)g2 * d + col], acc);
+    dm[col] = acc;
+  }
+  if (blockIdx.x == 0)
+    for (int g = tid; g < ng; g += blockDim.x) p.sD[row * ng + g] += delta[g];
+}
+
+// Q = s (W_int - z) in float, and the scales in float (Algorithm 1, line 13).
+__global__ void k_dequant(const unsigned char* __restrict__ codes, const double* __restrict__ sD,
+                          const int* __restrict__ z, float* __restrict__ What,
+                          float* __restrict__ s_out, long long rows, int d, int seg, int ng) {
+  const long long n = rows * d;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n;
+       i += (long long)gridDim.x * blockDim.x) {
+    const long long r = i / d;
+    const int k = (int)(i % d);
+    const long long so = r * ng + k / seg;
+    if (What) What[i] = (float)(sD[so] * ((double)codes[i] - (double)z[so]));
+    if (k % seg == 0) s_out[so] = (float)sD[so];
+  }
+}
+
+// loss[h] = sum_{j,i} H_out[j][i] G2[i][j],  G2 = Z dW^T  (tr(dW H_in dW^T H_out) + cross term)
+__global__ void __launch_bounds__(256) k_loss_hout(const float* __restrict__ Hout,
+                                                   const double* __restrict__ G2,
+                                                   double* __restrict__ loss, int dh) {
+  __shared__ double part[8];
+  const int h = blockIdx.x;
+  const float* Ho = Hout + (long long)h * dh * dh;
+  const double* G = G2 + (long long)h * dh * dh;
+  double acc = 0.0;
+  for (int idx = threadIdx.x; idx < dh * dh; idx += blockDim.x) {
+    const int j = idx / dh, i = idx % dh;
+    acc = fma((double)Ho[idx], G[(long long)i * dh + j], acc);
+  }
+  acc = warp_sum(acc);
+  if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double t = 0.0;
+    for (int i = 0; i < 8; ++i) t += part[i];
+    loss[h] = t;
+  }
+}
+
+// H_out = I: loss[h] = sum over the head's rows of <Z[r,:], dW[r,:]>
+__global__ void __launch_bounds__(256) k_loss_identity(const double* __restrict__ Z,
+                                                       const double* __restrict__ Dq,
+                                                       double* __restrict__ loss,
+                                                       long long rows_per_head, int d) {
+  __shared__ double part[8];
+  const int h = blockIdx.x;
+  const long long base = (long long)h * rows_per_head * d, n = rows_per_head * d;
+  double acc = 0.0;
+  for (long long i = threadIdx.x; i < n; i += blockDim.x) acc = fma(Z[base + i], Dq[base + i], acc);
+  acc = warp_sum(acc);
+  if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double t = 0.0;
+    for (int i = 0; i < 8; ++i) t += part[i];
+    loss[h] = t;
+  }
+}
+
+// ---------------------------------------------------------------------------
+// Host side
+// ---------------------------------------------------------------------------
+struct Plan {
+  int d_out, d, H, dh, n_hin, bits, seg, ng, g, S, maxq, n_cand, ncp, rt, cd_iters;
+  bool adaptive, cd, with_r, with_loss, has_hout;
+  int Mmax;
+  long long cd_rows;  // rows per coordinate-descent batch
+  // workspace
+  double *Wt, *Wk, *W0c, *E, *Err, *Warr, *sD, *T, *Dq, *Dm, *Yw, *n0, *Amat, *G2;
+  float* Wb;
+  size_t ws_total;
+};
+
+static int pow2_ceil(int v) {
+  int p = 1;
+  while (p < v) p <<= 1;
+  return p;
+}
+
+static tb_status make_plan(const tb_layer_desc* D, bool has_hout, bool with_r, bool with_loss,
+                           void* ws, Plan* pl) {
+  if (!D) return TB_ERR_INVALID_ARG;
+  if (D->d_out <= 0 || D->d_in <= 0 || D->n_heads <= 0 || D->d_head <= 0) return TB_ERR_INVALID_ARG;
+  if ((long long)D->n_heads * D->d_head != D->d_out) return TB_ERR_INVALID_ARG;
+  if (D->d_in % 128) return TB_ERR_UNSUPPORTED;
+  if (D->n_hin != 1 && D->n_hin != D->n_heads) return TB_ERR_INVALID_ARG;
+  if (D->bits < 2 || D->bits > 8) return TB_ERR_INVALID_ARG;
+  if (D->quant_group < 0) return TB_ERR_INVALID_ARG;
+  if (D->quant_group > 0 && (D->d_in % D->quant_group)) return TB_ERR_INVALID_ARG;
+  if (D->quant_group > 0 && (D->quant_group % 32)) return TB_ERR_UNSUPPORTED;
+  if (D->out_block < 1 || D->out_block > D->d_head || (D->d_head % D->out_block)) return TB_ERR_INVALID_ARG;
+  if (D->n_cand < 1 || D->n_cand > 32) return TB_ERR_INVALID_ARG;
+  if (D->cd_iters < 0) return TB_ERR_INVALID_ARG;
+  Plan& p = *pl;
+  p.d_out = D->d_out;
+  p.d = D->d_in;
+  p.H = D->n_heads;
+  p.dh = D->d_head;
+  p.n_hin = D->n_hin;
+  p.bits = D->bits;
+  p.seg = D->quant_group > 0 ? D->quant_group : D->d_in;
+  p.ng = p.d / p.seg;
+  p.has_hout = has_hout;
+  p.g = has_hout ? D->out_block : D->d_head;  // H_out = I: all rows of a head at once
+  p.S = p.dh / p.g;
+  p.maxq = (1 << D->bits) - 1;
+  p.n_cand = D->n_cand;
+  p.ncp = pow2_ceil(D->n_cand);
+  p.rt = 128 / p.ncp;
+  p.cd_iters = D->cd_iters;
+  p.adaptive = (D->flags & TB_F_ADAPTIVE_GRID) != 0;
+  p.cd = (D->flags & TB_F_CD_REFINE) != 0 && D->cd_iters > 0;
+  p.with_r = with_r;
+  p.with_loss = with_loss;
+  p.Mmax = p.H * p.g;
+  if (p.ng > 1024) return TB_ERR_UNSUPPORTED;
+
+  Bump b(ws);
+  const size_t dd = (size_t)p.d;
+  p.Wt = b.take<double>((size_t)p.d_out * dd);
+  p.Wk = b.take<double>((size_t)p.Mmax * dd);
+  p.E = b.take<double>((size_t)p.Mmax * dd);
+  p.W0c = with_r ? b.take<double>((size_t)p.Mmax * dd) : nullptr;
+  p.Err = b.take<double>((size_t)2 * p.Mmax * 128);
+  p.Warr = with_r ? b.take<double>((size_t)2 * p.Mmax * 128) : nullptr;
+  p.sD = b.take<double>((size_t)p.d_out * p.ng);
+  p.T = (has_hout && p.S > 1) ? b.take<double>((size_t)p.H * p.S * p.dh * p.g) : nullptr;
+  p.Dq = p.Dm = p.Yw = p.n0 = p.Amat = p.G2 = nullptr;
+  p.Wb = nullptr;
+  p.cd_rows = 0;
+  if (p.cd || with_loss) {
+    p.Dq = b.take<double>((size_t)p.d_out * dd);
+    p.Dm = b.take<double>((size_t)p.d_out * dd);
+  }
+  if (p.cd) {
+    p.Wb = b.take<float>((size_t)p.d_out * dd);
+    // batch of rows whose Yw fits 4 GiB: whole heads when rows of a head are coupled
+    const size_t per_row = (size_t)p.ng * dd * sizeof(double);
+    const size_t budget = (size_t)4 << 30;
+    long long unit_rows = (has_hout || p.n_hin > 1) ? p.dh : 1;
+    long long units = (long long)(budget / (per_row * unit_rows));
+    if (units < 1) units = 1;
+    long long rows = units * unit_rows;
+    if (rows > p.d_out) rows = p.d_out;
+    if (!(has_hout || p.n_hin > 1) && rows > 128) rows = (rows / 128) * 128;
+    p.cd_rows = rows;
+    p.Yw = b.take<double>((size_t)rows * p.ng * dd);
+    const long long lines = has_hout ? rows / p.dh : rows;
+    p.n0 = b.take<double>((size_t)lines * p.ng);
+    p.Amat = b.take<double>((size_t)lines * p.ng * p.ng);
+  }
+  if (with_loss && has_hout) p.G2 = b.take<double>((size_t)p.H * p.dh * p.dh);
+  p.ws_total = b.total();
+  return TB_OK;
+}
+
+static int ew_blocks(long long n) {
+  long long b = (n + 255) / 256;
+  if (b > 148 * 16) b = 148 * 16;
+  if (b < 1) b = 1;
+  return (int)b;
+}
+
+// ---------------------------------------------------------------------------
+// Optional phase timing (tb_profile_enable / tb_profile_read): CUDA events on
+// the launching stream around each phase of tb_quantize_layer.
+// ---------------------------------------------------------------------------
+enum { PH_SETUP = 0, PH_GRID, PH_SWEEP, PH_COMP, PH_CD, PH_OUTPUT, PH_LOSS, PH_COUNT };
+struct PhaseSpan {
+  int phase;
+  cudaEvent_t a, b;
+};
+static bool g_profile_on = false;
+static PhaseSpan g_spans[4096];
+static int g_n_spans = 0;
+
+struct PhaseScope {
+  int idx;
+  cudaStream_t st;
+  PhaseScope(int phase, cudaStream_t s) : idx(-1), st(s) {
+    if (!g_profile_on || g_n_spans >= 4096) return;
+    PhaseSpan& sp = g_spans[g_n_spans];
+    if (cudaEventCreate(&sp.a) != cudaSuccess) return;
+    if (cudaEventCreate(&sp.b) != cudaSuccess) {
+      cudaEventDestroy(sp.a);
+      return;
+    }
+    sp.phase = phase;
+    idx = g_n_spans++;
+    cudaEventRecord(sp.a, st);
+  }
+  ~PhaseScope() {
+    if (idx >= 0) cudaEventRecord(g_spans[idx].b, st);
+  }
+};
+
+static tb_status run_grid(const Plan& p, const float* H_in, float* scales, int* zeros,
+                          unsigned char* cand, RowMap rm, int M, cudaStream_t st) {
+  GridP gp;
+  gp.Wt = p.Wt;
+  gp.Hin = H_in;
+  gp.sD = p.sD;
+  gp.s_out = scales;
+  gp.z_out = zeros;
+  gp.cand_out = cand;
+  gp.rm = rm;
+  gp.M = M;
+  gp.d = p.d;
+  gp.seg = p.seg;
+  gp.ng = p.ng;
+  gp.maxq = p.maxq;
+  gp.n_cand = p.n_cand;
+  gp.ncp = p.ncp;
+  gp.rt = p.rt;
+  gp.units = (p.n_hin == 1) ? 1 : p.H;
+  gp.rows_per_unit = M / gp.units;
+  gp.tiles_per_unit = (gp.rows_per_unit + p.rt - 1) / p.rt;
+  static bool configured[64] = {false};
+  TB_TRY(allow_smem(k_grid, GemmSmem<double>::bytes, configured));
+  const long long ytiles = (long long)gp.units * gp.tiles_per_unit;
+  if (ytiles > 65535) return TB_ERR_UNSUPPORTED;
+  dim3 grid(p.ng, (unsigned)ytiles);
+  k_grid<<<grid, GEMM_THREADS, GemmSmem<double>::bytes, st>>>(gp);
+  TB_LAUNCH_CHECK();
+  return TB_OK;
+}
+
+static tb_status run_sweep(const Plan& p, const float* U_in, const float* P, unsigned char* codes,
+                           const int* zeros, tb_stats* stats, RowMap rm, int M, cudaStream_t st) {
+  SweepP sp;
+  sp.Wk = p.Wk;
+  sp.U = U_in;
+  sp.P = P;
+  sp.Err = p.Err;
+  sp.Warr = p.Warr;
+  sp.codes = codes;
+  sp.sD = p.sD;
+  sp.z = zeros;
+  sp.stats = stats;
+  sp.rm = rm;
+  sp.M = M;
+  sp.d = p.d;
+  sp.seg = p.seg;
+  sp.ng = p.ng;
+  sp.maxq = p.maxq;
+  sp.nblk = p.d / 128;
+  sp.units = (p.n_hin == 1) ? 1 : p.H;
+  sp.rows_per_unit = M / sp.units;
+  sp.panel_ctas_per_unit = (sp.rows_per_unit + 7) / 8;
+  sp.n_panel_ctas = sp.panel_ctas_per_unit * sp.units;
+  sp.trail_mtiles_per_unit = (sp.rows_per_unit + GEMM_BM - 1) / GEMM_BM;
+  const size_t smem = P ? (size_t)2 * 128 * 128 * sizeof(float) : GemmSmem<double>::bytes;
+  static bool configured[64] = {false};
+  TB_TRY(allow_smem(k_sweep_block, (size_t)2 * 128 * 128 * sizeof(float), configured));
+  for (int blk = 0; blk < sp.nblk; ++blk) {
+    sp.blk = blk;
+    sp.trail_ntiles = (blk > 0) ? (sp.nblk - blk - 1) : 0;
+    const long long ctas =
+        sp.n_panel_ctas + (long long)sp.units * sp.trail_mtiles_per_unit * sp.trail_ntiles;
+    k_sweep_block<<<(unsigned)ctas, GEMM_THREADS, smem, st>>>(sp);
+    TB_LAUNCH_CHECK();
+  }
+  return TB_OK;
+}
+
+}  // namespace tb
+
+using namespace tb;
+
+extern "C" size_t tb_quantize_layer_workspace(const tb_layer_desc* desc, int with_r, int with_loss) {
+  Plan p;
+  // the larger of the two H_out cases, so that one query serves both
+  size_t a = 0, b = 0;
+  if (make_plan(desc, true, with_r != 0, with_loss != 0, nullptr, &p) == TB_OK) a = p.ws_total;
+  if (make_plan(desc, false, with_r != 0, with_loss != 0, nullptr, &p) == TB_OK) b = p.ws_total;
+  return a > b ? a : b;
+}
+
+extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W, const float* H_in,
+                                       const float* U_in, const float* H_out, const float* U_out,
+                                       const float* R, const float* P, const float* C,
+                                       unsigned char* codes, float* scales, int* zeros,
+                                       unsigned char* cand, float* W_hat, double* loss,
+                                       tb_stats* stats, void* ws, size_t ws_bytes, void* stream) {
+  if (!desc || !W || !H_in || !U_in || !codes || !scales || !zeros) return TB_ERR_INVALID_ARG;
+  if ((H_out == nullptr) != (U_out == nullptr)) return TB_ERR_INVALID_ARG;
+  const bool with_r = (R != nullptr);
+  if (with_r != (P != nullptr) || with_r != (C != nullptr)) return TB_ERR_INVALID_ARG;
+  if (!aligned(W, 16) || !aligned(H_in, 16) || !aligned(U_in, 16) || (P && !aligned(P, 16)))
+    return TB_ERR_INVALID_ARG;
+  Plan p;
+  TB_TRY(make_plan(desc, H_out != nullptr, with_r, loss != nullptr, nullptr, &p));
+  if (!ws || !aligned(ws, 256) || ws_bytes < p.ws_total) return TB_ERR_WORKSPACE;
+  TB_TRY(make_plan(desc, H_out != nullptr, with_r, loss != nullptr, ws, &p));
+  cudaStream_t st = as_stream(stream);
+  const int d = p.d;
+  const long long n_all = (long long)p.d_out * d;
+  const long long dd = (long long)d * d;
+
+  if (stats) TB_CUDA_CHECK(cudaMemsetAsync(stats, 0, sizeof(tb_stats), st));
+  k_widen<<<ew_blocks(n_all), 256, 0, st>>>(W, p.Wt, n_all);
+  TB_LAUNCH_CHECK();
+  if (p.T) {
+    k_comp_matrices<<<dim3(p.S, p.H), 128, 0, st>>>(U_out, p.T, p.dh, p.g, p.S);
+    TB_LAUNCH_CHECK();
+  }
+  if (!p.adaptive) {
+    // fixed grid: every row, once, from the original weights
+    RowMap all{p.dh, p.dh, 0};
+    TB_TRY(run_grid(p, H_in, scales, zeros, cand, all, p.d_out, st));
+  }
+
+  for (int step = 0; step < p.S; ++step) {
+    const int i0 = step * p.g, M = p.H * p.g;
+    RowMap rm{p.g, p.dh, i0};
+    if (p.adaptive) TB_TRY(run_grid(p, H_in, scales, zeros, cand, rm, M, st));
+    k_gather<<<ew_blocks((long long)M * d), 256, 0, st>>>(p.Wt, p.Wk, p.W0c, rm, M, d);
+    TB_LAUNCH_CHECK();
+    TB_TRY(run_sweep(p, U_in, P, codes, zeros, stats, rm, M, st));
+    const int nrem = p.dh - i0 - p.g;
+    if (!p.has_hout || nrem <= 0) continue;
+    k_residual<<<ew_blocks((long long)M * d), 256, 0, st>>>(p.Wt, codes, p.sD, zeros, p.E, rm, M, d,
+                                                            p.seg, p.ng);
+    TB_LAUNCH_CHECK();
+    if (with_r) {
+      // E <- E - W0 (R H_in^{-1})   (Proposition 3.2)
+      GemmP g = gemm_params();
+      const int units = (p.n_hin == 1) ? 1 : p.H;
+      g.A = p.W0c;
+      g.a_m = d;
+      g.a_k = 1;
+      g.B = C;
+      g.b_k = d;
+      g.b_n = 1;
+      g.C = p.E;
+      g.ldc = d;
+      g.M = M / units;
+      g.N = d;
+      g.K = d;
+      g.n_batch = units;
+      g.a_batch = (long long)g.M * d;
+      g.c_batch = (long long)g.M * d;
+      g.b_batch = (units > 1) ? dd : 0;
+      g.alpha = -1.0;
+      g.beta = 1.0;
+      TB_TRY((gemm_launch<double, float, double, double, false, true>(g, st)));
+    }
+    {
+      // W~[rem rows of every head] -= T_i E   (Propositions 3.1 / 3.2; Algorithm 1 line 11)
+      GemmP g = gemm_params();
+      g.A = p.T + (long long)step * p.dh * p.g;
+      g.a_m = p.g;
+      g.a_k = 1;
+      g.a_batch = (long long)p.S * p.dh * p.g;
+      g.B = p.E;
+      g.b_k = d;
+      g.b_n = 1;
+      g.b_batch = (long long)p.g * d;
+      g.C = p.Wt + (long long)(i0 + p.g) * d;
+      g.ldc = d;
+      g.c_batch = (long long)p.dh * d;
+      g.M = nrem;
+      g.N = d;
+      g.K = p.g;
+      g.n_batch = p.H;
+      g.alpha = -1.0;
+      g.beta = 1.0;
+      TB_TRY((gemm_launch<double, double, double, double, false, true>(g, st)));
+    }
+  }
+
+  // ---- coordinate descent on the scales (Algorithm 3) ----
+  if (p.cd) {
+    const int units = (p.n_hin == 1) ? 1 : p.H;
+    k_cd_prep<<<ew_blocks(n_all), 256, 0, st>>>(W, codes, p.sD, zeros, p.Dq, p.Wb, p.d_out, d, p.seg,
+                                               p.ng);
+    TB_LAUNCH_CHECK();
+    for (long long r0 = 0; r0 < p.d_out; r0 += p.cd_rows) {
+      const long long rows = (p.d_out - r0 < p.cd_rows) ? (p.d_out - r0) : p.cd_rows;
+      // Dm = (Q - W) H_in (+ W R); Yw = blockwise Wbar H_in.  With one H_in per head the
+      // batch is whole heads and the products run head by head.
+      const long long rows_per_prod = (units > 1) ? p.dh : rows;
+      for (long long q0 = 0; q0 < rows; q0 += rows_per_prod) {
+        const long long rr = r0 + q0;
+        const float* Hh = H_in + ((units > 1) ? (rr / p.dh) * dd : 0);
+        GemmP g = gemm_params();
+        g.A = p.Dq + rr * d;
+        g.a_m = d;
+        g.a_k = 1;
+        g.B = Hh;
+        g.b_k = d;
+        g.b_n = 1;
+        g.C = p.Dm + rr * d;
+        g.ldc = d;
+        g.M = (int)rows_per_prod;
+        g.N = d;
+        g.K = d;
+        TB_TRY((gemm_launch<double, float, double, double, false, true>(g, st)));
+        if (with_r) {
+          GemmP h = g;
+          h.A = W + rr * d;
+          h.B = R + ((units > 1) ? (rr / p.dh) * dd : 0);
+          h.beta = 1.0;
+          TB_TRY((gemm_launch<float, float, double, double, false, true>(h, st)));
+        }
+        GemmP y = gemm_params();
+        y.A = p.Wb + rr * d;
+        y.a_m = d;
+        y.a_k = 1;
+        y.a_batch = p.seg;
+        y.B = Hh;
+        y.b_k = d;
+        y.b_n = 1;
+        y.b_batch = (long long)p.seg * d;
+        y.C = p.Yw + q0 * p.ng * d;
+        y.ldc = (long long)p.ng * d;
+        y.c_batch = d;
+        y.M = (int)rows_per_prod;
+        y.N = d;
+        y.K = p.seg;
+        y.n_batch = p.ng;
+        TB_TRY((gemm_launch<float, float, double, double, false, true>(y, st)));
+      }
+      CdP cp;
+      cp.Dm = p.Dm + r0 * d;
+      cp.Yw = p.Yw;
+      cp.Wb = p.Wb + r0 * d;
+      cp.sD = p.sD + r0 * p.ng;
+      cp.n0 = p.n0;
+      cp.Amat = p.Amat;
+      cp.d = d;
+      cp.seg = p.seg;
+      cp.ng = p.ng;
+      int lines, n_j;
+      if (p.has_hout) {
+        cp.Hout = H_out + (r0 / p.dh) * (long long)p.dh * p.dh;
+        cp.dh = p.dh;
+        cp.lines_per_head = 1;
+        lines = (int)(rows / p.dh);
+        n_j = p.dh;
+      } else {
+        // rows are independent: every row is its own "head" of one row
+        cp.Hout = nullptr;
+        cp.dh = 1;
+        cp.lines_per_head = 1;
+        lines = (int)rows;
+        n_j = 1;
+      }
+      // columns per CTA: whole groups, about 512 columns
+      int gpc = 512 / p.seg;
+      if (gpc < 1) gpc = 1;
+      if (gpc > p.ng) gpc = p.ng;
+      cp.groups_per_cta = gpc;
+      const int xctas = (p.ng + gpc - 1) / gpc;
+      const size_t sm_stats =
+          ((size_t)gpc * (p.seg / 32) * (p.ng + 1) + cp.dh) * sizeof(double);
+      size_t sm_upd = ((size_t)2 * p.ng + (size_t)p.ng * p.ng) * sizeof(double);
+      cp.a_in_smem = 1;
+      if (sm_upd > 200 * 1024) {
+        sm_upd = (size_t)2 * p.ng * sizeof(double);
+        cp.a_in_smem = 0;
+      }
+      static bool conf_stats[64] = {false}, conf_upd[64] = {false};
+      TB_TRY(allow_smem(k_cd_row_stats, 200 * 1024, conf_stats));
+      TB_TRY(allow_smem(k_cd_row_update, 200 * 1024, conf_upd));
+      if (sm_stats > 200 * 1024) return TB_ERR_UNSUPPORTED;
+      for (int it = 0; it < p.cd_iters; ++it) {
+        for (int j = 0; j < n_j; ++j) {
+          cp.j0 = j;
+          for (int l0 = 0; l0 < lines; l0 += 65535) {
+            const int nl = (lines - l0 < 65535) ? (lines - l0) : 65535;
+            CdP cq = cp;
+            // advance every per-line pointer by l0 lines (a line is one head, or one row)
+            const long long rows_per_line = cp.dh;
+            cq.Dm = cp.Dm + (long long)l0 * rows_per_line * d;
+            cq.Yw = cp.Yw + (long long)l0 * rows_per_line * p.ng * d;
+            cq.Wb = cp.Wb + (long long)l0 * rows_per_line * d;
+            cq.sD = cp.sD + (long long)l0 * rows_per_line * p.ng;
+            cq.n0 = cp.n0 + (long long)l0 * p.ng;
+            cq.Amat = cp.Amat + (long long)l0 * p.ng * p.ng;
+            if (cp.Hout) cq.Hout = cp.Hout + (long long)l0 * p.dh * p.dh;
+            k_cd_row_stats<<<dim3(xctas, nl), 256, sm_stats, st>>>(cq);
+            TB_LAUNCH_CHECK();
+            k_cd_row_update<<<dim3(xctas, nl), 256, sm_upd, st>>>(cq);
+            TB_LAUNCH_CHECK();
+          }
+        }
+      }
+    }
+  }
+
+  k_dequant<<<ew_blocks(n_all), 256, 0, st>>>(codes, p.sD, zeros, W_hat, scales, p.d_out, d, p.seg,
+                                             p.ng);
+  TB_LAUNCH_CHECK();
+
+  // ---- loss of the proofs of Propositions 3.1 / 3.2 ----
+  if (loss) {
+    const int units = (p.n_hin == 1) ? 1 : p.H;
+    k_cd_prep<<<ew_blocks(n_all), 256, 0, st>>>(W, codes, p.sD, zeros, p.Dq, nullptr, p.d_out, d,
+                                               p.seg, p.ng);
+    TB_LAUNCH_CHECK();
+    GemmP g = gemm_params();
+    g.A = p.Dq;
+    g.a_m = d;
+    g.a_k = 1;
+    g.B = H_in;
+    g.b_k = d;
+    g.b_n = 1;
+    g.C = p.Dm;
+    g.ldc = d;
+    g.M = p.d_out / units;
+    g.N = d;
+    g.K = d;
+    g.n_batch = units;
+    g.a_batch = g.c_batch = (long long)g.M * d;
+    g.b_batch = (units > 1) ? dd : 0;
+    TB_TRY((gemm_launch<double, float, double, double, false, true>(g, st)));
+    if (with_r) {
+      GemmP h = g;
+      h.A = W;
+      h.B = R;
+      h.alpha = 2.0;
+      h.beta = 1.0;
+      TB_TRY((gemm_launch<float, float, double, double, false, true>(h, st)));
+    }
+    if (p.has_hout) {
+      GemmP q = gemm_params();
+      q.A = p.Dm;  // Z
+      q.a_m = d;
+      q.a_k = 1;
+      q.a_batch = (long long)p.dh * d;
+      q.B = p.Dq;  // B(k, n) = dW[n][k]
+      q.b_k = 1;
+      q.b_n = d;
+      q.b_batch = (long long)p.dh * d;
+      q.C = p.G2;
+      q.ldc = p.dh;
+      q.c_batch = (long long)p.dh * p.dh;
+      q.M = p.dh;
+      q.N = p.dh;
+      q.K = d;
+      q.n_batch = p.H;
+      TB_TRY((gemm_launch<double, double, double, double, false, false>(q, st)));
+      k_loss_hout<<<p.H, 256, 0, st>>>(H_out, p.G2, loss, p.dh);
+    } else {
+      k_loss_identity<<<p.H, 256, 0, st>>>(p.Dm, p.Dq, loss, p.dh, d);
+    }
+    TB_LAUNCH_CHECK();
+  }
+  return TB_OK;
+}

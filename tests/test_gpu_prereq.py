@@ -1,0 +1,136 @@
+"""GPU parity of the prerequisites of the quantizer against the float64 oracle:
+Hessian accumulation and finalisation, H_out construction, the inverse Cholesky
+factor and the propagated-error operands.  All calls go through the C ABI."""
+import numpy as np
+import pytest
+
+import oracle
+import tb_inputs
+from parity_util import f32, rel_fro
+
+pytestmark = pytest.mark.gpu
+
+
+def _t(a, dtype=None):
+    import torch
+    t = torch.from_numpy(np.ascontiguousarray(a)).to("cuda:0")
+    return t if dtype is None else t.to(dtype)
+
+
+@pytest.mark.parametrize("n_tok,d,bf16", [(5000, 264, True), (4096, 256, False), (9000, 384, True)])
+def test_hessian_accumulation(n_tok, d, bf16):
+    """H = X^T X / n + damping (Table 1) over several launches with a ragged last
+    chunk and a width that is not a multiple of the tile.  Tolerance: products of
+    bf16 inputs are exact in float; each 4096-token launch adds ~sqrt(4096) * 2^-24
+    relative rounding and the running sum one more rounding per launch, far below 1e-5."""
+    import torch
+    import paper_2602_04929_b200 as tb
+    rec = tb_inputs.HeavyTailRecipe(d, seed=3)
+    X = rec.chunk(0, n_tok, bf16=bf16)
+    H = torch.zeros((d, d), dtype=torch.float32, device="cuda:0")
+    Xd = _t(X, torch.bfloat16 if bf16 else None)
+    half = (n_tok // 2 // 8) * 8
+    tb.tb_accumulate_hessian(H, Xd[:half].contiguous())      # running sum over two calls
+    tb.tb_accumulate_hessian(H, Xd[half:].contiguous())
+    Hsum = torch.empty_like(H)
+    tb.tb_finalize_hessian(H, None, n_tok, 0.01, Hsum_out=Hsum)
+    torch.cuda.synchronize()
+    Ho, Hso = oracle.hessian(X, damp=0.01, return_sum=True)
+    Hg = H.cpu().numpy()
+    assert rel_fro(Hg, Ho) <= 1e-5
+    assert rel_fro(Hsum.cpu().numpy(), Hso) <= 1e-5
+    assert np.array_equal(Hg, Hg.T)
+    scale = np.sqrt(np.outer(np.diag(Ho), np.diag(Ho)))
+    assert np.max(np.abs(Hg - Ho) / scale) <= 1e-5
+
+
+@pytest.mark.parametrize("bf16", [True, False])
+def test_cross_correlation(bf16):
+    """R = alpha (X - Xfp) X^T / n (Algorithm 1, line 5), not symmetric."""
+    import torch
+    import paper_2602_04929_b200 as tb
+    d, n_tok, alpha = 264, 6000, 0.25
+    rec = tb_inputs.DeviationRecipe(tb_inputs.HeavyTailRecipe(d, seed=5))
+    X, Xfp = rec.chunk(0, n_tok, bf16=bf16)
+    if bf16:
+        Xfp = tb_inputs.bf16_bits_to_f32(tb_inputs.to_bf16_bits(Xfp))
+    dt = torch.bfloat16 if bf16 else None
+    R = torch.zeros((d, d), dtype=torch.float32, device="cuda:0")
+    H = torch.zeros((d, d), dtype=torch.float32, device="cuda:0")
+    tb.tb_accumulate_cross(R, _t(X, dt), _t(Xfp, dt), alpha)
+    tb.tb_accumulate_hessian(H, _t(X, dt))
+    tb.tb_finalize_hessian(H, R, n_tok, 0.0)
+    torch.cuda.synchronize()
+    Ro = oracle.cross_correlation(X, Xfp, alpha)
+    assert rel_fro(R.cpu().numpy(), Ro) <= 1e-5
+
+
+@pytest.mark.parametrize("n_heads,g_heads,with_sum", [(4, 4, True), (2, 8, True), (8, 2, True), (4, 4, False)])
+def test_build_hout(n_heads, g_heads, with_sum):
+    """Table 1: H_out,h = G_h Hsum G_h^T (query / key side, also grouped-query
+    attention in both directions) or G_h G_h^T (value side)."""
+    import torch
+    import paper_2602_04929_b200 as tb
+    d, dh = 256, 64
+    X = tb_inputs.HeavyTailRecipe(d, seed=7).chunk(0, 2048)
+    _, Hs = oracle.hessian(X, return_sum=True)
+    Hs32 = f32(Hs)
+    G = tb_inputs.weight(7, g_heads * dh, d, tid=tb_inputs.T_WPARTNER)
+    Hout = tb.tb_build_hout(_t(G), _t(Hs32) if with_sum else None, n_heads, dh, 0.01)
+    torch.cuda.synchronize()
+    ref = oracle.hout_from_projection(G, Hs32 if with_sum else None, n_heads, dh, damp=0.01)
+    assert rel_fro(Hout.cpu().numpy(), ref) <= 1e-6
+
+
+@pytest.mark.parametrize("n_batch,d,cond", [(3, 200, 1e3), (1, 256, 1e5), (2, 64, 1e2), (1, 520, 1e4), (5, 128, 1e3)])
+def test_factor_matches_definition(n_batch, d, cond):
+    """U = chol(H^-1)^T (Eq. 2).  The GPU takes the reversed-Cholesky route in
+    double and rounds once to float; the oracle inverts and factors."""
+    import torch
+    import paper_2602_04929_b200 as tb
+    H = np.stack([tb_inputs.spd_matrix(11 + b, d, cond=cond) for b in range(n_batch)])
+    U, info, Hinv = tb.tb_factor(_t(H), want_inverse=True)
+    torch.cuda.synchronize()
+    assert info.cpu().tolist() == [0] * n_batch
+    Ug, Uo = U.cpu().numpy().astype(np.float64), oracle.factor_upper(H)
+    assert np.all(np.tril(Ug, -1) == 0.0)
+    assert np.all(np.diagonal(Ug, axis1=1, axis2=2) > 0)
+    for b in range(n_batch):
+        assert rel_fro(Ug[b], Uo[b]) <= 1e-6
+        I = Ug[b] @ H[b].astype(np.float64) @ Ug[b].T
+        assert np.max(np.abs(I - np.eye(d))) <= 1e-6 * cond ** 0.5 + 1e-5
+        assert rel_fro(Hinv.cpu().numpy()[b], np.linalg.inv(H[b].astype(np.float64))) <= 1e-5
+
+
+def test_factor_reports_a_non_positive_pivot():
+    """A matrix that is not positive definite yields a device-side info word, no fault."""
+    import torch
+    import paper_2602_04929_b200 as tb
+    H = np.stack([tb_inputs.spd_matrix(1, 96), -np.eye(96, dtype=np.float32), tb_inputs.spd_matrix(2, 96)])
+    H[2, 95, 95] = -1.0   # last row is eliminated first
+    U, info = tb.tb_factor(_t(H))
+    torch.cuda.synchronize()
+    info = info.cpu().tolist()
+    assert info[0] == 0 and info[1] == 1 and info[2] == 1
+
+
+@pytest.mark.parametrize("n_batch,d", [(1, 256), (2, 200)])
+def test_prepare_correction(n_batch, d):
+    """P = ((R U^T) masked strictly upper) U (Algorithm 2, line 2); C = R U^T U (Proposition 3.2)."""
+    import torch
+    import paper_2602_04929_b200 as tb
+    Rs, Us = [], []
+    for b in range(n_batch):
+        rec = tb_inputs.DeviationRecipe(tb_inputs.HeavyTailRecipe(d, seed=20 + b))
+        X, Xfp = rec.chunk(0, 2048)
+        H32 = f32(oracle.hessian(X, damp=0.01))
+        Us.append(f32(oracle.factor_upper(H32)))
+        Rs.append(f32(oracle.cross_correlation(X, Xfp, 0.25)))
+    R, U = np.stack(Rs), np.stack(Us)
+    P, C = tb.tb_prepare_correction(_t(R), _t(U))
+    torch.cuda.synchronize()
+    Po, Co = oracle.correction_operands(R, U)
+    Pg = P.cpu().numpy()
+    assert np.all(np.tril(Pg) == 0.0)
+    assert rel_fro(Pg, Po) <= 1e-5
+    assert rel_fro(C.cpu().numpy(), Co) <= 1e-5
