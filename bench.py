@@ -1,0 +1,415 @@
+#!/usr/bin/env python
+"""Benchmark of the TurboBoA quantizer path on B200.
+
+One "step" quantizes one projection from its calibration activations: Hessian
+accumulation and finalisation, H_out construction, both inverse Cholesky
+factors, then the out-channel-group loop, the scale refinement and the loss.
+The default workload is the Llama-2-7B-shaped q_proj (W 4096 x 4096, 128 x 2048
+synthetic heavy-tailed tokens in bf16, 32 heads x 128, INT2, column groups of
+128, out-block 32, adaptive grid + coordinate descent).
+
+    python bench.py --gpus 1 --steps 5 --warmup 3
+    python -m torch.distributed.run --nproc-per-node N ... bench.py --gpus N ...
+    python bench.py --impl reference        # the float64 CPU oracle on the host cores
+
+Prints ONE JSON line on rank 0.  With N > 1 every rank quantizes its own layer
+(independent problems, no collective on the data path): weak scaling.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import tb_inputs  # noqa: E402
+
+METRIC = "out_channels_quantized_per_s"
+UNIT = "out-channels/s"
+DAMP = 0.01
+FLAGS_ADAPT, FLAGS_CD = 1, 2
+# FP64 FMA peak of the CUDA cores: 148 SMs x 64 FP64 lanes x 2 flop x 1.965 GHz (TFLOP/s)
+FP64_ALU_PEAK_TFLOPS = 148 * 64 * 2 * 1.965e9 / 1e12
+# FP32 FMA peak: 148 SMs x 128 lanes x 2 x 1.965 GHz
+FP32_ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
+
+
+def workload(name: str):
+    cfg = tb_inputs.CONFIGS[name]
+    proj = cfg.projections[0]
+    return cfg, proj
+
+
+def gen_inputs(cfg, proj, seed: int, n_tok: int):
+    """Host-side synthetic inputs: W, partner projection G (W_K), X as bf16 bit patterns."""
+    W = tb_inputs.weight(seed, proj.d_out, proj.d_in)
+    G = tb_inputs.weight(seed, proj.d_out, proj.d_in, tid=tb_inputs.T_WPARTNER) if proj.partner else None
+    rec = tb_inputs.HeavyTailRecipe(proj.d_in, seed=seed)
+    Xb = np.empty((n_tok, proj.d_in), np.uint16)
+    step = 4096
+    for t0 in range(0, n_tok, step):
+        n = min(step, n_tok - t0)
+        Xb[t0:t0 + n] = tb_inputs.to_bf16_bits(rec.chunk(t0, n, bf16=False))
+    return W, G, Xb
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons, sampled while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def count_launches(cfg, proj, n_tok: int, with_loss=True) -> int:
+    """Kernel launches of one step, counted from the launch loops of the library."""
+    d, dh, H = proj.d_in, proj.d_head, proj.n_heads
+    g = cfg.out_block if proj.partner else dh
+    S = dh // g
+    nblk = d // 128
+    n = 0
+    n += -(-n_tok // 4096) + 1 + 2                      # accumulate launches, mirror, finalize (2)
+    if proj.partner:
+        n += 3                                          # G Hsum, per-head Gram, combine
+    for (dd, nb) in ((d, 1),) + (((dh, H),) if proj.partner else ()):
+        blocks = -(-dd // 64)
+        n += 1 + blocks + 3 * (blocks - 1) + 2 * (blocks - 1) + 1   # reverse, potrf, panel ops, inverse, reverse
+    n += 1 + (1 if S > 1 else 0)                        # widen, compensation matrices
+    n += (S if cfg.adaptive else 1)                     # grid
+    n += S * (1 + nblk)                                 # gather + one launch per column block
+    n += (S - 1) * 2 if proj.partner else 0             # residual + compensation GEMM
+    if cfg.cd:
+        n += 1 + 2 + 2 * (dh if proj.partner else 1)    # prep, Dm and Yw products, two kernels per row step
+    n += 1                                              # dequant
+    if with_loss:
+        n += 2 + (2 if proj.partner else 1)
+    return n
+
+
+def run_reference(args, cfg, proj, rank, world):
+    """The float64 CPU oracle, as it stands, on a bounded sample: one head of the workload
+    per step (heads are independent).  Rank 0 only."""
+    if rank != 0:
+        return
+    import oracle
+    d, dh = proj.d_in, proj.d_head
+    n_tok = 4096
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    import parity_util as pu
+    prob = pu.make_problem(0, d, 1, dh, n_tok, hout="proj" if proj.partner else None)
+    flags = (FLAGS_ADAPT if cfg.adaptive else 0) | (FLAGS_CD if cfg.cd else 0)
+    od = pu.oracle_desc(prob, cfg.bits, cfg.quant_group, cfg.out_block, flags)
+
+    def step():
+        oracle.quantize_layer(od, prob["W"], prob["Hin"][0], prob["Uin"][0], prob["Hout"], prob["Uout"])
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / max(args.steps, 1)
+    value = dh / dt
+    cores = oracle.num_threads()
+    sample = (f"group loop + scale refinement of 1 head ({dh} out-channels) of the {proj.d_out}x{d} layer per "
+              f"step; Hessian ({n_tok} tokens) and factors computed once outside the timed steps")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": cfg.name, "d_out": proj.d_out, "d_in": d, "bits": cfg.bits,
+                       "quant_group": cfg.quant_group, "out_block": cfg.out_block},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def cpu_baseline(cfg, proj, budget_s: float = 20.0):
+    """Oracle timed on the host cores on a bounded sample of the same workload."""
+    import oracle
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    import parity_util as pu
+    d, dh = proj.d_in, proj.d_head
+    prob = pu.make_problem(0, d, 1, dh, 4096, hout="proj" if proj.partner else None)
+    flags = (FLAGS_ADAPT if cfg.adaptive else 0) | (FLAGS_CD if cfg.cd else 0)
+    od = pu.oracle_desc(prob, cfg.bits, cfg.quant_group, cfg.out_block, flags)
+    t0 = time.perf_counter()
+    oracle.quantize_layer(od, prob["W"], prob["Hin"][0], prob["Uin"][0], prob["Hout"], prob["Uout"])
+    dt = time.perf_counter() - t0
+    return {"value": dh / dt, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"group loop + scale refinement of 1 of {proj.n_heads} heads ({dh} out-channels), "
+                      f"{dt:.1f} s; Hessian accumulation and factorisation not included"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="l2_7b_q")
+    ap.add_argument("--tokens", type=int, default=0, help="override the token count (default: the config's)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    cfg, proj = workload(args.workload)
+    if args.impl == "reference":
+        run_reference(args, cfg, proj, rank, world)
+        return
+
+    import torch
+    import paper_2602_04929_b200 as tb
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the quantizer has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    tb.load()
+
+    n_tok = args.tokens or cfg.n_tok
+    d, d_out, H, dh = proj.d_in, proj.d_out, proj.n_heads, proj.d_head
+    flags = (FLAGS_ADAPT if cfg.adaptive else 0) | (FLAGS_CD if cfg.cd else 0)
+    desc = tb.layer_desc(d_out, d, H, dh, cfg.bits, cfg.quant_group, cfg.out_block, flags=flags)
+    ng = desc.n_groups
+
+    W_h, G_h, Xb_h = gen_inputs(cfg, proj, seed=rank, n_tok=n_tok)
+    W = torch.from_numpy(W_h).to(dev)
+    G = torch.from_numpy(G_h).to(dev) if G_h is not None else None
+    X = torch.from_numpy(Xb_h.view(np.int16)).to(dev).view(torch.bfloat16)
+    g_heads = H if G is not None else 0
+
+    lib = tb.load()
+    Hin = torch.empty((d, d), dtype=torch.float32, device=dev)
+    Hsum = torch.empty_like(Hin)
+    out = tb.QuantizeResult(
+        codes=torch.empty((d_out, d), dtype=torch.uint8, device=dev),
+        scales=torch.empty((d_out, ng), dtype=torch.float32, device=dev),
+        zeros=torch.empty((d_out, ng), dtype=torch.int32, device=dev),
+        cand=torch.empty((d_out, ng), dtype=torch.uint8, device=dev),
+        w_hat=torch.empty((d_out, d), dtype=torch.float32, device=dev),
+        loss=torch.empty(H, dtype=torch.float64, device=dev),
+        stats=torch.zeros(8, dtype=torch.int64, device=dev))
+    ws = torch.empty(tb.tb_quantize_layer_workspace(desc, False, True), dtype=torch.uint8, device=dev)
+
+    phases = {}
+
+    def ev():
+        e = torch.cuda.Event(enable_timing=True)
+        e.record()
+        return e
+
+    def step(record=None):
+        marks = [("start", ev())] if record is not None else None
+        Hin.zero_()
+        tb.tb_accumulate_hessian(Hin, X)
+        tb.tb_finalize_hessian(Hin, None, n_tok, DAMP, Hsum_out=Hsum)
+        if marks is not None:
+            marks.append(("hessian", ev()))
+        Hout = Uout = None
+        if G is not None:
+            Hout = tb.tb_build_hout(G, Hsum, H, dh, DAMP)
+            if marks is not None:
+                marks.append(("hout", ev()))
+        Uin, info_in = tb.tb_factor(Hin)
+        if G is not None:
+            Uout, info_out = tb.tb_factor(Hout)
+        if marks is not None:
+            marks.append(("factor", ev()))
+        tb.tb_quantize_layer(desc, W, Hin, Uin, Hout, Uout, ws=ws, out=out)
+        if marks is not None:
+            marks.append(("quantize", ev()))
+            record.append(marks)
+        return info_in
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+
+    for _ in range(args.warmup):
+        info = step()
+    torch.cuda.synchronize()
+    assert int(info.max().item()) == 0, "H_in was not positive definite"
+
+    sampler = ClockSampler(local_rank)
+    tb.tb_profile_enable(True)
+    rec = []
+    barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    e0 = ev()
+    for _ in range(args.steps):
+        step(rec)
+    e1 = ev()
+    torch.cuda.synchronize()
+    barrier()
+    clocks = sampler.stop()
+    total_ms = e0.elapsed_time(e1)
+    q_ms = tb.tb_profile_read()
+    tb.tb_profile_enable(False)
+    for marks in rec:
+        for (_, a), (nm, b) in zip(marks[:-1], marks[1:]):
+            phases[nm] = phases.get(nm, 0.0) + a.elapsed_time(b)
+    K = max(args.steps, 1)
+    phases = {k: v / K for k, v in phases.items()}
+    q_ms = {k: v / K for k, v in q_ms.items()}
+    ms_per_step = total_ms / K
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([ms_per_step], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_per_step = float(t.item())
+
+    # ---- end to end from pinned host buffers through the C ABI ----
+    e2e = None
+    if not args.no_e2e:
+        Wp = torch.from_numpy(W_h).pin_memory()
+        Xp = torch.from_numpy(Xb_h.view(np.int16)).pin_memory()
+        Gp = torch.from_numpy(G_h).pin_memory() if G_h is not None else None
+        outs = {"codes": torch.empty((d_out, d), dtype=torch.uint8).pin_memory(),
+                "scales": torch.empty((d_out, ng), dtype=torch.float32).pin_memory(),
+                "zeros": torch.empty((d_out, ng), dtype=torch.int32).pin_memory(),
+                "w_hat": torch.empty((d_out, d), dtype=torch.float32).pin_memory(),
+                "loss": torch.empty(H, dtype=torch.float64).pin_memory()}
+        hws = torch.empty(tb.tb_quantize_from_host_workspace(desc, n_tok, g_heads), dtype=torch.uint8, device=dev)
+        tb.tb_quantize_from_host(desc, Wp, Xp, Gp, DAMP, DAMP, outs, hws)  # warm-up
+        n_e2e = min(K, 3)
+        barrier()
+        torch.cuda.synchronize()
+        a = ev()
+        for _ in range(n_e2e):
+            tb.tb_quantize_from_host(desc, Wp, Xp, Gp, DAMP, DAMP, outs, hws)
+        b = ev()
+        torch.cuda.synchronize()
+        e2e_ms = a.elapsed_time(b) / n_e2e
+        if world > 1:
+            import torch.distributed as dist
+            t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        h2d = Wp.numel() * 4 + Xp.numel() * 2 + (Gp.numel() * 4 if Gp is not None else 0)
+        d2h = sum(v.numel() * v.element_size() for v in outs.values())
+        e2e = {"value": d_out * world / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms, "steps": n_e2e,
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)}
+        assert np.array_equal(outs["codes"].numpy(), out.codes.cpu().numpy()), "host and device paths disagree"
+
+    if rank != 0:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+        return
+
+    # ---- rooflines (algorithmic work / measured phase time) ----
+    S = dh // (cfg.out_block if G is not None else dh)
+    seg = cfg.quant_group or d
+    fl = {
+        "hessian": 2.0 * n_tok * d * d,                           # X^T X (the symmetric half is skipped)
+        "sweep": 1.0 * d_out * d * d,                             # d_in^2 flop per out-channel
+        "grid": 2.0 * 16 * d_out * d * seg * (1 if cfg.adaptive else 1),
+        "cd": (4.0 * d_out * d * d) if cfg.cd else 0.0,           # (Q-W) H_in and the blockwise Wbar H_in
+    }
+    roof_all = {}
+    if phases.get("hessian"):
+        t = phases["hessian"] * 1e-3
+        roof_all["hessian"] = {"bound": "alu", "achieved": fl["hessian"] / t / 1e12, "peak": FP32_ALU_PEAK_TFLOPS,
+                               "unit": "TFLOP/s", "peak_kind": "FP32 FMA, 148 SM x 128 lanes x 2 x 1.965 GHz"}
+    for nm in ("sweep", "grid", "cd"):
+        if q_ms.get(nm) and fl[nm]:
+            t = q_ms[nm] * 1e-3
+            roof_all[nm] = {"bound": "alu", "achieved": fl[nm] / t / 1e12, "peak": FP64_ALU_PEAK_TFLOPS,
+                            "unit": "TFLOP/s", "peak_kind": "FP64 FMA, 148 SM x 64 lanes x 2 x 1.965 GHz"}
+    for v in roof_all.values():
+        v["frac"] = v["achieved"] / v["peak"]
+        v["traffic"] = None
+    times = {"hessian": phases.get("hessian", 0.0), "sweep": q_ms.get("sweep", 0.0), "grid": q_ms.get("grid", 0.0),
+             "cd": q_ms.get("cd", 0.0)}
+    dominant = max(times, key=times.get)
+    roofline = dict(roof_all.get(dominant, {}), kernel=dominant)
+    loop_ms = q_ms.get("grid", 0.0) + q_ms.get("sweep", 0.0) + q_ms.get("compensation", 0.0)
+
+    line = {
+        "metric": METRIC, "value": d_out * world / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "d_out": d_out, "d_in": d, "n_heads": H, "d_head": dh,
+                   "tokens": n_tok, "x_dtype": "bf16", "bits": cfg.bits, "quant_group": cfg.quant_group,
+                   "out_block": cfg.out_block, "adaptive_grid": cfg.adaptive, "cd_refine": cfg.cd,
+                   "l2": "inputs larger than L2 (activations %.1f GiB)" % (n_tok * d * 2 / 2 ** 30)},
+        "seconds_per_layer": ms_per_step * 1e-3,
+        "phases_ms": dict(phases, **{"quantize/" + k: v for k, v in q_ms.items()}),
+        "loop_ms": loop_ms,
+        "loop_out_channels_per_s": d_out / (loop_ms * 1e-3) if loop_ms else None,
+        "clocks": clocks, "gpu_launches": count_launches(cfg, proj, n_tok) * args.steps,
+        "roofline": roofline, "rooflines": roof_all,
+    }
+    if e2e is not None:
+        line["e2e"] = e2e
+    if world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(cfg, proj)
+    print(json.dumps(line))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

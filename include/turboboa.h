@@ -92,6 +92,14 @@ const char* tb_status_string(tb_status st);
 tb_status tb_accumulate_hessian(float* H, const void* X, tb_dtype x_type,
                                 long long n_tok, int d, void* stream);
 
+/* The bf16 path of tb_accumulate_hessian runs on the tensor cores and waits on
+ * hardware barriers with a bound of about two seconds.  If a bound ever runs
+ * out the kernel gives up (H is then incomplete) and raises a device word that
+ * this call reads and clears: 0 = no such event, 1 = a wait ran out
+ * (TB_ERR_TIMEOUT), -1 = the word could not be read.  Synchronises the device.
+ * No counterpart in the paper. */
+int tb_device_error_flag(void);
+
 /* R += alpha * (X - Xfp)^T X, the deviation correlation alpha (X - X~) X^T of
  * Algorithm 1 line 5 in the same un-normalised form: R[a][b] accumulates
  * alpha * sum_t (x_t[a] - xfp_t[a]) * x_t[b].  R: [d][d] float, not symmetric. */
@@ -184,6 +192,15 @@ tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W, const flo
                             unsigned char* codes, float* scales, int* zeros, unsigned char* cand,
                             float* W_hat, double* loss, tb_stats* stats, void* ws,
                             size_t ws_bytes, void* stream);
+
+/* Profiling aid with no counterpart in the paper.  While enabled, every
+ * tb_quantize_layer call records CUDA events on its stream around its phases;
+ * tb_profile_read waits for them, adds the elapsed milliseconds per phase into
+ * ms_by_phase[0..n) (host memory; order: setup, grid search, column sweep,
+ * compensation, coordinate descent, output, loss), forgets them and returns the
+ * number of phases (7).  Process-wide and not thread-safe; off by default. */
+void tb_profile_enable(int on);
+int tb_profile_read(double* ms_by_phase, int n);
 
 /* Whole path for one projection from HOST buffers: copies X (and G) to the
  * device, accumulates and finalises H_in, builds H_out, factors both, runs

@@ -57,6 +57,7 @@ _vp, _sz, _ll, _int, _f = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_longlong, c
 _SIGNATURES = {
     "tb_status_string": (ctypes.c_char_p, [_int]),
     "tb_accumulate_hessian": (_int, [_vp, _vp, _int, _ll, _int, _vp]),
+    "tb_device_error_flag": (_int, []),
     "tb_accumulate_cross": (_int, [_vp, _vp, _vp, _int, _ll, _int, _f, _vp]),
     "tb_finalize_hessian": (_int, [_vp, _vp, _vp, _int, _ll, _f, _vp]),
     "tb_build_hout_workspace": (_sz, [_int, _int, _int]),
@@ -67,6 +68,8 @@ _SIGNATURES = {
     "tb_prepare_correction": (_int, [_vp, _vp, _int, _int, _vp, _vp, _vp, _sz, _vp]),
     "tb_quantize_layer_workspace": (_sz, [ctypes.POINTER(LayerDesc), _int, _int]),
     "tb_quantize_layer": (_int, [ctypes.POINTER(LayerDesc)] + [_vp] * 15 + [_vp, _sz, _vp]),
+    "tb_profile_enable": (None, [_int]),
+    "tb_profile_read": (_int, [ctypes.POINTER(ctypes.c_double), _int]),
     "tb_quantize_from_host_workspace": (_sz, [ctypes.POINTER(LayerDesc), _ll, _int]),
     "tb_quantize_from_host": (_int, [ctypes.POINTER(LayerDesc), _vp, _vp, _ll, _vp, _int, _f, _f,
                                      _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
@@ -139,8 +142,13 @@ def _xtype(X):
 
 def tb_accumulate_hessian(H, X) -> None:
     n_tok, d = X.shape
-    _check(load().tb_accumulate_hessian(_ptr(H, torch.float32), _ptr(X), _xtype(X), n_tok, d, _stream()),
+    _check(load().tb_accumulate_hessian(_ptr(H, torch.float32), _ptr(X) if n_tok else None, _xtype(X), n_tok, d,
+                                        _stream()),
            "tb_accumulate_hessian")
+
+
+def tb_device_error_flag() -> int:
+    return int(load().tb_device_error_flag())
 
 
 def tb_accumulate_cross(R, X, Xfp, alpha: float) -> None:
@@ -270,3 +278,17 @@ def tb_quantize_from_host(desc: LayerDesc, W_host, X_host, G_host, damp_in: floa
         float(damp_out), hp(out_host["codes"]), hp(out_host["scales"]), hp(out_host["zeros"]),
         hp(out_host.get("w_hat")), hp(out_host.get("loss")), _ptr(dev_ws), dev_ws.numel(), _stream()),
         "tb_quantize_from_host")
+
+
+PHASES = ("setup", "grid", "sweep", "compensation", "cd", "output", "loss")
+
+
+def tb_profile_enable(on: bool) -> None:
+    load().tb_profile_enable(int(bool(on)))
+
+
+def tb_profile_read() -> dict:
+    """Milliseconds per phase of the tb_quantize_layer calls since tb_profile_enable(True)."""
+    buf = (ctypes.c_double * len(PHASES))()
+    load().tb_profile_read(buf, len(PHASES))
+    return dict(zip(PHASES, [float(v) for v in buf]))

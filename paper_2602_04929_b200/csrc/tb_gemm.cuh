@@ -57,17 +57,102 @@ inline GemmP gemm_params() {
 
 template <typename TAcc>
 struct GemmSmem {
-  static constexpr int LD = (sizeof(TAcc) == 8) ? 130 : 132;
+  static constexpr int LD = 132;
   static constexpr size_t bytes = 2ull * 2ull * GEMM_BK * LD * sizeof(TAcc);
 };
 
-template <typename T>
-__device__ __forceinline__ T zero_of() {
-  return T(0);
-}
+// Per-thread accumulators of a 128 x 128 tile: an 8 x 8 block per thread in
+// both engines, addressed as at(i, j) with tile-local row(i) and col(j).
+//   float : SIMT FFMA engine, rows ty*4+i / 64+ty*4+i-4, columns likewise in tx.
+//   double: FP64 tensor-core engine (mma.sync m8n8k4).  Warp w owns rows
+//           64 (w / 4) .. +63 and columns 32 (w % 4) .. +31 as 8 x 4 fragments of
+//           8 x 8; a fragment gives this thread row lane / 4 and columns
+//           2 (lane % 4), 2 (lane % 4) + 1.
+template <typename TAcc>
+struct GemmAcc;
+
 template <>
-__device__ __forceinline__ __nv_bfloat16 zero_of<__nv_bfloat16>() {
-  return __float2bfloat16(0.0f);
+struct GemmAcc<float> {
+  float v[8][8];
+  __device__ __forceinline__ void clear() {
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+      for (int j = 0; j < 8; ++j) v[i][j] = 0.0f;
+  }
+  __device__ __forceinline__ float at(int i, int j) const { return v[i][j]; }
+  static __device__ __forceinline__ int row(int i) {
+    const int ty = threadIdx.x >> 4;
+    return (i < 4) ? (ty * 4 + i) : (64 + ty * 4 + i - 4);
+  }
+  static __device__ __forceinline__ int col(int j) {
+    const int tx = threadIdx.x & 15;
+    return (j < 4) ? (tx * 4 + j) : (64 + tx * 4 + j - 4);
+  }
+};
+
+template <>
+struct GemmAcc<double> {
+  double v[8][4][2];
+  __device__ __forceinline__ void clear() {
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) v[i][j][0] = v[i][j][1] = 0.0;
+  }
+  __device__ __forceinline__ double at(int i, int j) const { return v[i][j >> 1][j & 1]; }
+  static __device__ __forceinline__ int row(int i) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    return (warp >> 2) * 64 + i * 8 + (lane >> 2);
+  }
+  static __device__ __forceinline__ int col(int j) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    return (warp & 3) * 32 + (j >> 1) * 8 + (lane & 3) * 2 + (j & 1);
+  }
+};
+
+// One K chunk (16) of the tile product from shared memory.
+__device__ __forceinline__ void gemm_chunk(GemmAcc<float>& acc, const float* as, const float* bs) {
+  constexpr int LD = GemmSmem<float>::LD;
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+#pragma unroll
+  for (int kk = 0; kk < GEMM_BK; ++kk) {
+    float a[8], b[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      a[i] = as[kk * LD + ty * 4 + i];
+      a[4 + i] = as[kk * LD + 64 + ty * 4 + i];
+      b[i] = bs[kk * LD + tx * 4 + i];
+      b[4 + i] = bs[kk * LD + 64 + tx * 4 + i];
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+      for (int j = 0; j < 8; ++j) acc.v[i][j] = fmaf(a[i], b[j], acc.v[i][j]);
+  }
+}
+
+__device__ __forceinline__ void gemm_chunk(GemmAcc<double>& acc, const double* as, const double* bs) {
+  constexpr int LD = GemmSmem<double>::LD;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int kq = lane & 3, rq = lane >> 2;
+  const double* ap = as + kq * LD + (warp >> 2) * 64 + rq;
+  const double* bp = bs + kq * LD + (warp & 3) * 32 + rq;
+#pragma unroll
+  for (int k4 = 0; k4 < GEMM_BK / 4; ++k4) {
+    double a[8], b[4];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) a[i] = ap[k4 * 4 * LD + i * 8];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) b[j] = bp[k4 * 4 * LD + j * 8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+                     : "+d"(acc.v[i][j][0]), "+d"(acc.v[i][j][1])
+                     : "d"(a[i]), "d"(b[j]));
+  }
 }
 
 // acc += A_tile * B_tile over k in [k_begin, k_end), k_begin a multiple of 16.
@@ -77,13 +162,12 @@ __device__ __forceinline__ __nv_bfloat16 zero_of<__nv_bfloat16>() {
 // GemmSmem<TAcc>::bytes.  On return all threads have passed a barrier, so the
 // shared buffer may be reused at once.
 template <typename TAcc, bool A_MCONTIG, bool B_NCONTIG, typename FA, typename FB>
-__device__ __forceinline__ void gemm_mainloop(TAcc (&acc)[8][8], FA load_a, FB load_b,
+__device__ __forceinline__ void gemm_mainloop(GemmAcc<TAcc>& acc, FA load_a, FB load_b,
                                               int k_begin, int k_end, unsigned char* smem) {
   constexpr int LD = GemmSmem<TAcc>::LD;
   TAcc* As = reinterpret_cast<TAcc*>(smem);  // [2][BK][LD]
   TAcc* Bs = As + 2 * GEMM_BK * LD;          // [2][BK][LD]
   const int tid = threadIdx.x;
-  const int tx = tid & 15, ty = tid >> 4;
 
   TAcc ra[8], rb[8];
   auto load_regs = [&](int k0) {
@@ -150,37 +234,11 @@ __device__ __forceinline__ void gemm_mainloop(TAcc (&acc)[8][8], FA load_a, FB l
   for (int k0 = k_begin; k0 < k_end; k0 += GEMM_BK) {
     const bool more = (k0 + GEMM_BK) < k_end;
     if (more) load_regs(k0 + GEMM_BK);
-    const TAcc* as = As + buf * GEMM_BK * LD;
-    const TAcc* bs = Bs + buf * GEMM_BK * LD;
-#pragma unroll
-    for (int kk = 0; kk < GEMM_BK; ++kk) {
-      TAcc a[8], b[8];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        a[i] = as[kk * LD + ty * 4 + i];
-        a[4 + i] = as[kk * LD + 64 + ty * 4 + i];
-        b[i] = bs[kk * LD + tx * 4 + i];
-        b[4 + i] = bs[kk * LD + 64 + tx * 4 + i];
-      }
-#pragma unroll
-      for (int i = 0; i < 8; ++i)
-#pragma unroll
-        for (int j = 0; j < 8; ++j) acc[i][j] = fma(a[i], b[j], acc[i][j]);
-    }
+    gemm_chunk(acc, As + buf * GEMM_BK * LD, Bs + buf * GEMM_BK * LD);
     if (more) store_smem(buf ^ 1);
     __syncthreads();
     buf ^= 1;
   }
-}
-
-// Tile-local row / column owned by accumulator index i (or j) of this thread.
-__device__ __forceinline__ int gemm_row_of(int i) {
-  const int ty = threadIdx.x >> 4;
-  return (i < 4) ? (ty * 4 + i) : (64 + ty * 4 + i - 4);
-}
-__device__ __forceinline__ int gemm_col_of(int j) {
-  const int tx = threadIdx.x & 15;
-  return (j < 4) ? (tx * 4 + j) : (64 + tx * 4 + j - 4);
 }
 
 // One 128 x 128 tile of the strided GEMM described by p.
@@ -198,11 +256,8 @@ __device__ __forceinline__ void gemm_tile(const GemmP& p, int m0, int n0, int ba
   if (p.atrim == 2) k_begin = max(k_begin, m0 + p.aoff);
   k_begin = (k_begin / GEMM_BK) * GEMM_BK;
 
-  TAcc acc[8][8];
-#pragma unroll
-  for (int i = 0; i < 8; ++i)
-#pragma unroll
-    for (int j = 0; j < 8; ++j) acc[i][j] = TAcc(0);
+  GemmAcc<TAcc> acc;
+  acc.clear();
 
   const int M = p.M, N = p.N;
   const long long a_m = p.a_m, a_k = p.a_k, b_k = p.b_k, b_n = p.b_n;
@@ -222,14 +277,14 @@ __device__ __forceinline__ void gemm_tile(const GemmP& p, int m0, int n0, int ba
   const bool use_c = (p.beta != 0.0);
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
-    const int m = m0 + gemm_row_of(i);
+    const int m = m0 + GemmAcc<TAcc>::row(i);
     if (m >= M) continue;
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-      const int n = n0 + gemm_col_of(j);
+      const int n = n0 + GemmAcc<TAcc>::col(j);
       if (n >= N) continue;
       TC* c = C + (long long)m * p.ldc + n;
-      TAcc v = alpha * acc[i][j];
+      TAcc v = alpha * acc.at(i, j);
       if (use_c) v = fma(beta, static_cast<TAcc>(*c), v);
       *c = static_cast<TC>(v);
     }

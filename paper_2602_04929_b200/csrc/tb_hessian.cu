@@ -8,6 +8,8 @@
 
 namespace tb {
 
+tb_status syrk_bf16_tensor(float* H, const __nv_bfloat16* X, long long n_tok, int d, cudaStream_t st);
+
 // Tokens per launch: partial sums of one launch stay in float registers, the
 // running sum in H absorbs one rounding per launch.
 static const long long kTokChunk = 4096;
@@ -30,11 +32,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
             long long n_tok, int d, float alpha) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int m0 = blockIdx.y * GEMM_BM, n0 = blockIdx.x * GEMM_BN;
-  float acc[8][8];
-#pragma unroll
-  for (int i = 0; i < 8; ++i)
-#pragma unroll
-    for (int j = 0; j < 8; ++j) acc[i][j] = 0.0f;
+  GemmAcc<float> acc;
+  acc.clear();
   const int K = (int)n_tok;
   auto la = [&](int mm, int k) -> float {
     const int m = m0 + mm;
@@ -49,12 +48,12 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
   gemm_mainloop<float, true, true>(acc, la, lb, 0, K, smem_raw);
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
-    const int m = m0 + gemm_row_of(i);
+    const int m = m0 + GemmAcc<float>::row(i);
     if (m >= d) continue;
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-      const int n = n0 + gemm_col_of(j);
-      if (n < d) R[(long long)m * d + n] = fmaf(alpha, acc[i][j], R[(long long)m * d + n]);
+      const int n = n0 + GemmAcc<float>::col(j);
+      if (n < d) R[(long long)m * d + n] = fmaf(alpha, acc.at(i, j), R[(long long)m * d + n]);
     }
   }
 }
@@ -178,20 +177,29 @@ using namespace tb;
 
 extern "C" tb_status tb_accumulate_hessian(float* H, const void* X, tb_dtype x_type,
                                            long long n_tok, int d, void* stream) {
-  if (!H || !X || n_tok < 0 || d <= 0 || (d % 8)) return TB_ERR_INVALID_ARG;
+  if (!H || n_tok < 0 || d <= 0 || (d % 8)) return TB_ERR_INVALID_ARG;
   if (x_type != TB_F32 && x_type != TB_BF16) return TB_ERR_INVALID_ARG;
-  if (n_tok == 0) return TB_OK;
+  if (n_tok == 0) return TB_OK;  // nothing to add; X may be NULL
+  if (!X) return TB_ERR_INVALID_ARG;
   cudaStream_t st = as_stream(stream);
-  if (x_type == TB_BF16)
-    return accumulate_typed<__nv_bfloat16>(H, static_cast<const __nv_bfloat16*>(X), n_tok, d, st);
+  if (x_type == TB_BF16) {
+    // bf16 activations: tensor cores (products exact in float, short float accumulations)
+    if (!aligned(X, 16) || !aligned(H, 16)) return TB_ERR_INVALID_ARG;
+    TB_TRY(syrk_bf16_tensor(H, static_cast<const __nv_bfloat16*>(X), n_tok, d, st));
+    k_mirror_lower<<<148 * 8, 256, 0, st>>>(H, d);
+    TB_LAUNCH_CHECK();
+    return TB_OK;
+  }
+  // float activations keep every product exact only on the FP32 pipe
   return accumulate_typed<float>(H, static_cast<const float*>(X), n_tok, d, st);
 }
 
 extern "C" tb_status tb_accumulate_cross(float* R, const void* X, const void* Xfp, tb_dtype x_type,
                                          long long n_tok, int d, float alpha, void* stream) {
-  if (!R || !X || !Xfp || n_tok < 0 || d <= 0 || (d % 8)) return TB_ERR_INVALID_ARG;
+  if (!R || n_tok < 0 || d <= 0 || (d % 8)) return TB_ERR_INVALID_ARG;
   if (x_type != TB_F32 && x_type != TB_BF16) return TB_ERR_INVALID_ARG;
   if (n_tok == 0) return TB_OK;
+  if (!X || !Xfp) return TB_ERR_INVALID_ARG;
   cudaStream_t st = as_stream(stream);
   if (x_type == TB_BF16)
     return cross_typed<__nv_bfloat16>(R, static_cast<const __nv_bfloat16*>(X),

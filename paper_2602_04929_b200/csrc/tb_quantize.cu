@@ -169,11 +169,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) k_grid(GridP p) {
   for (int i = 0; i < 8; ++i) jpart[i] = 0.0;
 
   for (int a0 = 0; a0 < seg; a0 += GEMM_BN) {
-    double acc[8][8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i)
-#pragma unroll
-      for (int j = 0; j < 8; ++j) acc[i][j] = 0.0;
+    GemmAcc<double> acc;
+    acc.clear();
     auto la = [&](int mm, int k) -> double { return err_at(mm, k); };
     auto lb = [&](int nn, int k) -> double {
       const int a = a0 + nn;
@@ -182,19 +179,24 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) k_grid(GridP p) {
     gemm_mainloop<double, true, true>(acc, la, lb, 0, seg, smem_raw);
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-      const int cr = gemm_row_of(i);
+      const int cr = GemmAcc<double>::row(i);
 #pragma unroll
-      for (int j = 0; j < 8; ++j) jpart[i] = fma(acc[i][j], err_at(cr, a0 + gemm_col_of(j)), jpart[i]);
+      for (int j = 0; j < 8; ++j)
+        jpart[i] = fma(acc.at(i, j), err_at(cr, a0 + GemmAcc<double>::col(j)), jpart[i]);
     }
   }
-  // sum over the 16 threads (tx) that share the same candidate rows
+  // A candidate row's score is spread over the 4 lanes of a quad and the 4 warps that
+  // share its rows; quads reduce by shuffle, warps through shared memory in a fixed order.
+  double* c_Jw = reinterpret_cast<double*>(smem_raw);  // [4][128], the tile buffers are free now
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     double v = jpart[i];
-#pragma unroll
-    for (int o = 8; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    if ((tid & 15) == 0) c_J[gemm_row_of(i)] = v;
+    v += __shfl_xor_sync(0xffffffffu, v, 1);
+    v += __shfl_xor_sync(0xffffffffu, v, 2);
+    if ((lane & 3) == 0) c_Jw[(warp & 3) * 128 + GemmAcc<double>::row(i)] = v;
   }
+  __syncthreads();
+  if (tid < 128) c_J[tid] = ((c_Jw[tid] + c_Jw[128 + tid]) + c_Jw[256 + tid]) + c_Jw[384 + tid];
   __syncthreads();
 
   // Phase 3: argmin per row, strict '<' so that the lowest k wins ties.
@@ -866,6 +868,29 @@ static tb_status run_sweep(const Plan& p, const float* U_in, const float* P, uns
 
 using namespace tb;
 
+extern "C" void tb_profile_enable(int on) {
+  for (int i = 0; i < g_n_spans; ++i) {
+    cudaEventDestroy(g_spans[i].a);
+    cudaEventDestroy(g_spans[i].b);
+  }
+  g_n_spans = 0;
+  g_profile_on = (on != 0);
+}
+
+extern "C" int tb_profile_read(double* ms_by_phase, int n) {
+  for (int i = 0; i < n; ++i) ms_by_phase[i] = 0.0;
+  for (int i = 0; i < g_n_spans; ++i) {
+    float ms = 0.0f;
+    if (cudaEventSynchronize(g_spans[i].b) == cudaSuccess &&
+        cudaEventElapsedTime(&ms, g_spans[i].a, g_spans[i].b) == cudaSuccess && g_spans[i].phase < n)
+      ms_by_phase[g_spans[i].phase] += (double)ms;
+    cudaEventDestroy(g_spans[i].a);
+    cudaEventDestroy(g_spans[i].b);
+  }
+  g_n_spans = 0;
+  return PH_COUNT;
+}
+
 extern "C" size_t tb_quantize_layer_workspace(const tb_layer_desc* desc, int with_r, int with_loss) {
   Plan p;
   // the larger of the two H_out cases, so that one query serves both
@@ -896,15 +921,19 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
   const long long n_all = (long long)p.d_out * d;
   const long long dd = (long long)d * d;
 
-  if (stats) TB_CUDA_CHECK(cudaMemsetAsync(stats, 0, sizeof(tb_stats), st));
-  k_widen<<<ew_blocks(n_all), 256, 0, st>>>(W, p.Wt, n_all);
-  TB_LAUNCH_CHECK();
-  if (p.T) {
-    k_comp_matrices<<<dim3(p.S, p.H), 128, 0, st>>>(U_out, p.T, p.dh, p.g, p.S);
+  {
+    PhaseScope ph(PH_SETUP, st);
+    if (stats) TB_CUDA_CHECK(cudaMemsetAsync(stats, 0, sizeof(tb_stats), st));
+    k_widen<<<ew_blocks(n_all), 256, 0, st>>>(W, p.Wt, n_all);
     TB_LAUNCH_CHECK();
+    if (p.T) {
+      k_comp_matrices<<<dim3(p.S, p.H), 128, 0, st>>>(U_out, p.T, p.dh, p.g, p.S);
+      TB_LAUNCH_CHECK();
+    }
   }
   if (!p.adaptive) {
     // fixed grid: every row, once, from the original weights
+    PhaseScope ph(PH_GRID, st);
     RowMap all{p.dh, p.dh, 0};
     TB_TRY(run_grid(p, H_in, scales, zeros, cand, all, p.d_out, st));
   }
@@ -912,12 +941,19 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
   for (int step = 0; step < p.S; ++step) {
     const int i0 = step * p.g, M = p.H * p.g;
     RowMap rm{p.g, p.dh, i0};
-    if (p.adaptive) TB_TRY(run_grid(p, H_in, scales, zeros, cand, rm, M, st));
-    k_gather<<<ew_blocks((long long)M * d), 256, 0, st>>>(p.Wt, p.Wk, p.W0c, rm, M, d);
-    TB_LAUNCH_CHECK();
-    TB_TRY(run_sweep(p, U_in, P, codes, zeros, stats, rm, M, st));
+    if (p.adaptive) {
+      PhaseScope ph(PH_GRID, st);
+      TB_TRY(run_grid(p, H_in, scales, zeros, cand, rm, M, st));
+    }
+    {
+      PhaseScope ph(PH_SWEEP, st);
+      k_gather<<<ew_blocks((long long)M * d), 256, 0, st>>>(p.Wt, p.Wk, p.W0c, rm, M, d);
+      TB_LAUNCH_CHECK();
+      TB_TRY(run_sweep(p, U_in, P, codes, zeros, stats, rm, M, st));
+    }
     const int nrem = p.dh - i0 - p.g;
     if (!p.has_hout || nrem <= 0) continue;
+    PhaseScope ph_comp(PH_COMP, st);
     k_residual<<<ew_blocks((long long)M * d), 256, 0, st>>>(p.Wt, codes, p.sD, zeros, p.E, rm, M, d,
                                                             p.seg, p.ng);
     TB_LAUNCH_CHECK();
@@ -970,6 +1006,7 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
 
   // ---- coordinate descent on the scales (Algorithm 3) ----
   if (p.cd) {
+    PhaseScope ph(PH_CD, st);
     const int units = (p.n_hin == 1) ? 1 : p.H;
     k_cd_prep<<<ew_blocks(n_all), 256, 0, st>>>(W, codes, p.sD, zeros, p.Dq, p.Wb, p.d_out, d, p.seg,
                                                p.ng);
@@ -1088,12 +1125,16 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
     }
   }
 
-  k_dequant<<<ew_blocks(n_all), 256, 0, st>>>(codes, p.sD, zeros, W_hat, scales, p.d_out, d, p.seg,
-                                             p.ng);
-  TB_LAUNCH_CHECK();
+  {
+    PhaseScope ph(PH_OUTPUT, st);
+    k_dequant<<<ew_blocks(n_all), 256, 0, st>>>(codes, p.sD, zeros, W_hat, scales, p.d_out, d, p.seg,
+                                               p.ng);
+    TB_LAUNCH_CHECK();
+  }
 
   // ---- loss of the proofs of Propositions 3.1 / 3.2 ----
   if (loss) {
+    PhaseScope ph(PH_LOSS, st);
     const int units = (p.n_hin == 1) ? 1 : p.H;
     k_cd_prep<<<ew_blocks(n_all), 256, 0, st>>>(W, codes, p.sD, zeros, p.Dq, nullptr, p.d_out, d,
                                                p.seg, p.ng);
