@@ -200,6 +200,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="l2_7b_q")
     ap.add_argument("--tokens", type=int, default=0, help="override the token count (default: the config's)")
+    ap.add_argument("--heads", type=int, default=0,
+                    help="keep only this many heads of the projection (small captures under a profiler)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -210,6 +212,9 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     cfg, proj = workload(args.workload)
+    if args.heads and proj.partner:
+        import dataclasses
+        proj = dataclasses.replace(proj, n_heads=args.heads, d_out=args.heads * proj.d_head)
     if args.impl == "reference":
         run_reference(args, cfg, proj, rank, world)
         return

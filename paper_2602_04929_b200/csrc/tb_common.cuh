@@ -64,6 +64,15 @@ __device__ __forceinline__ double cvt<double, __nv_bfloat16>(__nv_bfloat16 v) {
   return static_cast<double>(__bfloat162float(v));
 }
 
+template <typename T>
+__device__ __forceinline__ T zero_of() {
+  return T(0);
+}
+template <>
+__device__ __forceinline__ __nv_bfloat16 zero_of<__nv_bfloat16>() {
+  return __float2bfloat16(0.0f);
+}
+
 __device__ __forceinline__ double shfl_d(double v, int src) {
   return __shfl_sync(0xffffffffu, v, src);
 }

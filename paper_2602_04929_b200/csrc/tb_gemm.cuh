@@ -156,20 +156,24 @@ __device__ __forceinline__ void gemm_chunk(GemmAcc<double>& acc, const double* a
 }
 
 // acc += A_tile * B_tile over k in [k_begin, k_end), k_begin a multiple of 16.
-// load_a(mm, k) / load_b(nn, k) return the operand for tile-local row / column
-// 0..127 and absolute k, already converted to TAcc, and must return 0 outside
-// the problem.  Every thread of the CTA must call this; `smem` must hold
+// load_a(mm, k) / load_b(nn, k) fetch the raw operand for tile-local row /
+// column 0..127 and absolute k (a value that converts to 0 outside the
+// problem); conv_a(raw, mm, k) / conv_b(raw, nn, k) turn it into TAcc.  The
+// fetch of the next chunk is issued before the current chunk's arithmetic and
+// its conversion after it, so that the latency of global memory hides behind
+// the arithmetic.  Every thread of the CTA must call this; `smem` must hold
 // GemmSmem<TAcc>::bytes.  On return all threads have passed a barrier, so the
 // shared buffer may be reused at once.
-template <typename TAcc, bool A_MCONTIG, bool B_NCONTIG, typename FA, typename FB>
-__device__ __forceinline__ void gemm_mainloop(GemmAcc<TAcc>& acc, FA load_a, FB load_b,
+template <typename TAcc, bool A_MCONTIG, bool B_NCONTIG, typename FA, typename CA, typename FB, typename CB>
+__device__ __forceinline__ void gemm_mainloop(GemmAcc<TAcc>& acc, FA load_a, CA conv_a, FB load_b, CB conv_b,
                                               int k_begin, int k_end, unsigned char* smem) {
   constexpr int LD = GemmSmem<TAcc>::LD;
   TAcc* As = reinterpret_cast<TAcc*>(smem);  // [2][BK][LD]
   TAcc* Bs = As + 2 * GEMM_BK * LD;          // [2][BK][LD]
   const int tid = threadIdx.x;
 
-  TAcc ra[8], rb[8];
+  decltype(load_a(0, 0)) ra[8];
+  decltype(load_b(0, 0)) rb[8];
   auto load_regs = [&](int k0) {
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
@@ -196,7 +200,7 @@ __device__ __forceinline__ void gemm_mainloop(GemmAcc<TAcc>& acc, FA load_a, FB 
       rb[i] = load_b(nn, k0 + kk);
     }
   };
-  auto store_smem = [&](int buf) {
+  auto store_smem = [&](int buf, int k0) {
     TAcc* as = As + buf * GEMM_BK * LD;
     TAcc* bs = Bs + buf * GEMM_BK * LD;
 #pragma unroll
@@ -209,7 +213,7 @@ __device__ __forceinline__ void gemm_mainloop(GemmAcc<TAcc>& acc, FA load_a, FB 
         kk = tid & 15;
         mm = (tid >> 4) + 16 * i;
       }
-      as[kk * LD + mm] = ra[i];
+      as[kk * LD + mm] = conv_a(ra[i], mm, k0 + kk);
     }
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
@@ -221,13 +225,13 @@ __device__ __forceinline__ void gemm_mainloop(GemmAcc<TAcc>& acc, FA load_a, FB 
         kk = tid & 15;
         nn = (tid >> 4) + 16 * i;
       }
-      bs[kk * LD + nn] = rb[i];
+      bs[kk * LD + nn] = conv_b(rb[i], nn, k0 + kk);
     }
   };
 
   if (k_begin < k_end) {
     load_regs(k_begin);
-    store_smem(0);
+    store_smem(0, k_begin);
   }
   __syncthreads();
   int buf = 0;
@@ -235,7 +239,7 @@ __device__ __forceinline__ void gemm_mainloop(GemmAcc<TAcc>& acc, FA load_a, FB 
     const bool more = (k0 + GEMM_BK) < k_end;
     if (more) load_regs(k0 + GEMM_BK);
     gemm_chunk(acc, As + buf * GEMM_BK * LD, Bs + buf * GEMM_BK * LD);
-    if (more) store_smem(buf ^ 1);
+    if (more) store_smem(buf ^ 1, k0 + GEMM_BK);
     __syncthreads();
     buf ^= 1;
   }
@@ -261,17 +265,17 @@ __device__ __forceinline__ void gemm_tile(const GemmP& p, int m0, int n0, int ba
 
   const int M = p.M, N = p.N;
   const long long a_m = p.a_m, a_k = p.a_k, b_k = p.b_k, b_n = p.b_n;
-  auto la = [&](int mm, int k) -> TAcc {
+  auto la = [&](int mm, int k) -> TA {
     const int m = m0 + mm;
-    return (m < M && k < k_end) ? cvt<TAcc, TA>(A[(long long)m * a_m + (long long)k * a_k])
-                                : TAcc(0);
+    return (m < M && k < k_end) ? A[(long long)m * a_m + (long long)k * a_k] : zero_of<TA>();
   };
-  auto lb = [&](int nn, int k) -> TAcc {
+  auto lb = [&](int nn, int k) -> TB {
     const int n = n0 + nn;
-    return (n < N && k < k_end) ? cvt<TAcc, TB>(B[(long long)k * b_k + (long long)n * b_n])
-                                : TAcc(0);
+    return (n < N && k < k_end) ? B[(long long)k * b_k + (long long)n * b_n] : zero_of<TB>();
   };
-  gemm_mainloop<TAcc, A_MCONTIG, B_NCONTIG>(acc, la, lb, k_begin, k_end, smem);
+  auto ca = [](TA v, int, int) -> TAcc { return cvt<TAcc, TA>(v); };
+  auto cb = [](TB v, int, int) -> TAcc { return cvt<TAcc, TB>(v); };
+  gemm_mainloop<TAcc, A_MCONTIG, B_NCONTIG>(acc, la, ca, lb, cb, k_begin, k_end, smem);
 
   const TAcc alpha = static_cast<TAcc>(p.alpha), beta = static_cast<TAcc>(p.beta);
   const bool use_c = (p.beta != 0.0);

@@ -35,17 +35,26 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
   GemmAcc<float> acc;
   acc.clear();
   const int K = (int)n_tok;
-  auto la = [&](int mm, int k) -> float {
+  struct Pair {
+    TX x, xfp;
+  };
+  auto la = [&](int mm, int k) -> Pair {
     const int m = m0 + mm;
-    if (m >= d || k >= K) return 0.0f;
-    const long long o = (long long)k * d + m;
-    return cvt<float, TX>(X[o]) - cvt<float, TX>(Xfp[o]);
+    Pair p{zero_of<TX>(), zero_of<TX>()};
+    if (m < d && k < K) {
+      const long long o = (long long)k * d + m;
+      p.x = X[o];
+      p.xfp = Xfp[o];
+    }
+    return p;
   };
-  auto lb = [&](int nn, int k) -> float {
+  auto ca = [](Pair p, int, int) -> float { return cvt<float, TX>(p.x) - cvt<float, TX>(p.xfp); };
+  auto lb = [&](int nn, int k) -> TX {
     const int n = n0 + nn;
-    return (n < d && k < K) ? cvt<float, TX>(X[(long long)k * d + n]) : 0.0f;
+    return (n < d && k < K) ? X[(long long)k * d + n] : zero_of<TX>();
   };
-  gemm_mainloop<float, true, true>(acc, la, lb, 0, K, smem_raw);
+  auto cb = [](TX v, int, int) -> float { return cvt<float, TX>(v); };
+  gemm_mainloop<float, true, true>(acc, la, ca, lb, cb, 0, K, smem_raw);
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     const int m = m0 + GemmAcc<float>::row(i);

@@ -153,15 +153,19 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) k_grid(GridP p) {
   const double* Wt = p.Wt;
   const int d = p.d, seg = p.seg;
 
-  // quantization error of candidate row cr at segment column a
-  auto err_at = [&](int cr, int a) -> double {
-    const long long grow = c_row[cr];
-    if (grow < 0 || a >= seg) return 0.0;
-    const double w = Wt[grow * d + seg0 + a];
+  // round-to-nearest error of weight w on the grid of candidate row cr (0 for w = 0,
+  // which is what rows and columns outside the problem are given)
+  auto err_of = [&](int cr, double w) -> double {
     const double s = c_s[cr], z = c_z[cr];
     double q = rne(fma(w, c_rs[cr], z));
     q = fmin(fmax(q, 0.0), maxq);
     return w - s * (q - z);
+  };
+  // quantization error of candidate row cr at segment column a
+  auto err_at = [&](int cr, int a) -> double {
+    const long long grow = c_row[cr];
+    if (grow < 0 || a >= seg) return 0.0;
+    return err_of(cr, Wt[grow * d + seg0 + a]);
   };
 
   double jpart[8];
@@ -171,12 +175,18 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) k_grid(GridP p) {
   for (int a0 = 0; a0 < seg; a0 += GEMM_BN) {
     GemmAcc<double> acc;
     acc.clear();
-    auto la = [&](int mm, int k) -> double { return err_at(mm, k); };
-    auto lb = [&](int nn, int k) -> double {
-      const int a = a0 + nn;
-      return (a < seg && k < seg) ? (double)H[(long long)(seg0 + k) * d + seg0 + a] : 0.0;
+    // fetch the weight; the candidate's error is formed when the chunk is staged
+    auto la = [&](int mm, int k) -> double {
+      const long long grow = c_row[mm];
+      return (grow >= 0 && k < seg) ? Wt[grow * d + seg0 + k] : 0.0;
     };
-    gemm_mainloop<double, true, true>(acc, la, lb, 0, seg, smem_raw);
+    auto ca = [&](double w, int mm, int) -> double { return err_of(mm, w); };
+    auto lb = [&](int nn, int k) -> float {
+      const int a = a0 + nn;
+      return (a < seg && k < seg) ? H[(long long)(seg0 + k) * d + seg0 + a] : 0.0f;
+    };
+    auto cb = [](float v, int, int) -> double { return (double)v; };
+    gemm_mainloop<double, true, true>(acc, la, ca, lb, cb, 0, seg, smem_raw);
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const int cr = GemmAcc<double>::row(i);
