@@ -143,6 +143,31 @@ size_t tb_factor_workspace(int n_batch, int d);
 tb_status tb_factor(const float* H, int n_batch, int d, float* U, float* Hinv, int* info,
                     void* ws, size_t ws_bytes, void* stream);
 
+/* tb_factor without a caller-provided workspace and without any allocation.
+ * The paper has no counterpart: this entry point exists for callers that must
+ * not, or cannot, obtain device memory when they need a factor -- a process
+ * that has handed all free device memory to its own pool at start-up (a later
+ * cudaMalloc would fail), or a latency-critical loop in which cudaMalloc /
+ * cudaFree are banned because they synchronise the whole device.
+ *
+ * The scratch is a fixed array of tb_factor_static_capacity() bytes (32 MiB)
+ * inside the library; every GPU on which the library is loaded holds it until
+ * the process exits.  Inputs and outputs are still the caller's.  Same results
+ * and same info semantics as tb_factor (no Hinv output).  A problem whose
+ * tb_factor_workspace(n_batch, d) exceeds the capacity is rejected with
+ * TB_ERR_UNSUPPORTED before anything is enqueued (64 matrices of 128 x 128, or
+ * one of 1024 x 1024, fit).
+ *
+ * The first call on each device looks up the array's device address (the
+ * device must be current); make that first call outside any stream capture.
+ * All calls share the one array: it keeps whatever the previous call left
+ * (the call clears what it needs zeroed), and two calls whose work overlaps on
+ * the GPU -- different streams, or different host threads -- race on it.
+ * Calls on one stream are safe.  No cudaMalloc, cudaFree or other allocating
+ * routine is called. */
+size_t tb_factor_static_capacity(void);
+tb_status tb_factor_static(const float* H, int n_batch, int d, float* U, int* info, void* stream);
+
 /* Operands of the propagated-error terms from R and U_in:
  *   P = ((R U^T) masked to its strictly upper triangle) U   (Algorithm 2, line 2)
  *   C = R U^T U = R H_in^{-1}                               (Proposition 3.2)

@@ -64,6 +64,8 @@ _SIGNATURES = {
     "tb_build_hout": (_int, [_vp, _vp, _vp, _int, _int, _int, _int, _f, _vp, _sz, _vp]),
     "tb_factor_workspace": (_sz, [_int, _int]),
     "tb_factor": (_int, [_vp, _int, _int, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "tb_factor_static_capacity": (_sz, []),
+    "tb_factor_static": (_int, [_vp, _int, _int, _vp, _vp, _vp]),
     "tb_prepare_correction_workspace": (_sz, [_int, _int]),
     "tb_prepare_correction": (_int, [_vp, _vp, _int, _int, _vp, _vp, _vp, _sz, _vp]),
     "tb_quantize_layer_workspace": (_sz, [ctypes.POINTER(LayerDesc), _int, _int]),
@@ -194,6 +196,22 @@ def tb_factor(H, want_inverse: bool = False):
         U = U[0]
         Hinv = Hinv[0] if want_inverse else None
     return (U, info, Hinv) if want_inverse else (U, info)
+
+
+def tb_factor_static(H, U=None, info=None):
+    """tb_factor through the library's own fixed scratch array: no workspace is
+    allocated here or in the library.  Pass preallocated U and info to make the
+    call itself allocation-free; otherwise they are created with torch."""
+    squeeze = H.dim() == 2
+    Hb = H.unsqueeze(0) if squeeze else H
+    n_batch, d, _ = Hb.shape
+    if U is None:
+        U = torch.empty_like(Hb)
+    if info is None:
+        info = torch.empty(n_batch, dtype=torch.int32, device=H.device)
+    _check(load().tb_factor_static(_ptr(Hb, torch.float32), n_batch, d, _ptr(U, torch.float32), _ptr(info),
+                                   _stream()), "tb_factor_static")
+    return (U[0] if squeeze and U.dim() == 3 else U), info
 
 
 def tb_prepare_correction(R, U_in):
