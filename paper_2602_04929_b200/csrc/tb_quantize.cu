@@ -450,6 +450,208 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) k_sweep_block(SweepP p) {
   }
 }
 
+// ---------------------------------------------------------------------------
+// Column sweep without the propagated-error term, one launch per step
+// (Algorithm 2 with P = 0; Eq. 2).  Rows never interact inside the sweep, so a
+// CTA keeps 8 active rows for the whole sweep and no CTA ever waits for another.
+//
+// Left-looking form: the values of block b on arrival are
+//   w[:, b] = W0[:, b] - Err[:, 0 : 128 b] U[0 : 128 b, b],
+// where Err holds the normalised errors of the columns already quantized.
+// 16 warps: warps 0-7 are the panel warps (one row each, one lane per column,
+// the 128 columns of a block strictly in order); warps 8-15 are the update
+// warps.  While the panel warps walk block b, the update warps form the part
+// of the sum for block b+1 that needs only blocks < b (8 x 128b x 128, on the
+// FP64 tensor pipe, U streamed through a cp.async ring of 32-row chunks, the
+// contraction split over the 8 warps and reduced in a fixed order); the last
+// 128 terms follow when the panel is done.  Only __syncthreads and one named
+// barrier among the update warps are used; every trip count depends on b alone.
+// ---------------------------------------------------------------------------
+enum { RS_THREADS = 512, RS_STAGES = 4, RS_LDB = 136, RS_CHUNK = 32 };
+struct RowSweepP {
+  const double* Wt;      // [d_out][d] current W~ (rows of the step are read, never written)
+  const float* U;        // [n_hin][d][d]
+  double* ErrG;          // [M][d] normalised errors of the step's rows
+  unsigned char* codes;  // [d_out][d]
+  const double* sD;      // [d_out][ng]
+  const int* z;          // [d_out][ng]
+  tb_stats* stats;       // or nullptr
+  RowMap rm;
+  int M, d, seg, ng, maxq, nblk;
+  int units, rows_per_unit, ctas_per_unit;
+};
+struct RowSweepSmem {
+  float sU[128 * 128];                          // diagonal block of U
+  float ring[RS_STAGES][RS_CHUNK][RS_LDB];      // streamed rows of U
+  double red[8][8][128];                        // per-warp partial sums of the update
+  double wblk[8][128];                          // arrival values of the current block
+  double Es[8][128];                            // normalised errors of the current block
+};
+
+__device__ __forceinline__ void mma_f64(double (&c)[2], double a, double b) {
+  asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+               : "+d"(c[0]), "+d"(c[1])
+               : "d"(a), "d"(b));
+}
+
+__global__ void __launch_bounds__(RS_THREADS, 1) k_sweep_rows(RowSweepP p) {
+  extern __shared__ __align__(16) unsigned char rs_raw[];
+  RowSweepSmem& sm = *reinterpret_cast<RowSweepSmem*>(rs_raw);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int unit = blockIdx.x / p.ctas_per_unit;
+  const int r_first = (blockIdx.x % p.ctas_per_unit) * 8;  // first row of this CTA inside its unit
+  const int d = p.d;
+  const float* U = p.U + (long long)unit * d * d * (p.units > 1 ? 1 : 0);
+  const double maxq = (double)p.maxq;
+  const int m_base = unit * p.rows_per_unit + r_first;
+
+  // fragment coordinates of this lane: row fr of the 8 rows, k / column pair index fk
+  const int fr = lane >> 2, fk = lane & 3;
+  const bool fr_valid = (r_first + fr) < p.rows_per_unit;
+  const long long fr_grow = fr_valid ? p.rm.row(m_base + fr) : 0;
+
+  // block 0 arrives unchanged
+  for (int idx = tid; idx < 8 * 128; idx += RS_THREADS) {
+    const int r = idx >> 7, c = idx & 127;
+    sm.wblk[r][c] = (r_first + r < p.rows_per_unit) ? p.Wt[p.rm.row(m_base + r) * d + c] : 0.0;
+  }
+
+  unsigned int n_near = 0, n_clamp = 0;
+  for (int b = 0; b < p.nblk; ++b) {
+    const int c0 = b * 128;
+    // diagonal block of U for the panel
+    for (int idx = tid; idx < 128 * 32; idx += RS_THREADS) {
+      const int j = idx >> 5, c4 = (idx & 31) * 4;
+      *reinterpret_cast<float4*>(sm.sU + j * 128 + c4) =
+          *reinterpret_cast<const float4*>(U + (long long)(c0 + j) * d + c0 + c4);
+    }
+    __syncthreads();
+
+    if (warp < 8) {
+      // ------------------------- panel: row `warp`, columns c0 .. c0+127 -------------------------
+      const bool valid = (r_first + warp) < p.rows_per_unit;
+      const long long grow = valid ? p.rm.row(m_base + warp) : 0;
+      double w[4];
+#pragma unroll
+      for (int sb = 0; sb < 4; ++sb) w[sb] = sm.wblk[warp][sb * 32 + lane];
+#pragma unroll 1
+      for (int sb = 0; sb < 4; ++sb) {
+        const int cl = sb * 32 + lane, col = c0 + cl;
+        const long long so = grow * p.ng + col / p.seg;
+        const double s_l = valid ? p.sD[so] : 1.0, z_l = valid ? (double)p.z[so] : 0.0;
+        const double rs_l = 1.0 / s_l;
+        const double rd_l = 1.0 / (double)sm.sU[cl * 128 + cl];
+        const double srd_l = s_l * rd_l;
+        float u[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) u[j] = sm.sU[(sb * 32 + j) * 128 + cl];
+        double v = (sb == 0) ? w[0] : (sb == 1) ? w[1] : (sb == 2) ? w[2] : w[3];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const double ard = fma(s_l, z_l, v) * rd_l;
+          double q = rne(fma(v, rs_l, z_l));
+          q = fmin(fmax(q, 0.0), maxq);
+          const double e = fma(-srd_l, q, ard);
+          const double ej = shfl_d(e, j);
+          if (lane > j) v = fma(-ej, (double)u[j], v);
+        }
+        const double x = fma(v, rs_l, z_l);
+        const double xr = rne(x);
+        const double q = fmin(fmax(xr, 0.0), maxq);
+        const double e_mine = fma(-srd_l, q, fma(s_l, z_l, v) * rd_l);
+        sm.Es[warp][cl] = valid ? e_mine : 0.0;
+        if (valid) {
+          p.codes[grow * d + col] = (unsigned char)(int)q;
+          p.ErrG[(long long)(m_base + warp) * d + col] = e_mine;
+          const double fl = floor(x);
+          const double a0 = fmin(fmax(fl, 0.0), maxq), a1 = fmin(fmax(fl + 1.0, 0.0), maxq);
+          if (fabs(x - (fl + 0.5)) < 1e-6 && a0 != a1) ++n_near;
+          if (xr != q) ++n_clamp;
+        }
+        // the sub-block's errors update the later sub-blocks of this block
+        for (int j = 0; j < 32; ++j) {
+          const double ej = shfl_d(e_mine, j);
+          const float* ur = sm.sU + (sb * 32 + j) * 128 + lane;
+          if (sb < 1) w[1] = fma(-ej, (double)ur[32], w[1]);
+          if (sb < 2) w[2] = fma(-ej, (double)ur[64], w[2]);
+          if (sb < 3) w[3] = fma(-ej, (double)ur[96], w[3]);
+        }
+      }
+    } else if (b + 1 < p.nblk) {
+      // ------------------------- update warps: part of block b+1 from blocks < b -------------------------
+      const int uw = warp - 8, ut = tid - 256;
+      const int cn = c0 + 128;     // first column of block b+1
+      const int nchunk = 4 * b;    // 32-row chunks of U[0 : 128 b, block b+1]
+      double acc[16][2];
+#pragma unroll
+      for (int nt = 0; nt < 16; ++nt) acc[nt][0] = acc[nt][1] = 0.0;
+      auto issue = [&](int c) {
+        if (c < nchunk) {
+          float* dst = &sm.ring[c % RS_STAGES][0][0];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int piece = ut + 256 * i;  // 0 .. 1023 : row = piece / 32, 16-byte piece = piece % 32
+            const int r = piece >> 5, q4 = (piece & 31) * 4;
+            const float* src = U + (long long)(c * RS_CHUNK + r) * d + cn + q4;
+            const unsigned int sa = (unsigned int)__cvta_generic_to_shared(dst + r * RS_LDB + q4);
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sa), "l"(src) : "memory");
+          }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+      };
+      for (int c = 0; c < RS_STAGES - 1; ++c) issue(c);
+      const double* erow = p.ErrG + (long long)(m_base + fr) * d + 4 * uw + fk;
+      double a_next = (fr_valid && nchunk > 0) ? erow[0] : 0.0;
+      for (int c = 0; c < nchunk; ++c) {
+        asm volatile("cp.async.wait_group %0;" ::"n"(RS_STAGES - 2) : "memory");
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        issue(c + RS_STAGES - 1);
+        const double a = a_next;
+        if (c + 1 < nchunk) a_next = fr_valid ? erow[(c + 1) * RS_CHUNK] : 0.0;
+        const float* bp = &sm.ring[c % RS_STAGES][4 * uw + fk][fr];
+#pragma unroll
+        for (int nt = 0; nt < 16; ++nt) mma_f64(acc[nt], a, (double)bp[nt * 8]);
+      }
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+#pragma unroll
+      for (int nt = 0; nt < 16; ++nt) {
+        sm.red[uw][fr][nt * 8 + 2 * fk] = acc[nt][0];
+        sm.red[uw][fr][nt * 8 + 2 * fk + 1] = acc[nt][1];
+      }
+    }
+    __syncthreads();
+
+    if (b + 1 < p.nblk) {
+      // ------------------------- last 128 terms and hand-over of block b+1 -------------------------
+      // warp `warp` owns the 8 columns cn + 8 warp .. +7 for all 8 rows
+      const int cn = c0 + 128, nt = warp;
+      double acc[2] = {0.0, 0.0};
+      const float* ub = U + (long long)(c0 + fk) * d + cn + nt * 8 + fr;
+#pragma unroll 8
+      for (int q = 0; q < 32; ++q) mma_f64(acc, sm.Es[fr][4 * q + fk], (double)ub[(long long)(4 * q) * d]);
+      const int cc = nt * 8 + 2 * fk;
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        double t = 0.0;
+#pragma unroll
+        for (int w8 = 0; w8 < 8; ++w8) t += sm.red[w8][fr][cc + e];
+        const double w0 = fr_valid ? p.Wt[fr_grow * d + cn + cc + e] : 0.0;
+        sm.wblk[fr][cc + e] = (w0 - t) - acc[e];
+      }
+    }
+    __syncthreads();
+  }
+  if (p.stats && warp < 8) {
+    n_near = __reduce_add_sync(0xffffffffu, n_near);
+    n_clamp = __reduce_add_sync(0xffffffffu, n_clamp);
+    if (lane == 0) {
+      if (n_near) atomicAdd(&p.stats->near_tie_codes, (unsigned long long)n_near);
+      if (n_clamp) atomicAdd(&p.stats->clamped_codes, (unsigned long long)n_clamp);
+      if (blockIdx.x == 0 && warp == 0) atomicAdd(&p.stats->column_steps, (unsigned long long)d);
+    }
+  }
+}
+
 // E[m][k] = W~[row(m)][k] - s (code - z): the quantization error of the group on
 // the weights it saw (Proposition 3.1's W_B - Q_B).
 __global__ void k_residual(const double* __restrict__ Wt, const unsigned char* __restrict__ codes,
@@ -836,6 +1038,34 @@ static tb_status run_grid(const Plan& p, const float* H_in, float* scales, int* 
   return TB_OK;
 }
 
+static tb_status run_sweep_rows(const Plan& p, const float* U_in, unsigned char* codes,
+                                const int* zeros, tb_stats* stats, RowMap rm, int M, cudaStream_t st) {
+  RowSweepP sp;
+  sp.Wt = p.Wt;
+  sp.U = U_in;
+  sp.ErrG = p.Wk;  // the working-row buffer of the multi-launch sweep doubles as the error history
+  sp.codes = codes;
+  sp.sD = p.sD;
+  sp.z = zeros;
+  sp.stats = stats;
+  sp.rm = rm;
+  sp.M = M;
+  sp.d = p.d;
+  sp.seg = p.seg;
+  sp.ng = p.ng;
+  sp.maxq = p.maxq;
+  sp.nblk = p.d / 128;
+  sp.units = (p.n_hin == 1) ? 1 : p.H;
+  sp.rows_per_unit = M / sp.units;
+  sp.ctas_per_unit = (sp.rows_per_unit + 7) / 8;
+  static bool configured[64] = {false};
+  TB_TRY(allow_smem(k_sweep_rows, sizeof(RowSweepSmem), configured));
+  const long long ctas = (long long)sp.ctas_per_unit * sp.units;
+  k_sweep_rows<<<(unsigned)ctas, RS_THREADS, sizeof(RowSweepSmem), st>>>(sp);
+  TB_LAUNCH_CHECK();
+  return TB_OK;
+}
+
 static tb_status run_sweep(const Plan& p, const float* U_in, const float* P, unsigned char* codes,
                            const int* zeros, tb_stats* stats, RowMap rm, int M, cudaStream_t st) {
   SweepP sp;
@@ -957,9 +1187,14 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
     }
     {
       PhaseScope ph(PH_SWEEP, st);
-      k_gather<<<ew_blocks((long long)M * d), 256, 0, st>>>(p.Wt, p.Wk, p.W0c, rm, M, d);
-      TB_LAUNCH_CHECK();
-      TB_TRY(run_sweep(p, U_in, P, codes, zeros, stats, rm, M, st));
+      if (with_r) {
+        // with the propagated-error term: one launch per column block
+        k_gather<<<ew_blocks((long long)M * d), 256, 0, st>>>(p.Wt, p.Wk, p.W0c, rm, M, d);
+        TB_LAUNCH_CHECK();
+        TB_TRY(run_sweep(p, U_in, P, codes, zeros, stats, rm, M, st));
+      } else {
+        TB_TRY(run_sweep_rows(p, U_in, codes, zeros, stats, rm, M, st));
+      }
     }
     const int nrem = p.dh - i0 - p.g;
     if (!p.has_hout || nrem <= 0) continue;
