@@ -460,14 +460,15 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) k_sweep_block(SweepP p) {
 // where Err holds the normalised errors of the columns already quantized.
 // 16 warps: warps 0-7 are the panel warps (one row each, one lane per column,
 // the 128 columns of a block strictly in order); warps 8-15 are the update
-// warps.  While the panel warps walk block b, the update warps form the part
-// of the sum for block b+1 that needs only blocks < b (8 x 128b x 128, on the
-// FP64 tensor pipe, U streamed through a cp.async ring of 32-row chunks, the
-// contraction split over the 8 warps and reduced in a fixed order); the last
-// 128 terms follow when the panel is done.  Only __syncthreads and one named
-// barrier among the update warps are used; every trip count depends on b alone.
+// warps (two 8-column fragments each, on the FP64 tensor pipe).  While the
+// panel warps walk block b, the update warps form the part of block b+1's sum
+// that needs only blocks < b, streaming 32-row chunks of U and of the error
+// history through a cp.async ring; when the panel is done they add the last
+// 128 terms (errors of block b straight from shared memory) and hand block b+1
+// over.  Synchronisation is by hardware barriers only (ids 1-3, fixed
+// participant counts); every trip count depends on the block index alone.
 // ---------------------------------------------------------------------------
-enum { RS_THREADS = 512, RS_STAGES = 4, RS_LDB = 136, RS_CHUNK = 32 };
+enum { RS_THREADS = 512, RS_STAGES = 7, RS_LDB = 136, RS_LDE = 36, RS_CHUNK = 32, RS_LDW = 132 };
 struct RowSweepP {
   const double* Wt;      // [d_out][d] current W~ (rows of the step are read, never written)
   const float* U;        // [n_hin][d][d]
@@ -480,12 +481,15 @@ struct RowSweepP {
   int M, d, seg, ng, maxq, nblk;
   int units, rows_per_unit, ctas_per_unit;
 };
+struct RowSweepStage {
+  float Ub[RS_CHUNK][RS_LDB];   // 32 rows of U, 128 columns of the target block
+  double Eb[8][RS_LDE];         // the same 32 columns of the error history, 8 rows
+};
 struct RowSweepSmem {
-  float sU[128 * 128];                          // diagonal block of U
-  float ring[RS_STAGES][RS_CHUNK][RS_LDB];      // streamed rows of U
-  double red[8][8][128];                        // per-warp partial sums of the update
-  double wblk[8][128];                          // arrival values of the current block
-  double Es[8][128];                            // normalised errors of the current block
+  float sU[128 * 128];          // diagonal block of U
+  RowSweepStage ring[RS_STAGES];
+  double wblk[8][RS_LDW];       // arrival values of the current block
+  double Es[8][RS_LDW];         // normalised errors of the current block
 };
 
 __device__ __forceinline__ void mma_f64(double (&c)[2], double a, double b) {
@@ -493,6 +497,7 @@ __device__ __forceinline__ void mma_f64(double (&c)[2], double a, double b) {
                : "+d"(c[0]), "+d"(c[1])
                : "d"(a), "d"(b));
 }
+__device__ __forceinline__ void bar_all() { asm volatile("bar.sync 3, 512;" ::: "memory"); }
 
 __global__ void __launch_bounds__(RS_THREADS, 1) k_sweep_rows(RowSweepP p) {
   extern __shared__ __align__(16) unsigned char rs_raw[];
@@ -504,33 +509,31 @@ __global__ void __launch_bounds__(RS_THREADS, 1) k_sweep_rows(RowSweepP p) {
   const float* U = p.U + (long long)unit * d * d * (p.units > 1 ? 1 : 0);
   const double maxq = (double)p.maxq;
   const int m_base = unit * p.rows_per_unit + r_first;
+  const int rows_here = min(8, p.rows_per_unit - r_first);
 
-  // fragment coordinates of this lane: row fr of the 8 rows, k / column pair index fk
-  const int fr = lane >> 2, fk = lane & 3;
-  const bool fr_valid = (r_first + fr) < p.rows_per_unit;
-  const long long fr_grow = fr_valid ? p.rm.row(m_base + fr) : 0;
-
-  // block 0 arrives unchanged
+  // block 0 arrives unchanged; error rows of absent rows stay zero in every ring stage
   for (int idx = tid; idx < 8 * 128; idx += RS_THREADS) {
     const int r = idx >> 7, c = idx & 127;
-    sm.wblk[r][c] = (r_first + r < p.rows_per_unit) ? p.Wt[p.rm.row(m_base + r) * d + c] : 0.0;
+    sm.wblk[r][c] = (r < rows_here) ? p.Wt[p.rm.row(m_base + r) * d + c] : 0.0;
   }
+  for (int idx = tid; idx < RS_STAGES * 8 * RS_LDE; idx += RS_THREADS)
+    sm.ring[idx / (8 * RS_LDE)].Eb[(idx / RS_LDE) % 8][idx % RS_LDE] = 0.0;
+  bar_all();
 
-  unsigned int n_near = 0, n_clamp = 0;
-  for (int b = 0; b < p.nblk; ++b) {
-    const int c0 = b * 128;
-    // diagonal block of U for the panel
-    for (int idx = tid; idx < 128 * 32; idx += RS_THREADS) {
-      const int j = idx >> 5, c4 = (idx & 31) * 4;
-      *reinterpret_cast<float4*>(sm.sU + j * 128 + c4) =
-          *reinterpret_cast<const float4*>(U + (long long)(c0 + j) * d + c0 + c4);
-    }
-    __syncthreads();
-
-    if (warp < 8) {
-      // ------------------------- panel: row `warp`, columns c0 .. c0+127 -------------------------
-      const bool valid = (r_first + warp) < p.rows_per_unit;
-      const long long grow = valid ? p.rm.row(m_base + warp) : 0;
+  if (warp < 8) {
+    // =========================== panel warps: row `warp` ===========================
+    const bool valid = warp < rows_here;
+    const long long grow = valid ? p.rm.row(m_base + warp) : 0;
+    const double magic = 6755399441055744.0;  // 1.5 * 2^52: adding it rounds to an integer, ties to even
+    unsigned int n_near = 0, n_clamp = 0;
+    for (int b = 0; b < p.nblk; ++b) {
+      const int c0 = b * 128;
+      for (int idx = tid; idx < 128 * 32; idx += 256) {
+        const int j = idx >> 5, c4 = (idx & 31) * 4;
+        *reinterpret_cast<float4*>(sm.sU + j * 128 + c4) =
+            *reinterpret_cast<const float4*>(U + (long long)(c0 + j) * d + c0 + c4);
+      }
+      asm volatile("bar.sync 2, 256;" ::: "memory");
       double w[4];
 #pragma unroll
       for (int sb = 0; sb < 4; ++sb) w[sb] = sm.wblk[warp][sb * 32 + lane];
@@ -542,21 +545,23 @@ __global__ void __launch_bounds__(RS_THREADS, 1) k_sweep_rows(RowSweepP p) {
         const double rs_l = 1.0 / s_l;
         const double rd_l = 1.0 / (double)sm.sU[cl * 128 + cl];
         const double srd_l = s_l * rd_l;
+        const double zm_l = z_l + magic, hi_l = magic + maxq;
         float u[32];
 #pragma unroll
         for (int j = 0; j < 32; ++j) u[j] = sm.sU[(sb * 32 + j) * 128 + cl];
         double v = (sb == 0) ? w[0] : (sb == 1) ? w[1] : (sb == 2) ? w[2] : w[3];
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
+          // e = (v - s (q - z)) / U_jj = (v + s z) / U_jj - (s / U_jj) q, with q = clamp(rne(v / s + z)):
+          // the fused multiply-add into z + 1.5 * 2^52 performs the rounding itself
           const double ard = fma(s_l, z_l, v) * rd_l;
-          double q = rne(fma(v, rs_l, z_l));
-          q = fmin(fmax(q, 0.0), maxq);
-          const double e = fma(-srd_l, q, ard);
+          const double qm = fmin(fmax(fma(v, rs_l, zm_l), magic), hi_l);
+          const double e = fma(-srd_l, qm - magic, ard);
           const double ej = shfl_d(e, j);
           if (lane > j) v = fma(-ej, (double)u[j], v);
         }
         const double x = fma(v, rs_l, z_l);
-        const double xr = rne(x);
+        const double xr = fma(v, rs_l, zm_l) - magic;
         const double q = fmin(fmax(xr, 0.0), maxq);
         const double e_mine = fma(-srd_l, q, fma(s_l, z_l, v) * rd_l);
         sm.Es[warp][cl] = valid ? e_mine : 0.0;
@@ -569,86 +574,103 @@ __global__ void __launch_bounds__(RS_THREADS, 1) k_sweep_rows(RowSweepP p) {
           if (xr != q) ++n_clamp;
         }
         // the sub-block's errors update the later sub-blocks of this block
-        for (int j = 0; j < 32; ++j) {
-          const double ej = shfl_d(e_mine, j);
-          const float* ur = sm.sU + (sb * 32 + j) * 128 + lane;
-          if (sb < 1) w[1] = fma(-ej, (double)ur[32], w[1]);
-          if (sb < 2) w[2] = fma(-ej, (double)ur[64], w[2]);
-          if (sb < 3) w[3] = fma(-ej, (double)ur[96], w[3]);
+        if (sb < 3) {
+#pragma unroll 4
+          for (int j = 0; j < 32; ++j) {
+            const double ej = shfl_d(e_mine, j);
+            const float* ur = sm.sU + (sb * 32 + j) * 128 + lane;
+            if (sb < 1) w[1] = fma(-ej, (double)ur[32], w[1]);
+            if (sb < 2) w[2] = fma(-ej, (double)ur[64], w[2]);
+            w[3] = fma(-ej, (double)ur[96], w[3]);
+          }
         }
       }
-    } else if (b + 1 < p.nblk) {
-      // ------------------------- update warps: part of block b+1 from blocks < b -------------------------
-      const int uw = warp - 8, ut = tid - 256;
-      const int cn = c0 + 128;     // first column of block b+1
-      const int nchunk = 4 * b;    // 32-row chunks of U[0 : 128 b, block b+1]
-      double acc[16][2];
+      bar_all();  // block b is quantized: its errors are in Es and in the history
+      bar_all();  // block b+1 has been handed over in wblk
+    }
+    if (p.stats) {
+      n_near = __reduce_add_sync(0xffffffffu, n_near);
+      n_clamp = __reduce_add_sync(0xffffffffu, n_clamp);
+      if (lane == 0) {
+        if (n_near) atomicAdd(&p.stats->near_tie_codes, (unsigned long long)n_near);
+        if (n_clamp) atomicAdd(&p.stats->clamped_codes, (unsigned long long)n_clamp);
+        if (blockIdx.x == 0 && warp == 0) atomicAdd(&p.stats->column_steps, (unsigned long long)d);
+      }
+    }
+    return;
+  }
+
+  // =========================== update warps ===========================
+  const int uw = warp - 8, ut = tid - 256;
+  const int fr = lane >> 2, fk = lane & 3;   // fragment row / k (and column-pair) index of this lane
+  const bool fr_valid = fr < rows_here;
+  const long long fr_grow = fr_valid ? p.rm.row(m_base + fr) : 0;
+  const int n_lo = uw * 16;                  // this warp owns columns n_lo .. n_lo+15 of the target block
+  for (int b = 0; b < p.nblk; ++b) {
+    if (b + 1 >= p.nblk) {  // nothing left to prepare
+      bar_all();
+      bar_all();
+      break;
+    }
+    const int cn = (b + 1) * 128;            // first column of the target block
+    const int n_hist = 4 * b;                // chunks whose errors come from the history (blocks < b)
+    const int n_all = n_hist + 4;            // plus the four chunks of block b itself
+    double acc[2][2][2];
 #pragma unroll
-      for (int nt = 0; nt < 16; ++nt) acc[nt][0] = acc[nt][1] = 0.0;
-      auto issue = [&](int c) {
-        if (c < nchunk) {
-          float* dst = &sm.ring[c % RS_STAGES][0][0];
+    for (int i = 0; i < 8; ++i) (&acc[0][0][0])[i] = 0.0;
+    // the block's own weights, needed at the end
+    double w0[2][2];
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const int piece = ut + 256 * i;  // 0 .. 1023 : row = piece / 32, 16-byte piece = piece % 32
-            const int r = piece >> 5, q4 = (piece & 31) * 4;
-            const float* src = U + (long long)(c * RS_CHUNK + r) * d + cn + q4;
-            const unsigned int sa = (unsigned int)__cvta_generic_to_shared(dst + r * RS_LDB + q4);
+    for (int t = 0; t < 2; ++t)
+#pragma unroll
+      for (int e = 0; e < 2; ++e)
+        w0[t][e] = fr_valid ? p.Wt[fr_grow * d + cn + n_lo + t * 8 + 2 * fk + e] : 0.0;
+
+    auto issue = [&](int c) {
+      if (c < n_all) {
+        RowSweepStage& st = sm.ring[c % RS_STAGES];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int piece = ut + 256 * i;  // row = piece / 32, 16-byte piece = piece % 32
+          const int r = piece >> 5, q4 = (piece & 31) * 4;
+          const float* src = U + (long long)(c * RS_CHUNK + r) * d + cn + q4;
+          const unsigned int sa = (unsigned int)__cvta_generic_to_shared(&st.Ub[r][q4]);
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sa), "l"(src) : "memory");
+        }
+        if (c < n_hist && ut < 128) {
+          const int r = ut >> 4, q2 = (ut & 15) * 2;  // 8 rows x 16 pieces of two doubles
+          if (r < rows_here) {
+            const double* src = p.ErrG + (long long)(m_base + r) * d + c * RS_CHUNK + q2;
+            const unsigned int sa = (unsigned int)__cvta_generic_to_shared(&st.Eb[r][q2]);
             asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sa), "l"(src) : "memory");
           }
         }
-        asm volatile("cp.async.commit_group;" ::: "memory");
-      };
-      for (int c = 0; c < RS_STAGES - 1; ++c) issue(c);
-      const double* erow = p.ErrG + (long long)(m_base + fr) * d + 4 * uw + fk;
-      double a_next = (fr_valid && nchunk > 0) ? erow[0] : 0.0;
-      for (int c = 0; c < nchunk; ++c) {
-        asm volatile("cp.async.wait_group %0;" ::"n"(RS_STAGES - 2) : "memory");
-        asm volatile("bar.sync 1, 256;" ::: "memory");
-        issue(c + RS_STAGES - 1);
-        const double a = a_next;
-        if (c + 1 < nchunk) a_next = fr_valid ? erow[(c + 1) * RS_CHUNK] : 0.0;
-        const float* bp = &sm.ring[c % RS_STAGES][4 * uw + fk][fr];
-#pragma unroll
-        for (int nt = 0; nt < 16; ++nt) mma_f64(acc[nt], a, (double)bp[nt * 8]);
       }
-      asm volatile("cp.async.wait_group 0;" ::: "memory");
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    for (int c = 0; c < RS_STAGES - 1; ++c) issue(c);
+    for (int c = 0; c < n_all; ++c) {
+      if (c == n_hist) bar_all();  // the panel warps have finished block b: Es is complete
+      asm volatile("cp.async.wait_group %0;" ::"n"(RS_STAGES - 2) : "memory");
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      issue(c + RS_STAGES - 1);
+      const RowSweepStage& st = sm.ring[c % RS_STAGES];
+      const double* ap = (c < n_hist) ? &st.Eb[fr][fk] : &sm.Es[fr][(c - n_hist) * RS_CHUNK + fk];
+      const float* bp = &st.Ub[fk][n_lo + fr];
 #pragma unroll
-      for (int nt = 0; nt < 16; ++nt) {
-        sm.red[uw][fr][nt * 8 + 2 * fk] = acc[nt][0];
-        sm.red[uw][fr][nt * 8 + 2 * fk + 1] = acc[nt][1];
+      for (int q = 0; q < 8; ++q) {
+        const double a = ap[4 * q];
+        mma_f64(acc[0][q & 1], a, (double)bp[4 * q * RS_LDB]);
+        mma_f64(acc[1][q & 1], a, (double)bp[4 * q * RS_LDB + 8]);
       }
     }
-    __syncthreads();
-
-    if (b + 1 < p.nblk) {
-      // ------------------------- last 128 terms and hand-over of block b+1 -------------------------
-      // warp `warp` owns the 8 columns cn + 8 warp .. +7 for all 8 rows
-      const int cn = c0 + 128, nt = warp;
-      double acc[2] = {0.0, 0.0};
-      const float* ub = U + (long long)(c0 + fk) * d + cn + nt * 8 + fr;
-#pragma unroll 8
-      for (int q = 0; q < 32; ++q) mma_f64(acc, sm.Es[fr][4 * q + fk], (double)ub[(long long)(4 * q) * d]);
-      const int cc = nt * 8 + 2 * fk;
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
 #pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        double t = 0.0;
+    for (int t = 0; t < 2; ++t)
 #pragma unroll
-        for (int w8 = 0; w8 < 8; ++w8) t += sm.red[w8][fr][cc + e];
-        const double w0 = fr_valid ? p.Wt[fr_grow * d + cn + cc + e] : 0.0;
-        sm.wblk[fr][cc + e] = (w0 - t) - acc[e];
-      }
-    }
-    __syncthreads();
-  }
-  if (p.stats && warp < 8) {
-    n_near = __reduce_add_sync(0xffffffffu, n_near);
-    n_clamp = __reduce_add_sync(0xffffffffu, n_clamp);
-    if (lane == 0) {
-      if (n_near) atomicAdd(&p.stats->near_tie_codes, (unsigned long long)n_near);
-      if (n_clamp) atomicAdd(&p.stats->clamped_codes, (unsigned long long)n_clamp);
-      if (blockIdx.x == 0 && warp == 0) atomicAdd(&p.stats->column_steps, (unsigned long long)d);
-    }
+      for (int e = 0; e < 2; ++e)
+        sm.wblk[fr][n_lo + t * 8 + 2 * fk + e] = w0[t][e] - (acc[t][0][e] + acc[t][1][e]);
+    bar_all();  // block b+1 handed over
   }
 }
 
