@@ -528,35 +528,51 @@ __global__ void __launch_bounds__(RS_THREADS, 1) k_sweep_rows(RowSweepP p) {
     unsigned int n_near = 0, n_clamp = 0;
     for (int b = 0; b < p.nblk; ++b) {
       const int c0 = b * 128;
+      // grids of this lane's four columns (fetched while the diagonal block is staged)
+      double s4[4], z4[4];
+#pragma unroll
+      for (int sb = 0; sb < 4; ++sb) {
+        const long long so = grow * p.ng + (c0 + sb * 32 + lane) / p.seg;
+        s4[sb] = valid ? p.sD[so] : 1.0;
+        z4[sb] = valid ? (double)p.z[so] : 0.0;
+      }
       for (int idx = tid; idx < 128 * 32; idx += 256) {
         const int j = idx >> 5, c4 = (idx & 31) * 4;
         *reinterpret_cast<float4*>(sm.sU + j * 128 + c4) =
             *reinterpret_cast<const float4*>(U + (long long)(c0 + j) * d + c0 + c4);
       }
       asm volatile("bar.sync 2, 256;" ::: "memory");
-      double w[4];
+      double w[4], rs4[4], rd4[4];
 #pragma unroll
-      for (int sb = 0; sb < 4; ++sb) w[sb] = sm.wblk[warp][sb * 32 + lane];
+      for (int sb = 0; sb < 4; ++sb) {
+        w[sb] = sm.wblk[warp][sb * 32 + lane];
+        rs4[sb] = 1.0 / s4[sb];
+        rd4[sb] = 1.0 / (double)sm.sU[(sb * 32 + lane) * 129];
+      }
 #pragma unroll 1
       for (int sb = 0; sb < 4; ++sb) {
         const int cl = sb * 32 + lane, col = c0 + cl;
-        const long long so = grow * p.ng + col / p.seg;
-        const double s_l = valid ? p.sD[so] : 1.0, z_l = valid ? (double)p.z[so] : 0.0;
-        const double rs_l = 1.0 / s_l;
-        const double rd_l = 1.0 / (double)sm.sU[cl * 128 + cl];
+        const double s_l = (sb == 0) ? s4[0] : (sb == 1) ? s4[1] : (sb == 2) ? s4[2] : s4[3];
+        const double z_l = (sb == 0) ? z4[0] : (sb == 1) ? z4[1] : (sb == 2) ? z4[2] : z4[3];
+        const double rs_l = (sb == 0) ? rs4[0] : (sb == 1) ? rs4[1] : (sb == 2) ? rs4[2] : rs4[3];
+        const double rd_l = (sb == 0) ? rd4[0] : (sb == 1) ? rd4[1] : (sb == 2) ? rd4[2] : rd4[3];
         const double srd_l = s_l * rd_l;
-        const double zm_l = z_l + magic, hi_l = magic + maxq;
+        const double zm_l = z_l + magic;
         float u[32];
 #pragma unroll
         for (int j = 0; j < 32; ++j) u[j] = sm.sU[(sb * 32 + j) * 128 + cl];
         double v = (sb == 0) ? w[0] : (sb == 1) ? w[1] : (sb == 2) ? w[2] : w[3];
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
-          // e = (v - s (q - z)) / U_jj = (v + s z) / U_jj - (s / U_jj) q, with q = clamp(rne(v / s + z)):
-          // the fused multiply-add into z + 1.5 * 2^52 performs the rounding itself
+          // e = (v - s (q - z)) / U_jj = (v + s z) / U_jj - (s / U_jj) q, with q = clamp(rne(v / s + z)).
+          // The fused multiply-add into z + 1.5 * 2^52 performs the rounding itself and leaves the
+          // integer in the low word of the result (|v / s + z| < 2^31 assumed), where the clamp is
+          // two integer instructions instead of two slow double-precision min / max.
           const double ard = fma(s_l, z_l, v) * rd_l;
-          const double qm = fmin(fmax(fma(v, rs_l, zm_l), magic), hi_l);
-          const double e = fma(-srd_l, qm - magic, ard);
+          int n = __double2loint(fma(v, rs_l, zm_l));
+          n = min(max(n, 0), p.maxq);
+          const double q = __hiloint2double(0x43380000, n) - magic;
+          const double e = fma(-srd_l, q, ard);
           const double ej = shfl_d(e, j);
           if (lane > j) v = fma(-ej, (double)u[j], v);
         }
