@@ -17,6 +17,7 @@
 // different decision changes every later code of its row.
 #include "tb_common.cuh"
 #include "tb_gemm.cuh"
+#include "tb_tma.cuh"
 
 namespace tb {
 
@@ -462,13 +463,17 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) k_sweep_block(SweepP p) {
 // the 128 columns of a block strictly in order); warps 8-15 are the update
 // warps (two 8-column fragments each, on the FP64 tensor pipe).  While the
 // panel warps walk block b, the update warps form the part of block b+1's sum
-// that needs only blocks < b, streaming 32-row chunks of U and of the error
-// history through a cp.async ring; when the panel is done they add the last
-// 128 terms (errors of block b straight from shared memory) and hand block b+1
-// over.  Synchronisation is by hardware barriers only (ids 1-3, fixed
-// participant counts); every trip count depends on the block index alone.
+// that needs only blocks < b: 64-row chunks of U and of the error history
+// arrive by TMA (one box each, 8 spare columns per row so that fragment loads
+// are free of bank conflicts) in a 3-stage ring guarded by full / empty
+// mbarriers; when the panel is done they add the last 128 terms (errors of
+// block b straight from shared memory) and hand block b+1 over.  The two warp
+// groups meet at hardware barriers with fixed participant counts; every trip
+// count depends on the block index alone.  mbarrier waits are bounded: when a
+// bound runs out the kernel raises a device error word and stops computing, but
+// still passes every barrier, so it always terminates.
 // ---------------------------------------------------------------------------
-enum { RS_THREADS = 512, RS_STAGES = 7, RS_LDB = 136, RS_LDE = 36, RS_CHUNK = 32, RS_LDW = 132 };
+enum { RS_THREADS = 512, RS_STAGES = 3, RS_LDB = 136, RS_LDE = 68, RS_CHUNK = 64, RS_LDW = 132 };
 struct RowSweepP {
   const double* Wt;      // [d_out][d] current W~ (rows of the step are read, never written)
   const float* U;        // [n_hin][d][d]
@@ -482,15 +487,18 @@ struct RowSweepP {
   int units, rows_per_unit, ctas_per_unit;
 };
 struct RowSweepStage {
-  float Ub[RS_CHUNK][RS_LDB];   // 32 rows of U, 128 columns of the target block
-  double Eb[8][RS_LDE];         // the same 32 columns of the error history, 8 rows
+  float Ub[RS_CHUNK][RS_LDB];   // 64 rows of U: 128 columns of the target block + 8 spare
+  double Eb[8][RS_LDE];         // the same 64 columns of the error history (+ 4 spare), 8 rows
 };
 struct RowSweepSmem {
   float sU[128 * 128];          // diagonal block of U
   RowSweepStage ring[RS_STAGES];
   double wblk[8][RS_LDW];       // arrival values of the current block
   double Es[8][RS_LDW];         // normalised errors of the current block
+  unsigned long long full_bar[RS_STAGES], empty_bar[RS_STAGES];
+  int abort_flag;
 };
+__device__ int g_sweep_error = 0;
 
 __device__ __forceinline__ void mma_f64(double (&c)[2], double a, double b) {
   asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
@@ -499,8 +507,9 @@ __device__ __forceinline__ void mma_f64(double (&c)[2], double a, double b) {
 }
 __device__ __forceinline__ void bar_all() { asm volatile("bar.sync 3, 512;" ::: "memory"); }
 
-__global__ void __launch_bounds__(RS_THREADS, 1) k_sweep_rows(RowSweepP p) {
-  extern __shared__ __align__(16) unsigned char rs_raw[];
+__global__ void __launch_bounds__(RS_THREADS, 1)
+    k_sweep_rows(RowSweepP p, const __grid_constant__ CUtensorMap map_u, const __grid_constant__ CUtensorMap map_e) {
+  extern __shared__ __align__(128) unsigned char rs_raw[];
   RowSweepSmem& sm = *reinterpret_cast<RowSweepSmem*>(rs_raw);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int unit = blockIdx.x / p.ctas_per_unit;
@@ -516,8 +525,14 @@ __global__ void __launch_bounds__(RS_THREADS, 1) k_sweep_rows(RowSweepP p) {
     const int r = idx >> 7, c = idx & 127;
     sm.wblk[r][c] = (r < rows_here) ? p.Wt[p.rm.row(m_base + r) * d + c] : 0.0;
   }
-  for (int idx = tid; idx < RS_STAGES * 8 * RS_LDE; idx += RS_THREADS)
-    sm.ring[idx / (8 * RS_LDE)].Eb[(idx / RS_LDE) % 8][idx % RS_LDE] = 0.0;
+  if (tid == 0) {
+    for (int s = 0; s < RS_STAGES; ++s) {
+      mbar_init(smem_u32(&sm.full_bar[s]), 1);
+      mbar_init(smem_u32(&sm.empty_bar[s]), 8);  // one arrival per update warp
+    }
+    sm.abort_flag = 0;
+    mbar_fence_init();
+  }
   bar_all();
 
   if (warp < 8) {
@@ -601,6 +616,8 @@ __global__ void __launch_bounds__(RS_THREADS, 1) k_sweep_rows(RowSweepP p) {
           }
         }
       }
+      // the error history is read back by TMA (async proxy): order these stores before it
+      asm volatile("fence.proxy.async;" ::: "memory");
       bar_all();  // block b is quantized: its errors are in Es and in the history
       bar_all();  // block b+1 has been handed over in wblk
     }
@@ -617,11 +634,19 @@ __global__ void __launch_bounds__(RS_THREADS, 1) k_sweep_rows(RowSweepP p) {
   }
 
   // =========================== update warps ===========================
-  const int uw = warp - 8, ut = tid - 256;
-  const int fr = lane >> 2, fk = lane & 3;   // fragment row / k (and column-pair) index of this lane
+  const int uw = warp - 8;
+  const int fr = lane >> 2, fk = lane & 3;   // fragment row / k (and column) index of this lane
   const bool fr_valid = fr < rows_here;
   const long long fr_grow = fr_valid ? p.rm.row(m_base + fr) : 0;
-  const int n_lo = uw * 16;                  // this warp owns columns n_lo .. n_lo+15 of the target block
+  // This warp owns columns n_lo .. n_lo+15 of the target block: fragment 0 the even ones,
+  // fragment 1 the odd ones, so that one 8-byte load feeds both.
+  const int n_lo = uw * 16;
+  volatile int* abort_flag = &sm.abort_flag;
+  const bool producer = (uw == 0 && lane == 0);
+  const int u_row0 = unit * d * (p.units > 1 ? 1 : 0);
+  // ring positions: `c_*` of the consumers (all update warps), `p_*` of the producer thread
+  int c_slot = 0, p_slot = 0;
+  uint32_t c_phase = 0, p_phase = 0;
   for (int b = 0; b < p.nblk; ++b) {
     if (b + 1 >= p.nblk) {  // nothing left to prepare
       bar_all();
@@ -629,65 +654,79 @@ __global__ void __launch_bounds__(RS_THREADS, 1) k_sweep_rows(RowSweepP p) {
       break;
     }
     const int cn = (b + 1) * 128;            // first column of the target block
-    const int n_hist = 4 * b;                // chunks whose errors come from the history (blocks < b)
-    const int n_all = n_hist + 4;            // plus the four chunks of block b itself
+    const int n_hist = 2 * b;                // chunks whose errors come from the history (blocks < b)
+    const int n_all = n_hist + 2;            // plus the two chunks of block b itself
     double acc[2][2][2];
 #pragma unroll
     for (int i = 0; i < 8; ++i) (&acc[0][0][0])[i] = 0.0;
-    // the block's own weights, needed at the end
+    // the block's own weights, needed at the end: tile-column ci = 2 fk + e is column n_lo + 2 ci + t
     double w0[2][2];
 #pragma unroll
     for (int t = 0; t < 2; ++t)
 #pragma unroll
       for (int e = 0; e < 2; ++e)
-        w0[t][e] = fr_valid ? p.Wt[fr_grow * d + cn + n_lo + t * 8 + 2 * fk + e] : 0.0;
+        w0[t][e] = fr_valid ? p.Wt[fr_grow * d + cn + n_lo + 2 * (2 * fk + e) + t] : 0.0;
 
-    auto issue = [&](int c) {
+    auto produce = [&](int c) {   // producer thread only
       if (c < n_all) {
-        RowSweepStage& st = sm.ring[c % RS_STAGES];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const int piece = ut + 256 * i;  // row = piece / 32, 16-byte piece = piece % 32
-          const int r = piece >> 5, q4 = (piece & 31) * 4;
-          const float* src = U + (long long)(c * RS_CHUNK + r) * d + cn + q4;
-          const unsigned int sa = (unsigned int)__cvta_generic_to_shared(&st.Ub[r][q4]);
-          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sa), "l"(src) : "memory");
+        RowSweepStage& st = sm.ring[p_slot];
+        const uint32_t fb = smem_u32(&sm.full_bar[p_slot]);
+        if (mbar_wait(smem_u32(&sm.empty_bar[p_slot]), p_phase ^ 1u, abort_flag, &g_sweep_error)) {
+          const bool hist = c < n_hist;
+          mbar_expect_tx(fb, (uint32_t)(sizeof(st.Ub) + (hist ? sizeof(st.Eb) : 0)));
+          tma_load_2d(smem_u32(&st.Ub[0][0]), &map_u, cn, u_row0 + c * RS_CHUNK, fb);
+          if (hist) tma_load_2d(smem_u32(&st.Eb[0][0]), &map_e, c * RS_CHUNK, m_base, fb);
         }
-        if (c < n_hist && ut < 128) {
-          const int r = ut >> 4, q2 = (ut & 15) * 2;  // 8 rows x 16 pieces of two doubles
-          if (r < rows_here) {
-            const double* src = p.ErrG + (long long)(m_base + r) * d + c * RS_CHUNK + q2;
-            const unsigned int sa = (unsigned int)__cvta_generic_to_shared(&st.Eb[r][q2]);
-            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sa), "l"(src) : "memory");
-          }
+        if (++p_slot == RS_STAGES) {
+          p_slot = 0;
+          p_phase ^= 1u;
         }
       }
-      asm volatile("cp.async.commit_group;" ::: "memory");
     };
-    for (int c = 0; c < RS_STAGES - 1; ++c) issue(c);
+    if (producer) {
+      produce(0);
+      produce(1);
+    }
     for (int c = 0; c < n_all; ++c) {
       if (c == n_hist) bar_all();  // the panel warps have finished block b: Es is complete
-      asm volatile("cp.async.wait_group %0;" ::"n"(RS_STAGES - 2) : "memory");
-      asm volatile("bar.sync 1, 256;" ::: "memory");
-      issue(c + RS_STAGES - 1);
-      const RowSweepStage& st = sm.ring[c % RS_STAGES];
-      const double* ap = (c < n_hist) ? &st.Eb[fr][fk] : &sm.Es[fr][(c - n_hist) * RS_CHUNK + fk];
-      const float* bp = &st.Ub[fk][n_lo + fr];
+      const RowSweepStage& st = sm.ring[c_slot];
+      const bool ok = mbar_wait(smem_u32(&sm.full_bar[c_slot]), c_phase, abort_flag, &g_sweep_error);
+      if (ok) {
+        const double* ap = (c < n_hist) ? &st.Eb[fr][fk] : &sm.Es[fr][(c - n_hist) * RS_CHUNK + fk];
+        const float* bp = &st.Ub[fk][n_lo + 2 * fr];
 #pragma unroll
-      for (int q = 0; q < 8; ++q) {
-        const double a = ap[4 * q];
-        mma_f64(acc[0][q & 1], a, (double)bp[4 * q * RS_LDB]);
-        mma_f64(acc[1][q & 1], a, (double)bp[4 * q * RS_LDB + 8]);
+        for (int q = 0; q < 16; ++q) {
+          const double a = ap[4 * q];
+          const float2 bb = *reinterpret_cast<const float2*>(bp + 4 * q * RS_LDB);
+          mma_f64(acc[0][q & 1], a, (double)bb.x);
+          mma_f64(acc[1][q & 1], a, (double)bb.y);
+        }
       }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&sm.empty_bar[c_slot]));  // this warp is done with the stage
+      if (++c_slot == RS_STAGES) {
+        c_slot = 0;
+        c_phase ^= 1u;
+      }
+      if (producer) produce(c + 2);
     }
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
 #pragma unroll
     for (int t = 0; t < 2; ++t)
 #pragma unroll
       for (int e = 0; e < 2; ++e)
-        sm.wblk[fr][n_lo + t * 8 + 2 * fk + e] = w0[t][e] - (acc[t][0][e] + acc[t][1][e]);
+        sm.wblk[fr][n_lo + 2 * (2 * fk + e) + t] = w0[t][e] - (acc[t][0][e] + acc[t][1][e]);
     bar_all();  // block b+1 handed over
   }
+}
+
+int sweep_error_read_clear() {
+  int v = 0;
+  if (cudaMemcpyFromSymbol(&v, g_sweep_error, sizeof(int)) != cudaSuccess) return -1;
+  if (v) {
+    int z = 0;
+    cudaMemcpyToSymbol(g_sweep_error, &z, sizeof(int));
+  }
+  return v;
 }
 
 // E[m][k] = W~[row(m)][k] - s (code - z): the quantization error of the group on
@@ -1098,8 +1137,14 @@ static tb_status run_sweep_rows(const Plan& p, const float* U_in, unsigned char*
   sp.ctas_per_unit = (sp.rows_per_unit + 7) / 8;
   static bool configured[64] = {false};
   TB_TRY(allow_smem(k_sweep_rows, sizeof(RowSweepSmem), configured));
+  CUtensorMap map_u, map_e;
+  const unsigned box_u = (unsigned)((p.d >= RS_LDB) ? RS_LDB : p.d), box_e = (unsigned)((p.d >= RS_LDE) ? RS_LDE : p.d);
+  TB_TRY(make_map_2d(&map_u, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, sizeof(float), U_in, (unsigned long long)p.d,
+                     (unsigned long long)p.d * sp.units, box_u, RS_CHUNK, CU_TENSOR_MAP_SWIZZLE_NONE));
+  TB_TRY(make_map_2d(&map_e, CU_TENSOR_MAP_DATA_TYPE_FLOAT64, sizeof(double), sp.ErrG, (unsigned long long)p.d,
+                     (unsigned long long)M, box_e, 8, CU_TENSOR_MAP_SWIZZLE_NONE));
   const long long ctas = (long long)sp.ctas_per_unit * sp.units;
-  k_sweep_rows<<<(unsigned)ctas, RS_THREADS, sizeof(RowSweepSmem), st>>>(sp);
+  k_sweep_rows<<<(unsigned)ctas, RS_THREADS, sizeof(RowSweepSmem), st>>>(sp, map_u, map_e);
   TB_LAUNCH_CHECK();
   return TB_OK;
 }

@@ -20,9 +20,8 @@
 // MMA issuer.  Every wait on an mbarrier is bounded; when a bound runs out the
 // kernel raises a device error word, leaves its loops, frees its tensor memory
 // and returns.
-#include <cuda.h>
-
 #include "tb_common.cuh"
+#include "tb_tma.cuh"
 
 namespace tb {
 
@@ -41,51 +40,6 @@ enum {
 };
 
 __device__ int g_tc_error = 0;
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait: gives up after about two seconds, raises the error words and reports failure.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  const long long t0 = clock64();
-  while (!mbar_try_wait(bar, parity)) {
-    if (*abort_flag) return false;
-    if (clock64() - t0 > 4000000000ll) {
-      *abort_flag = 1;
-      atomicExch(&g_tc_error, 1);
-      return false;
-    }
-  }
-  return true;
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
-      "l"(map), "r"(x), "r"(y), "r"(bar)
-      : "memory");
-}
 
 // MN-major, SWIZZLE_128B shared-memory matrix descriptor (see the file header).
 __device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t addr) {
@@ -156,7 +110,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
       mbar_init(acce_bar(b), 8);  // one arrival per epilogue warp
     }
     *abort_flag = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_fence_init();
   }
   if (warp == 8) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512u)
@@ -197,7 +151,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
         for (int st = 0; st < n_stages; ++st, ++it) {
           const int s = it % TC_STAGES;
           const uint32_t ph = (it / TC_STAGES) & 1u;
-          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) break;
+          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, &g_tc_error)) break;
           mbar_expect_tx(full_bar(s), TC_STAGE_BYTES);
           const uint32_t sa = base + s * TC_STAGE_BYTES, sb = sa + TC_A_BYTES;
           const int k0 = st * TC_BK;
@@ -219,12 +173,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
           const int b = chunk_it & 1;
           if (in_chunk == 0) {
             // the accumulator buffer must have been drained by the epilogue warps
-            if (!mbar_wait(acce_bar(b), ((chunk_it >> 1) & 1u) ^ 1u, abort_flag)) break;
+            if (!mbar_wait(acce_bar(b), ((chunk_it >> 1) & 1u) ^ 1u, abort_flag, &g_tc_error)) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           }
           const int s = it % TC_STAGES;
           const uint32_t ph = (it / TC_STAGES) & 1u;
-          if (!mbar_wait(full_bar(s), ph, abort_flag)) break;
+          if (!mbar_wait(full_bar(s), ph, abort_flag, &g_tc_error)) break;
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint32_t sa = base + s * TC_STAGE_BYTES, sb = sa + TC_A_BYTES;
           const uint32_t tmem_d = tmem_base + (uint32_t)b * TC_BN;
@@ -257,7 +211,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
       bool ok = true;
       for (int st0 = 0; st0 < n_stages && ok; st0 += TC_CHUNK, ++chunk_it) {
         const int b = chunk_it & 1;
-        ok = mbar_wait(accf_bar(b), (chunk_it >> 1) & 1u, abort_flag);
+        ok = mbar_wait(accf_bar(b), (chunk_it >> 1) & 1u, abort_flag, &g_tc_error);
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * TC_BN + hf * 128);
@@ -295,37 +249,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
   }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
-        qres == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(p);
-  }
-  return fn;
-}
-
 // H += X^T X for bf16 X on the tensor cores: tiles on or below the diagonal
 // (128-row blocks x 256-column blocks); the caller mirrors the rest.
 tb_status syrk_bf16_tensor(float* H, const __nv_bfloat16* X, long long n_tok, int d, cudaStream_t st) {
-  EncodeTiledFn enc = encode_fn();
-  if (!enc) return TB_ERR_CUDA;
   if (n_tok > 0x7fffffffll) return TB_ERR_UNSUPPORTED;
   CUtensorMap map;
-  const cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)n_tok};
-  const cuuint64_t strides[1] = {(cuuint64_t)d * sizeof(__nv_bfloat16)};
-  const cuuint32_t box[2] = {64, 64};
-  const cuuint32_t estr[2] = {1, 1};
-  if (enc(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(X), dims, strides, box, estr,
-          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-    return TB_ERR_CUDA;
+  TB_TRY(make_map_2d(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, sizeof(__nv_bfloat16), X, (unsigned long long)d,
+                     (unsigned long long)n_tok, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B));
   const int m_blocks = (d + TC_BM - 1) / TC_BM;
   int n_tiles = 0;
   for (int mi = 0; mi < m_blocks; ++mi) n_tiles += mi / 2 + 1;
@@ -347,6 +277,10 @@ tb_status syrk_bf16_tensor(float* H, const __nv_bfloat16* X, long long n_tok, in
 }  // namespace tb
 
 // 0, or 1 once a bounded wait inside a tensor-core kernel has run out (sticky until read).
+namespace tb {
+int sweep_error_read_clear();  // the same word of the column-sweep kernel (tb_quantize.cu)
+}
+
 extern "C" int tb_device_error_flag(void) {
   int v = 0;
   if (cudaMemcpyFromSymbol(&v, tb::g_tc_error, sizeof(int)) != cudaSuccess) return -1;
@@ -354,5 +288,7 @@ extern "C" int tb_device_error_flag(void) {
     int z = 0;
     cudaMemcpyToSymbol(tb::g_tc_error, &z, sizeof(int));
   }
-  return v;
+  const int w = tb::sweep_error_read_clear();
+  if (w < 0) return -1;
+  return (v || w) ? 1 : 0;
 }

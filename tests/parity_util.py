@@ -91,6 +91,7 @@ def run_gpu(prob, bits, quant_group, out_block, flags, n_cand=16, cd_iters=1, wa
     res = tb.tb_quantize_layer(desc, t(prob["W"]), t(prob["Hin"]), t(prob["Uin"]), t(prob["Hout"]),
                                t(prob["Uout"]), t(prob["R"]), t(prob["P"]), t(prob["C"]), want_loss=want_loss)
     torch.cuda.synchronize()
+    assert tb.tb_device_error_flag() == 0, "a bounded device-side wait ran out"
     return dict(codes=res.codes.cpu().numpy(), scales=res.scales.cpu().numpy(), zeros=res.zeros.cpu().numpy(),
                 cand=res.cand.cpu().numpy(), w_hat=res.w_hat.cpu().numpy(),
                 loss=None if res.loss is None else res.loss.cpu().numpy(), stats=res.stats_dict())
