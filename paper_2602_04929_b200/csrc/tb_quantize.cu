@@ -572,6 +572,7 @@ __global__ void __launch_bounds__(RS_THREADS, 1)
         const double rs_l = (sb == 0) ? rs4[0] : (sb == 1) ? rs4[1] : (sb == 2) ? rs4[2] : rs4[3];
         const double rd_l = (sb == 0) ? rd4[0] : (sb == 1) ? rd4[1] : (sb == 2) ? rd4[2] : rd4[3];
         const double srd_l = s_l * rd_l;
+        const double szrd_l = s_l * z_l * rd_l;
         const double zm_l = z_l + magic;
         float u[32];
 #pragma unroll
@@ -579,11 +580,11 @@ __global__ void __launch_bounds__(RS_THREADS, 1)
         double v = (sb == 0) ? w[0] : (sb == 1) ? w[1] : (sb == 2) ? w[2] : w[3];
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
-          // e = (v - s (q - z)) / U_jj = (v + s z) / U_jj - (s / U_jj) q, with q = clamp(rne(v / s + z)).
+          // e = (v - s (q - z)) / U_jj = (v / U_jj + s z / U_jj) - (s / U_jj) q, with q = clamp(rne(v / s + z)).
           // The fused multiply-add into z + 1.5 * 2^52 performs the rounding itself and leaves the
           // integer in the low word of the result (|v / s + z| < 2^31 assumed), where the clamp is
           // two integer instructions instead of two slow double-precision min / max.
-          const double ard = fma(s_l, z_l, v) * rd_l;
+          const double ard = fma(v, rd_l, szrd_l);
           int n = __double2loint(fma(v, rs_l, zm_l));
           n = min(max(n, 0), p.maxq);
           const double q = __hiloint2double(0x43380000, n) - magic;
@@ -594,7 +595,7 @@ __global__ void __launch_bounds__(RS_THREADS, 1)
         const double x = fma(v, rs_l, z_l);
         const double xr = fma(v, rs_l, zm_l) - magic;
         const double q = fmin(fmax(xr, 0.0), maxq);
-        const double e_mine = fma(-srd_l, q, fma(s_l, z_l, v) * rd_l);
+        const double e_mine = fma(-srd_l, q, fma(v, rd_l, szrd_l));  // the value broadcast at step `lane`
         sm.Es[warp][cl] = valid ? e_mine : 0.0;
         if (valid) {
           p.codes[grow * d + col] = (unsigned char)(int)q;
@@ -604,15 +605,29 @@ __global__ void __launch_bounds__(RS_THREADS, 1)
           if (fabs(x - (fl + 0.5)) < 1e-6 && a0 != a1) ++n_near;
           if (xr != q) ++n_clamp;
         }
-        // the sub-block's errors update the later sub-blocks of this block
-        if (sb < 3) {
-#pragma unroll 4
+        // the sub-block's errors update the later sub-blocks of this block (one branch-free loop
+        // per case, so that shuffles, loads and multiply-adds of different j overlap)
+        const float* ub = sm.sU + (sb * 32) * 128 + lane;
+        if (sb == 0) {
+#pragma unroll 8
           for (int j = 0; j < 32; ++j) {
             const double ej = shfl_d(e_mine, j);
-            const float* ur = sm.sU + (sb * 32 + j) * 128 + lane;
-            if (sb < 1) w[1] = fma(-ej, (double)ur[32], w[1]);
-            if (sb < 2) w[2] = fma(-ej, (double)ur[64], w[2]);
-            w[3] = fma(-ej, (double)ur[96], w[3]);
+            w[1] = fma(-ej, (double)ub[j * 128 + 32], w[1]);
+            w[2] = fma(-ej, (double)ub[j * 128 + 64], w[2]);
+            w[3] = fma(-ej, (double)ub[j * 128 + 96], w[3]);
+          }
+        } else if (sb == 1) {
+#pragma unroll 8
+          for (int j = 0; j < 32; ++j) {
+            const double ej = shfl_d(e_mine, j);
+            w[2] = fma(-ej, (double)ub[j * 128 + 64], w[2]);
+            w[3] = fma(-ej, (double)ub[j * 128 + 96], w[3]);
+          }
+        } else if (sb == 2) {
+#pragma unroll 8
+          for (int j = 0; j < 32; ++j) {
+            const double ej = shfl_d(e_mine, j);
+            w[3] = fma(-ej, (double)ub[j * 128 + 96], w[3]);
           }
         }
       }
