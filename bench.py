@@ -125,7 +125,8 @@ def count_launches(cfg, proj, n_tok: int, with_loss=True) -> int:
         n += 3                                          # G Hsum, per-head Gram, combine
     for (dd, nb) in ((d, 1),) + (((dh, H),) if proj.partner else ()):
         blocks = -(-dd // 64)
-        n += 1 + blocks + 3 * (blocks - 1) + 2 * (blocks - 1) + 1   # reverse, potrf, panel ops, inverse, reverse
+        levels = max(0, (blocks - 1).bit_length())
+        n += 1 + blocks + (blocks - 1) + 1 + 2 * levels * (nb if blocks > 2 and nb > 1 else 1) + 1   # reverse, panels, trailing updates, block inverses, doubling levels, reverse
     n += 1 + (1 if S > 1 else 0)                        # widen, compensation matrices
     n += (S if cfg.adaptive else 1)                     # grid
     n += S * (1 + nblk)                                 # gather + one launch per column block

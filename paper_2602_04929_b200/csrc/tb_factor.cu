@@ -8,14 +8,19 @@
 // No inverse of H is formed.  Everything runs in double: with cond(H_in) ~ 1e5
 // a float factorisation would lose most of U's digits.
 //
+// The matrix is embedded in a dp x dp one (dp = 64 * 2^k >= d, identity in the
+// padding) so that every block step below is uniform.
 //   1. A = J H J                                        (k_reverse_in)
-//   2. right-looking blocked Cholesky, 64-column panels:
-//        k_potrf64   factor the 64 x 64 diagonal block in shared memory and
-//                    invert it (forward substitution, one thread per column)
-//        GEMM        panel below the block  <- panel * inv(L_kk)^T
-//        GEMM        trailing matrix -= panel panel^T   (tiles on/below the diagonal)
-//   3. L^{-1} by block rows: X[i, 0:i] = -inv(L_ii) (L[i, 0:i] X[0:i, 0:i])
-//   4. U = J L^{-1} J, written as float with an explicit zero lower triangle.
+//   2. right-looking blocked Cholesky, 64-column panels, two launches per panel:
+//        k_chol_panel  every CTA factors the 64 x 64 diagonal block (one thread
+//                      per row, the row in registers, left-looking) and then
+//                      solves its 128 rows of the panel against it
+//        GEMM          trailing matrix -= panel panel^T  (tiles on/below the diagonal)
+//   3. inverses of the 64 x 64 diagonal blocks, all at once (k_inv_diag64)
+//   4. L^{-1} by recursive doubling: for block size s = 64, 128, ... every pair of
+//      neighbouring inverted blocks A, B with coupling C = L[B rows, A cols] gets
+//      its off-diagonal block -B^{-1} C A^{-1} from two batched GEMMs
+//   5. U = J L^{-1} J, written as float with an explicit zero lower triangle.
 #include "tb_common.cuh"
 #include "tb_gemm.cuh"
 
@@ -23,99 +28,128 @@ namespace tb {
 
 enum { FNB = 64 };
 
-__global__ void k_reverse_in(const float* __restrict__ H, double* __restrict__ A, int d) {
-  const long long n = (long long)d * d;
-  const float* Hb = H + (long long)blockIdx.y * n;
+// A (dp x dp) <- J H J in the leading d x d block, identity elsewhere
+__global__ void k_reverse_in(const float* __restrict__ H, double* __restrict__ A, int d, int dp) {
+  const long long n = (long long)dp * dp;
+  const float* Hb = H + (long long)blockIdx.y * d * d;
   double* Ab = A + (long long)blockIdx.y * n;
   for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < n;
        idx += (long long)gridDim.x * blockDim.x) {
-    const int i = (int)(idx / d), j = (int)(idx % d);
-    Ab[idx] = (double)Hb[(long long)(d - 1 - i) * d + (d - 1 - j)];
+    const int i = (int)(idx / dp), j = (int)(idx % dp);
+    double v = (i == j) ? 1.0 : 0.0;
+    if (i < d && j < d) v = (double)Hb[(long long)(d - 1 - i) * d + (d - 1 - j)];
+    Ab[idx] = v;
   }
 }
 
-__global__ void k_reverse_out(const double* __restrict__ Li, float* __restrict__ U, int d) {
+__global__ void k_reverse_out(const double* __restrict__ Li, float* __restrict__ U, int d, int dp) {
   const long long n = (long long)d * d;
-  const double* Lb = Li + (long long)blockIdx.y * n;
+  const double* Lb = Li + (long long)blockIdx.y * dp * dp;
   float* Ub = U + (long long)blockIdx.y * n;
   for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < n;
        idx += (long long)gridDim.x * blockDim.x) {
     const int i = (int)(idx / d), j = (int)(idx % d);
-    Ub[idx] = (j >= i) ? (float)Lb[(long long)(d - 1 - i) * d + (d - 1 - j)] : 0.0f;
+    Ub[idx] = (j >= i) ? (float)Lb[(long long)(d - 1 - i) * dp + (d - 1 - j)] : 0.0f;
   }
 }
 
-// Factor the diagonal block [k0, k0 + nb) of A in place (lower Cholesky) and
-// write its inverse to Dinv (64 x 64, zero above the diagonal) and to the
-// diagonal block of Li.  A non-positive pivot is recorded in info (first one
-// wins) and replaced by 1 so that no NaN or Inf is produced by this kernel.
-__global__ void __launch_bounds__(256) k_potrf64(double* __restrict__ A, double* __restrict__ Li,
-                                                 double* __restrict__ Dinv, int* __restrict__ info,
-                                                 int d, int k0, int nb, int n_blk) {
+// One panel step of the Cholesky factorisation, columns k0 .. k0+63 of the dp x dp matrix.
+// Every CTA factors the diagonal block itself (same arithmetic everywhere, so the same
+// result); CTA x then solves rows k0+64+128x .. +127 of the panel, X L_kk^T = A_panel.
+// A non-positive pivot is recorded in info (first one wins) and replaced by 1.
+__global__ void __launch_bounds__(128) k_chol_panel(double* __restrict__ A, int* __restrict__ info,
+                                                    int dp, int k0) {
+  __shared__ double sL[FNB][FNB + 1];
+  __shared__ double rdiag[FNB];
+  const int tid = threadIdx.x, b = blockIdx.y;
+  double* Ab = A + (long long)b * dp * dp;
+  if (tid < FNB) {
+    // left-looking factorisation, thread r owns row r of the block
+    const int r = tid;
+    double a[FNB];
+    const double* src = Ab + (long long)(k0 + r) * dp + k0;
+#pragma unroll
+    for (int c = 0; c < FNB; ++c) a[c] = src[c];
+#pragma unroll
+    for (int j = 0; j < FNB; ++j) {
+      // t = a[r][j] - sum_{k<j} L[r][k] L[j][k]
+      double t0 = a[j], t1 = 0.0;
+#pragma unroll
+      for (int k = 0; k + 1 < j; k += 2) {
+        t0 = fma(-a[k], sL[j][k], t0);
+        t1 = fma(-a[k + 1], sL[j][k + 1], t1);
+      }
+      if (j & 1) t0 = fma(-a[j - 1], sL[j][j - 1], t0);
+      const double t = t0 + t1;
+      if (r == j) {
+        const bool bad = !(t > 0.0);
+        if (bad && blockIdx.x == 0) atomicCAS(&info[b], 0, k0 + j + 1);
+        const double dj = bad ? 1.0 : sqrt(t);
+        sL[j][j] = dj;
+        rdiag[j] = 1.0 / dj;
+        a[j] = dj;
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");  // all 128 threads (the other 64 pass the same barriers below)
+      if (r > j) {
+        a[j] = t * rdiag[j];
+        sL[r][j] = a[j];
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+    }
+    if (blockIdx.x == 0) {
+      double* dst = Ab + (long long)(k0 + r) * dp + k0;
+#pragma unroll
+      for (int c = 0; c < FNB; ++c)
+        if (c <= r) dst[c] = a[c];
+    }
+  } else {
+#pragma unroll 1
+    for (int j = 0; j < 2 * FNB; ++j) asm volatile("bar.sync 1, 128;" ::: "memory");
+  }
+  // rows of the panel below the block
+  const long long row = (long long)k0 + FNB + (long long)blockIdx.x * 128 + tid;
+  if (row < dp) {
+    double x[FNB];
+    double* src = Ab + row * dp + k0;
+#pragma unroll
+    for (int c = 0; c < FNB; ++c) x[c] = src[c];
+#pragma unroll
+    for (int j = 0; j < FNB; ++j) {
+      double t0 = x[j], t1 = 0.0;
+#pragma unroll
+      for (int k = 0; k + 1 < j; k += 2) {
+        t0 = fma(-x[k], sL[j][k], t0);
+        t1 = fma(-x[k + 1], sL[j][k + 1], t1);
+      }
+      if (j & 1) t0 = fma(-x[j - 1], sL[j][j - 1], t0);
+      x[j] = (t0 + t1) * rdiag[j];
+    }
+#pragma unroll
+    for (int c = 0; c < FNB; ++c) src[c] = x[c];
+  }
+}
+
+// Inverse of every 64 x 64 diagonal block of L into the same block of Li (lower triangular):
+// forward substitution, one thread per column, the column in registers.
+__global__ void __launch_bounds__(64) k_inv_diag64(const double* __restrict__ A, double* __restrict__ Li, int dp) {
   __shared__ double Ls[FNB][FNB + 1];
   __shared__ double rdiag[FNB];
-  const int b = blockIdx.x, tid = threadIdx.x;
-  double* Ab = A + (long long)b * d * d;
-  for (int idx = tid; idx < FNB * FNB; idx += 256) {
-    const int r = idx / FNB, c = idx % FNB;
-    double v = (r == c) ? 1.0 : 0.0;
-    if (r < nb && c < nb) v = Ab[(long long)(k0 + r) * d + k0 + c];
-    Ls[r][c] = v;
-  }
+  const int blk = blockIdx.x, b = blockIdx.y, c = threadIdx.x;
+  const long long off = (long long)b * dp * dp + (long long)blk * FNB * (dp + 1);
+  for (int r = 0; r < FNB; ++r) Ls[r][c] = A[off + (long long)r * dp + c];
   __syncthreads();
-  for (int j = 0; j < FNB; ++j) {
-    const double pv = Ls[j][j];
-    const bool bad = !(pv > 0.0);
-    const double dj = bad ? 1.0 : sqrt(pv);
-    if (bad && tid == 0 && j < nb) atomicCAS(&info[b], 0, k0 + j + 1);
-    __syncthreads();
-    if (tid == 0) Ls[j][j] = dj;
-    if (tid > j && tid < FNB) Ls[tid][j] = Ls[tid][j] / dj;
-    __syncthreads();
-    for (int idx = tid; idx < FNB * FNB; idx += 256) {
-      const int r = idx / FNB, c = idx % FNB;
-      if (c > j && c <= r) Ls[r][c] = fma(-Ls[r][j], Ls[c][j], Ls[r][c]);
-    }
-    __syncthreads();
-  }
-  for (int idx = tid; idx < FNB * FNB; idx += 256) {
-    const int r = idx / FNB, c = idx % FNB;
-    if (r < nb && c < nb && c <= r) Ab[(long long)(k0 + r) * d + k0 + c] = Ls[r][c];
-  }
-  if (tid < FNB) rdiag[tid] = 1.0 / Ls[tid][tid];
+  rdiag[c] = 1.0 / Ls[c][c];
   __syncthreads();
-  if (tid < FNB) {
-    // column `tid` of inv(L): L x = e_tid by forward substitution, x in registers
-    const int c = tid;
-    double x[FNB];
+  double x[FNB];
 #pragma unroll
-    for (int r = 0; r < FNB; ++r) {
-      double s = (r == c) ? 1.0 : 0.0;
+  for (int r = 0; r < FNB; ++r) {
+    double s0 = (r == c) ? 1.0 : 0.0;
 #pragma unroll
-      for (int k = 0; k < r; ++k) s = fma(-Ls[r][k], x[k], s);
-      x[r] = (r < c) ? 0.0 : s * rdiag[r];
-    }
-    double* Db = Dinv + ((long long)b * n_blk + k0 / FNB) * FNB * FNB;
-    double* Lb = Li + (long long)b * d * d;
-#pragma unroll
-    for (int r = 0; r < FNB; ++r) {
-      Db[r * FNB + c] = x[r];
-      if (r < nb && c < nb) Lb[(long long)(k0 + r) * d + k0 + c] = x[r];
-    }
+    for (int k = 0; k < r; ++k) s0 = fma(-Ls[r][k], x[k], s0);
+    x[r] = (r < c) ? 0.0 : s0 * rdiag[r];
   }
-}
-
-__global__ void k_copy_panel(const double* __restrict__ A, double* __restrict__ Pn, int d, int r0,
-                             int k0, int nb) {
-  const long long rows = d - r0;
-  const double* Ab = A + (long long)blockIdx.y * d * d;
-  double* Pb = Pn + (long long)blockIdx.y * d * FNB;
-  for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < rows * nb;
-       idx += (long long)gridDim.x * blockDim.x) {
-    const long long r = idx / nb;
-    const int c = (int)(idx % nb);
-    Pb[r * FNB + c] = Ab[(r0 + r) * d + k0 + c];
-  }
+#pragma unroll
+  for (int r = 0; r < FNB; ++r) Li[off + (long long)r * dp + c] = x[r];
 }
 
 // strictly-upper mask of a square matrix (Algorithm 2 line 2: (R U^T) .* M_U)
@@ -129,20 +163,25 @@ __global__ void k_mask_strict_upper(const double* __restrict__ src, double* __re
 }
 
 struct FactorWs {
-  double *A, *Li, *Dinv, *Pn, *tmp;
-  int n_blk;
+  double *A, *Li, *tmp;
+  int dp;
   size_t total;
 };
+
+static int padded_dim(int d) {
+  int dp = FNB;
+  while (dp < d) dp <<= 1;
+  return dp;
+}
 
 static FactorWs factor_ws(int n_batch, int d, void* ws) {
   FactorWs f;
   Bump b(ws);
-  f.n_blk = (d + FNB - 1) / FNB;
-  f.A = b.take<double>((size_t)n_batch * d * d);
-  f.Li = b.take<double>((size_t)n_batch * d * d);
-  f.Dinv = b.take<double>((size_t)n_batch * f.n_blk * FNB * FNB);
-  f.Pn = b.take<double>((size_t)n_batch * d * FNB);
-  f.tmp = b.take<double>((size_t)n_batch * FNB * d);
+  f.dp = padded_dim(d);
+  const size_t n = (size_t)f.dp * f.dp;
+  f.A = b.take<double>((size_t)n_batch * n);
+  f.Li = b.take<double>((size_t)n_batch * n);
+  f.tmp = b.take<double>((size_t)n_batch * n / 4 + 64);
   f.total = b.total();
   return f;
 }
@@ -162,54 +201,38 @@ extern "C" tb_status tb_factor(const float* H, int n_batch, int d, float* U, flo
   if (!ws || !aligned(ws, 256) || ws_bytes < tb_factor_workspace(n_batch, d)) return TB_ERR_WORKSPACE;
   cudaStream_t st = as_stream(stream);
   FactorWs f = factor_ws(n_batch, d, ws);
-  const long long dd = (long long)d * d;
+  const int dp = f.dp;
+  const long long pp = (long long)dp * dp;
   TB_CUDA_CHECK(cudaMemsetAsync(info, 0, sizeof(int) * (size_t)n_batch, st));
-  TB_CUDA_CHECK(cudaMemsetAsync(f.Li, 0, sizeof(double) * (size_t)n_batch * dd, st));
-  int eb = (int)((dd + 255) / 256);
+  TB_CUDA_CHECK(cudaMemsetAsync(f.Li, 0, sizeof(double) * (size_t)n_batch * pp, st));
+  int eb = (int)((pp + 255) / 256);
   if (eb > 148 * 8) eb = 148 * 8;
-  k_reverse_in<<<dim3(eb, n_batch), 256, 0, st>>>(H, f.A, d);
+  k_reverse_in<<<dim3(eb, n_batch), 256, 0, st>>>(H, f.A, d, dp);
   TB_LAUNCH_CHECK();
 
-  for (int k0 = 0; k0 < d; k0 += FNB) {
-    const int nb = (d - k0 < FNB) ? (d - k0) : FNB;
-    k_potrf64<<<n_batch, 256, 0, st>>>(f.A, f.Li, f.Dinv, info, d, k0, nb, f.n_blk);
+  // the padding is an identity block decoupled from the rest: factor the leading part only
+  const int d_fact = ((d + FNB - 1) / FNB) * FNB;
+  for (int k0 = 0; k0 < d_fact; k0 += FNB) {
+    const int r0 = k0 + FNB, m = d_fact - r0;
+    const int xt = (m > 0) ? (m + 127) / 128 : 1;
+    k_chol_panel<<<dim3(xt, n_batch), 128, 0, st>>>(f.A, info, dp, k0);
     TB_LAUNCH_CHECK();
-    const int r0 = k0 + nb, m = d - r0;
     if (m <= 0) break;
-    k_copy_panel<<<dim3(64, n_batch), 256, 0, st>>>(f.A, f.Pn, d, r0, k0, nb);
-    TB_LAUNCH_CHECK();
-    GemmP g = gemm_params();  // panel <- panel inv(L_kk)^T
-    g.A = f.Pn;
-    g.a_m = FNB;
-    g.a_k = 1;
-    g.a_batch = (long long)d * FNB;
-    g.B = f.Dinv + (long long)(k0 / FNB) * FNB * FNB;  // B(k, n) = Dinv[n][k]
-    g.b_k = 1;
-    g.b_n = FNB;
-    g.b_batch = (long long)f.n_blk * FNB * FNB;
-    g.C = f.A + (long long)r0 * d + k0;
-    g.ldc = d;
-    g.c_batch = dd;
-    g.M = m;
-    g.N = nb;
-    g.K = nb;
-    g.n_batch = n_batch;
-    TB_TRY((gemm_launch<double, double, double, double, false, false>(g, st)));
     GemmP s = gemm_params();  // trailing -= panel panel^T, tiles on or below the diagonal
-    s.A = f.A + (long long)r0 * d + k0;
-    s.a_m = d;
+    s.A = f.A + (long long)r0 * dp + k0;
+    s.a_m = dp;
     s.a_k = 1;
-    s.a_batch = dd;
-    s.B = f.A + (long long)r0 * d + k0;  // B(k, n) = panel[n][k]
+    s.a_batch = pp;
+    s.B = f.A + (long long)r0 * dp + k0;  // B(k, n) = panel[n][k]
     s.b_k = 1;
-    s.b_n = d;
-    s.b_batch = dd;
-    s.C = f.A + (long long)r0 * d + r0;
-    s.ldc = d;
-    s.c_batch = dd;
+    s.b_n = dp;
+    s.b_batch = pp;
+    s.C = f.A + (long long)r0 * dp + r0;
+    s.ldc = dp;
+    s.c_batch = pp;
     s.M = m;
     s.N = m;
-    s.K = nb;
+    s.K = FNB;
     s.n_batch = n_batch;
     s.alpha = -1.0;
     s.beta = 1.0;
@@ -217,65 +240,78 @@ extern "C" tb_status tb_factor(const float* H, int n_batch, int d, float* U, flo
     TB_TRY((gemm_launch<double, double, double, double, false, false>(s, st)));
   }
 
-  // L^{-1}, block row by block row (diagonal blocks are already in place)
-  for (int r0 = FNB; r0 < d; r0 += FNB) {
-    const int nb = (d - r0 < FNB) ? (d - r0) : FNB;
-    GemmP g = gemm_params();  // tmp = L[r0:r0+nb, 0:r0] * Li[0:r0, 0:r0]
-    g.A = f.A + (long long)r0 * d;
-    g.a_m = d;
-    g.a_k = 1;
-    g.a_batch = dd;
-    g.B = f.Li;
-    g.b_k = d;
-    g.b_n = 1;
-    g.b_batch = dd;
-    g.C = f.tmp;
-    g.ldc = d;
-    g.c_batch = (long long)FNB * d;
-    g.M = nb;
-    g.N = r0;
-    g.K = r0;
-    g.n_batch = n_batch;
-    g.btrim = 2;  // Li is lower triangular: Li(k, n) = 0 for k < n
-    g.boff = 0;
-    TB_TRY((gemm_launch<double, double, double, double, false, true>(g, st)));
-    GemmP h = gemm_params();  // Li[r0:r0+nb, 0:r0] = -inv(L_ii) tmp
-    h.A = f.Dinv + (long long)(r0 / FNB) * FNB * FNB;
-    h.a_m = FNB;
-    h.a_k = 1;
-    h.a_batch = (long long)f.n_blk * FNB * FNB;
-    h.B = f.tmp;
-    h.b_k = d;
-    h.b_n = 1;
-    h.b_batch = (long long)FNB * d;
-    h.C = f.Li + (long long)r0 * d;
-    h.ldc = d;
-    h.c_batch = dd;
-    h.M = nb;
-    h.N = r0;
-    h.K = nb;
-    h.n_batch = n_batch;
-    h.alpha = -1.0;
-    TB_TRY((gemm_launch<double, double, double, double, false, true>(h, st)));
+  // L^{-1}: diagonal blocks, then recursive doubling
+  k_inv_diag64<<<dim3(dp / FNB, n_batch), 64, 0, st>>>(f.A, f.Li, dp);
+  TB_LAUNCH_CHECK();
+  for (int sblk = FNB; sblk < dp; sblk <<= 1) {
+    const int pairs = dp / (2 * sblk);
+    // one batched launch covers all pairs of one matrix, or (a single pair per matrix) all matrices
+    const int outer = (pairs == 1) ? 1 : n_batch;
+    for (int mb = 0; mb < outer; ++mb) {
+      const long long moff = (long long)mb * pp;
+      const long long pair_stride = (pairs == 1) ? pp : (long long)2 * sblk * (dp + 1);
+      const int batch = (pairs == 1) ? n_batch : pairs;
+      double* tmp = f.tmp + (long long)mb * (pp / 4);
+      const long long tmp_stride = (pairs == 1) ? (pp / 4) : (long long)sblk * sblk;
+      GemmP g = gemm_params();  // T = C A^{-1}: C = L[s:2s, 0:s], A^{-1} = Li[0:s, 0:s] (lower triangular)
+      g.A = f.A + moff + (long long)sblk * dp;
+      g.a_m = dp;
+      g.a_k = 1;
+      g.a_batch = pair_stride;
+      g.B = f.Li + moff;
+      g.b_k = dp;
+      g.b_n = 1;
+      g.b_batch = pair_stride;
+      g.C = tmp;
+      g.ldc = sblk;
+      g.c_batch = tmp_stride;
+      g.M = sblk;
+      g.N = sblk;
+      g.K = sblk;
+      g.n_batch = batch;
+      g.btrim = 2;
+      TB_TRY((gemm_launch<double, double, double, double, false, true>(g, st)));
+      GemmP h = gemm_params();  // Li[s:2s, 0:s] = -B^{-1} T, B^{-1} = Li[s:2s, s:2s] (lower triangular)
+      h.A = f.Li + moff + (long long)sblk * (dp + 1);
+      h.a_m = dp;
+      h.a_k = 1;
+      h.a_batch = pair_stride;
+      h.B = tmp;
+      h.b_k = sblk;
+      h.b_n = 1;
+      h.b_batch = tmp_stride;
+      h.C = f.Li + moff + (long long)sblk * dp;
+      h.ldc = dp;
+      h.c_batch = pair_stride;
+      h.M = sblk;
+      h.N = sblk;
+      h.K = sblk;
+      h.n_batch = batch;
+      h.alpha = -1.0;
+      h.atrim = 1;
+      TB_TRY((gemm_launch<double, double, double, double, false, true>(h, st)));
+    }
   }
-  k_reverse_out<<<dim3(eb, n_batch), 256, 0, st>>>(f.Li, U, d);
+  int eo = (int)(((long long)d * d + 255) / 256);
+  if (eo > 148 * 8) eo = 148 * 8;
+  k_reverse_out<<<dim3(eo, n_batch), 256, 0, st>>>(f.Li, U, d, dp);
   TB_LAUNCH_CHECK();
 
   if (Hinv) {
-    // Hinv = U^T U with U(k, m) = Li[d-1-k][d-1-m]: negative strides from the last element
+    // Hinv = U^T U with U(k, m) = Li[d-1-k][d-1-m]: negative strides from element (d-1, d-1)
     GemmP g = gemm_params();
-    const double* last = f.Li + dd - 1;
+    const double* last = f.Li + (long long)(d - 1) * dp + (d - 1);
     g.A = last;  // A(m, k) = U[k][m]
     g.a_m = -1;
-    g.a_k = -(long long)d;
-    g.a_batch = dd;
+    g.a_k = -(long long)dp;
+    g.a_batch = pp;
     g.B = last;  // B(k, n) = U[k][n]
-    g.b_k = -(long long)d;
+    g.b_k = -(long long)dp;
     g.b_n = -1;
-    g.b_batch = dd;
+    g.b_batch = pp;
     g.C = Hinv;
     g.ldc = d;
-    g.c_batch = dd;
+    g.c_batch = (long long)d * d;
     g.M = d;
     g.N = d;
     g.K = d;
