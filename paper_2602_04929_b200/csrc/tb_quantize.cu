@@ -904,6 +904,124 @@ __global__ void __launch_bounds__(256) k_cd_row_update(CdP p) {
     for (int g = tid; g < ng; g += blockDim.x) p.sD[row * ng + g] += delta[g];
 }
 
+// ---------------------------------------------------------------------------
+// One Gauss-Seidel pass of Algorithm 3 over ALL rows of one head in a single
+// launch: one CTA per head walks the head's rows in order.  It works on
+//   G = H_out Dm    (rows of the head, formed once by a batched GEMM),
+// whose row j is what the numerator of Proposition 3.3 needs.  A step on the
+// scales of row i adds u_i = sum_g2 delta_g2 Yw[i][g2][:] to row i of Dm, hence
+// H_out[j][i] u_i to every row j of G.  Those rank-1 terms are applied lazily:
+// rows of the current block of 16 read the u_i of their block on the fly, and
+// when a block is finished its 16 vectors are folded into the rows of G that
+// are still to come.  The u_i are kept (Uacc) so that Dm can be refreshed
+// after the pass.  All sums have a fixed order.
+// ---------------------------------------------------------------------------
+enum { CDH_THREADS = 512, CDH_BLOCK = 16 };
+struct CdHeadP {
+  double* G;           // [heads*dh][d]   H_out Dm, updated in place
+  double* Uacc;        // [heads*dh][d]   out: the rank-1 vectors u_i
+  const double* Yw;    // [heads*dh][ng][d]
+  const float* Wb;     // [heads*dh][d]
+  const float* Hout;   // [heads][dh][dh]
+  double* sD;          // [heads*dh][ng]
+  int d, seg, ng, dh;
+};
+
+__global__ void __launch_bounds__(CDH_THREADS, 1) k_cd_head(CdHeadP p) {
+  extern __shared__ double cdh_sm[];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int head = blockIdx.x;
+  const int d = p.d, seg = p.seg, ng = p.ng, dh = p.dh;
+  const int n_chunks = d / 32;                 // 32-column chunks of a row
+  const int chunks_per_group = seg / 32;
+  double* part = cdh_sm;                        // [n_chunks][ng + 1]
+  double* Am = part + (size_t)n_chunks * (ng + 1);  // [ng][ng]  (entries g2 <= g)
+  double* num = Am + (size_t)ng * ng;           // [ng]
+  double* delta = num + ng;                     // [ng]
+  const long long row0 = (long long)head * dh;
+  const float* Ho = p.Hout + (long long)head * dh * dh;
+
+  for (int j = 0; j < dh; ++j) {
+    const long long row = row0 + j;
+    const int blk0 = (j / CDH_BLOCK) * CDH_BLOCK;
+    const double hjj = (double)Ho[(long long)j * dh + j];
+    const double* Yr = p.Yw + row * ng * d;
+    const float* wbr = p.Wb + row * d;
+    double* Gr = p.G + row * d;
+    // ---- statistics of the row: n0[g] and A[g2][g] for g2 <= g ----
+    for (int q = warp; q < n_chunks; q += CDH_THREADS / 32) {
+      const int col = q * 32 + lane;
+      const int g = q / chunks_per_group;
+      double gv = Gr[col];
+      for (int i = blk0; i < j; ++i) gv = fma((double)Ho[(long long)j * dh + i], p.Uacc[(row0 + i) * d + col], gv);
+      const double wb = (double)wbr[col];
+      const double v = warp_sum(wb * gv);
+      if (lane == 0) part[(size_t)q * (ng + 1) + ng] = v;
+      for (int g2 = 0; g2 <= g; ++g2) {
+        const double a = warp_sum(Yr[(long long)g2 * d + col] * wb);
+        if (lane == 0) part[(size_t)q * (ng + 1) + g2] = a;
+      }
+    }
+    __syncthreads();
+    for (int idx = tid; idx < ng * (ng + 1); idx += CDH_THREADS) {
+      const int g = idx / (ng + 1), g2 = idx % (ng + 1);
+      if (g2 != ng && g2 > g) continue;
+      double t = 0.0;
+      for (int c = 0; c < chunks_per_group; ++c) t += part[(size_t)(g * chunks_per_group + c) * (ng + 1) + g2];
+      if (g2 == ng)
+        num[g] = t;
+      else
+        Am[(size_t)g2 * ng + g] = t;
+    }
+    __syncthreads();
+    // ---- the scalar chain over the row's groups ----
+    if (warp == 0) {
+      for (int g2 = 0; g2 < ng; ++g2) {
+        const double den = Am[(size_t)g2 * ng + g2] * hjj;
+        const double dl = (den == 0.0) ? 0.0 : -num[g2] / den;
+        if (lane == 0) delta[g2] = dl;
+        for (int g = g2 + 1 + lane; g < ng; g += 32) num[g] = fma(hjj * dl, Am[(size_t)g2 * ng + g], num[g]);
+        __syncwarp();
+      }
+    }
+    __syncthreads();
+    // ---- u_j and the scales ----
+    double* ur = p.Uacc + row * d;
+    for (int col = tid; col < d; col += CDH_THREADS) {
+      double acc = 0.0;
+      for (int g2 = 0; g2 < ng; ++g2) acc = fma(delta[g2], Yr[(long long)g2 * d + col], acc);
+      ur[col] = acc;
+    }
+    for (int g = tid; g < ng; g += CDH_THREADS) p.sD[row * ng + g] += delta[g];
+    __syncthreads();
+    // ---- end of a block: fold its vectors into the rows of G still to come ----
+    if (((j + 1) % CDH_BLOCK == 0 || j + 1 == dh) && j + 1 < dh) {
+      const int nb = j + 1 - blk0;
+      for (int col = tid; col < d; col += CDH_THREADS) {
+        double u[CDH_BLOCK];
+#pragma unroll
+        for (int i = 0; i < CDH_BLOCK; ++i) u[i] = (i < nb) ? p.Uacc[(row0 + blk0 + i) * d + col] : 0.0;
+        for (int jj = j + 1; jj < dh; ++jj) {
+          const float* hr = Ho + (long long)jj * dh + blk0;
+          double gv = p.G[(row0 + jj) * d + col];
+#pragma unroll
+          for (int i = 0; i < CDH_BLOCK; ++i)
+            if (i < nb) gv = fma((double)hr[i], u[i], gv);
+          p.G[(row0 + jj) * d + col] = gv;
+        }
+      }
+      __syncthreads();
+    }
+  }
+}
+
+// Dm += Uacc (the effect of one pass on (Q - W) H_in + W R)
+__global__ void k_axpy(double* __restrict__ y, const double* __restrict__ x, long long n) {
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n;
+       i += (long long)gridDim.x * blockDim.x)
+    y[i] += x[i];
+}
+
 // Q = s (W_int - z) in float, and the scales in float (Algorithm 1, line 13).
 __global__ void k_dequant(const unsigned char* __restrict__ codes, const double* __restrict__ sD,
                           const int* __restrict__ z, float* __restrict__ What,
@@ -1400,6 +1518,51 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
         y.n_batch = p.ng;
         TB_TRY((gemm_launch<float, float, double, double, false, true>(y, st)));
       }
+      if (p.has_hout) {
+        // rows of a head are coupled through H_out: one CTA per head walks them in order
+        const int heads_b = (int)(rows / p.dh);
+        const long long nb_el = rows * d;
+        CdHeadP hp;
+        hp.G = p.Wt + r0 * d;      // W~ is no longer needed: its buffer holds G = H_out Dm
+        hp.Uacc = p.Dq + r0 * d;   // (Q - W) has been consumed by the product above
+        hp.Yw = p.Yw;
+        hp.Wb = p.Wb + r0 * d;
+        hp.Hout = H_out + (r0 / p.dh) * (long long)p.dh * p.dh;
+        hp.sD = p.sD + r0 * p.ng;
+        hp.d = d;
+        hp.seg = p.seg;
+        hp.ng = p.ng;
+        hp.dh = p.dh;
+        const size_t sm_head = ((size_t)(d / 32) * (p.ng + 1) + (size_t)p.ng * p.ng + 2 * (size_t)p.ng) * sizeof(double);
+        if (sm_head > 200 * 1024) return TB_ERR_UNSUPPORTED;
+        static bool conf_head[64] = {false};
+        TB_TRY(allow_smem(k_cd_head, 200 * 1024, conf_head));
+        for (int it = 0; it < p.cd_iters; ++it) {
+          GemmP g = gemm_params();  // G = H_out Dm, head by head
+          g.A = hp.Hout;
+          g.a_m = p.dh;
+          g.a_k = 1;
+          g.a_batch = (long long)p.dh * p.dh;
+          g.B = p.Dm + r0 * d;
+          g.b_k = d;
+          g.b_n = 1;
+          g.b_batch = (long long)p.dh * d;
+          g.C = hp.G;
+          g.ldc = d;
+          g.c_batch = (long long)p.dh * d;
+          g.M = p.dh;
+          g.N = d;
+          g.K = p.dh;
+          g.n_batch = heads_b;
+          TB_TRY((gemm_launch<float, double, double, double, false, true>(g, st)));
+          k_cd_head<<<heads_b, CDH_THREADS, sm_head, st>>>(hp);
+          TB_LAUNCH_CHECK();
+          k_axpy<<<ew_blocks(nb_el), 256, 0, st>>>(p.Dm + r0 * d, hp.Uacc, nb_el);
+          TB_LAUNCH_CHECK();
+        }
+        continue;
+      }
+      // H_out = I: rows are independent, every row is its own line of one row
       CdP cp;
       cp.Dm = p.Dm + r0 * d;
       cp.Yw = p.Yw;
@@ -1410,29 +1573,18 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
       cp.d = d;
       cp.seg = p.seg;
       cp.ng = p.ng;
-      int lines, n_j;
-      if (p.has_hout) {
-        cp.Hout = H_out + (r0 / p.dh) * (long long)p.dh * p.dh;
-        cp.dh = p.dh;
-        cp.lines_per_head = 1;
-        lines = (int)(rows / p.dh);
-        n_j = p.dh;
-      } else {
-        // rows are independent: every row is its own "head" of one row
-        cp.Hout = nullptr;
-        cp.dh = 1;
-        cp.lines_per_head = 1;
-        lines = (int)rows;
-        n_j = 1;
-      }
+      cp.Hout = nullptr;
+      cp.dh = 1;
+      cp.lines_per_head = 1;
+      cp.j0 = 0;
+      const int lines = (int)rows;
       // columns per CTA: whole groups, about 512 columns
       int gpc = 512 / p.seg;
       if (gpc < 1) gpc = 1;
       if (gpc > p.ng) gpc = p.ng;
       cp.groups_per_cta = gpc;
       const int xctas = (p.ng + gpc - 1) / gpc;
-      const size_t sm_stats =
-          ((size_t)gpc * (p.seg / 32) * (p.ng + 1) + cp.dh) * sizeof(double);
+      const size_t sm_stats = ((size_t)gpc * (p.seg / 32) * (p.ng + 1) + cp.dh) * sizeof(double);
       size_t sm_upd = ((size_t)2 * p.ng + (size_t)p.ng * p.ng) * sizeof(double);
       cp.a_in_smem = 1;
       if (sm_upd > 200 * 1024) {
@@ -1444,25 +1596,19 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
       TB_TRY(allow_smem(k_cd_row_update, 200 * 1024, conf_upd));
       if (sm_stats > 200 * 1024) return TB_ERR_UNSUPPORTED;
       for (int it = 0; it < p.cd_iters; ++it) {
-        for (int j = 0; j < n_j; ++j) {
-          cp.j0 = j;
-          for (int l0 = 0; l0 < lines; l0 += 65535) {
-            const int nl = (lines - l0 < 65535) ? (lines - l0) : 65535;
-            CdP cq = cp;
-            // advance every per-line pointer by l0 lines (a line is one head, or one row)
-            const long long rows_per_line = cp.dh;
-            cq.Dm = cp.Dm + (long long)l0 * rows_per_line * d;
-            cq.Yw = cp.Yw + (long long)l0 * rows_per_line * p.ng * d;
-            cq.Wb = cp.Wb + (long long)l0 * rows_per_line * d;
-            cq.sD = cp.sD + (long long)l0 * rows_per_line * p.ng;
-            cq.n0 = cp.n0 + (long long)l0 * p.ng;
-            cq.Amat = cp.Amat + (long long)l0 * p.ng * p.ng;
-            if (cp.Hout) cq.Hout = cp.Hout + (long long)l0 * p.dh * p.dh;
-            k_cd_row_stats<<<dim3(xctas, nl), 256, sm_stats, st>>>(cq);
-            TB_LAUNCH_CHECK();
-            k_cd_row_update<<<dim3(xctas, nl), 256, sm_upd, st>>>(cq);
-            TB_LAUNCH_CHECK();
-          }
+        for (int l0 = 0; l0 < lines; l0 += 65535) {
+          const int nl = (lines - l0 < 65535) ? (lines - l0) : 65535;
+          CdP cq = cp;  // advance every per-line pointer by l0 rows
+          cq.Dm = cp.Dm + (long long)l0 * d;
+          cq.Yw = cp.Yw + (long long)l0 * p.ng * d;
+          cq.Wb = cp.Wb + (long long)l0 * d;
+          cq.sD = cp.sD + (long long)l0 * p.ng;
+          cq.n0 = cp.n0 + (long long)l0 * p.ng;
+          cq.Amat = cp.Amat + (long long)l0 * p.ng * p.ng;
+          k_cd_row_stats<<<dim3(xctas, nl), 256, sm_stats, st>>>(cq);
+          TB_LAUNCH_CHECK();
+          k_cd_row_update<<<dim3(xctas, nl), 256, sm_upd, st>>>(cq);
+          TB_LAUNCH_CHECK();
         }
       }
     }
