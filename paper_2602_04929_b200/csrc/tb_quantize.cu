@@ -15,9 +15,13 @@
 // accumulated rounding error of the chain (a few 1e-6 code units) exceeds the
 // 1e-6 band inside which a rounding decision may legitimately differ, and one
 // different decision changes every later code of its row.
+#include <cooperative_groups.h>
+
 #include "tb_common.cuh"
 #include "tb_gemm.cuh"
 #include "tb_tma.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace tb {
 
@@ -906,15 +910,20 @@ __global__ void __launch_bounds__(256) k_cd_row_update(CdP p) {
 
 // ---------------------------------------------------------------------------
 // One Gauss-Seidel pass of Algorithm 3 over ALL rows of one head in a single
-// launch: one CTA per head walks the head's rows in order.  It works on
+// launch.  A thread-block cluster of C CTAs owns a head; CTA r owns the column
+// groups r ng/C .. (r+1) ng/C - 1 (whole groups, so every sum over a group is
+// local to one CTA).  The cluster walks the head's rows in order and works on
 //   G = H_out Dm    (rows of the head, formed once by a batched GEMM),
 // whose row j is what the numerator of Proposition 3.3 needs.  A step on the
 // scales of row i adds u_i = sum_g2 delta_g2 Yw[i][g2][:] to row i of Dm, hence
 // H_out[j][i] u_i to every row j of G.  Those rank-1 terms are applied lazily:
 // rows of the current block of 16 read the u_i of their block on the fly, and
 // when a block is finished its 16 vectors are folded into the rows of G that
-// are still to come.  The u_i are kept (Uacc) so that Dm can be refreshed
-// after the pass.  All sums have a fixed order.
+// are still to come.  Per row, each CTA forms n0[g] and A[.][g] for its groups,
+// stores them into the shared memory of every CTA of the cluster (distributed
+// shared memory, two buffers by row parity), and after one cluster barrier every
+// CTA runs the short scalar chain itself.  The u_i are kept (Uacc) so that Dm
+// can be refreshed after the pass.  All sums have a fixed order.
 // ---------------------------------------------------------------------------
 enum { CDH_THREADS = 512, CDH_BLOCK = 16 };
 struct CdHeadP {
@@ -925,94 +934,151 @@ struct CdHeadP {
   const float* Hout;   // [heads][dh][dh]
   double* sD;          // [heads*dh][ng]
   int d, seg, ng, dh;
+  int csize;           // CTAs per cluster (divides ng)
+  int uw;              // columns per work unit (a divisor of seg, multiple of 32, at most 128)
 };
 
 __global__ void __launch_bounds__(CDH_THREADS, 1) k_cd_head(CdHeadP p) {
   extern __shared__ double cdh_sm[];
+  cg::cluster_group cluster = cg::this_cluster();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int head = blockIdx.x;
-  const int d = p.d, seg = p.seg, ng = p.ng, dh = p.dh;
-  const int n_chunks = d / 32;                 // 32-column chunks of a row
-  const int chunks_per_group = seg / 32;
-  double* part = cdh_sm;                        // [n_chunks][ng + 1]
-  double* Am = part + (size_t)n_chunks * (ng + 1);  // [ng][ng]  (entries g2 <= g)
-  double* num = Am + (size_t)ng * ng;           // [ng]
-  double* delta = num + ng;                     // [ng]
+  const int rank = (int)cluster.block_rank();
+  const int head = blockIdx.x / p.csize;
+  const int d = p.d, seg = p.seg, ng = p.ng, dh = p.dh, uw = p.uw;
+  const int gpc = ng / p.csize;                 // groups of this CTA
+  const int g_lo = rank * gpc;
+  const int upg = seg / uw;                     // units per group
+  const int n_units = gpc * upg;                // units of this CTA
+  const int c_lo = g_lo * seg, c_cnt = gpc * seg;  // its columns
+  double* part = cdh_sm;                                   // [n_units][ng + 1]
+  double* Am = part + (size_t)n_units * (ng + 1);          // [2][ng][ng]  (entries g2 <= g)
+  double* num = Am + (size_t)2 * ng * ng;                  // [2][ng]
+  double* delta = num + 2 * ng;                            // [ng]
   const long long row0 = (long long)head * dh;
   const float* Ho = p.Hout + (long long)head * dh * dh;
 
   for (int j = 0; j < dh; ++j) {
     const long long row = row0 + j;
+    const int buf = j & 1;
     const int blk0 = (j / CDH_BLOCK) * CDH_BLOCK;
     const double hjj = (double)Ho[(long long)j * dh + j];
     const double* Yr = p.Yw + row * ng * d;
     const float* wbr = p.Wb + row * d;
-    double* Gr = p.G + row * d;
-    // ---- statistics of the row: n0[g] and A[g2][g] for g2 <= g ----
-    for (int q = warp; q < n_chunks; q += CDH_THREADS / 32) {
-      const int col = q * 32 + lane;
-      const int g = q / chunks_per_group;
-      double gv = Gr[col];
-      for (int i = blk0; i < j; ++i) gv = fma((double)Ho[(long long)j * dh + i], p.Uacc[(row0 + i) * d + col], gv);
-      const double wb = (double)wbr[col];
-      const double v = warp_sum(wb * gv);
-      if (lane == 0) part[(size_t)q * (ng + 1) + ng] = v;
-      for (int g2 = 0; g2 <= g; ++g2) {
-        const double a = warp_sum(Yr[(long long)g2 * d + col] * wb);
-        if (lane == 0) part[(size_t)q * (ng + 1) + g2] = a;
+    const double* Gr = p.G + row * d;
+    const float* hrow = Ho + (long long)j * dh;
+    // ---- statistics of the row for this CTA's groups: n0[g] and A[g2][g], g2 <= g ----
+    for (int u = warp; u < n_units; u += CDH_THREADS / 32) {
+      const int g = g_lo + u / upg;
+      const int cbase = g * seg + (u % upg) * uw;
+      double wb[4], gv[4];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const int col = cbase + lane + 32 * c;
+        const bool on = lane + 32 * c < uw;
+        wb[c] = on ? (double)wbr[col] : 0.0;
+        gv[c] = on ? Gr[col] : 0.0;
+      }
+      for (int i = blk0; i < j; ++i) {
+        const double h = (double)hrow[i];
+        const double* ui = p.Uacc + (row0 + i) * d + cbase + lane;
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+          if (lane + 32 * c < uw) gv[c] = fma(h, ui[32 * c], gv[c]);
+      }
+      double v = 0.0;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) v = fma(wb[c], gv[c], v);
+      v = warp_sum(v);
+      if (lane == 0) part[(size_t)u * (ng + 1) + ng] = v;
+      const double* yb = Yr + cbase + lane;
+      int g2 = 0;
+      for (; g2 + 4 <= g + 1; g2 += 4) {
+        double a4[4] = {0.0, 0.0, 0.0, 0.0};
+#pragma unroll
+        for (int t = 0; t < 4; ++t)
+#pragma unroll
+          for (int c = 0; c < 4; ++c)
+            if (lane + 32 * c < uw) a4[t] = fma(yb[(long long)(g2 + t) * d + 32 * c], wb[c], a4[t]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+          for (int t = 0; t < 4; ++t) a4[t] += __shfl_xor_sync(0xffffffffu, a4[t], o);
+        if (lane < 4) part[(size_t)u * (ng + 1) + g2 + lane] = (lane == 0) ? a4[0] : (lane == 1) ? a4[1] : (lane == 2) ? a4[2] : a4[3];
+      }
+      for (; g2 <= g; ++g2) {
+        double a = 0.0;
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+          if (lane + 32 * c < uw) a = fma(yb[(long long)g2 * d + 32 * c], wb[c], a);
+        a = warp_sum(a);
+        if (lane == 0) part[(size_t)u * (ng + 1) + g2] = a;
       }
     }
     __syncthreads();
-    for (int idx = tid; idx < ng * (ng + 1); idx += CDH_THREADS) {
-      const int g = idx / (ng + 1), g2 = idx % (ng + 1);
+    // ---- reduce the units of each group in order and publish to every CTA of the cluster ----
+    for (int idx = tid; idx < gpc * (ng + 1); idx += CDH_THREADS) {
+      const int gl = idx / (ng + 1), g2 = idx % (ng + 1), g = g_lo + gl;
       if (g2 != ng && g2 > g) continue;
       double t = 0.0;
-      for (int c = 0; c < chunks_per_group; ++c) t += part[(size_t)(g * chunks_per_group + c) * (ng + 1) + g2];
-      if (g2 == ng)
-        num[g] = t;
-      else
-        Am[(size_t)g2 * ng + g] = t;
+      for (int c = 0; c < upg; ++c) t += part[(size_t)(gl * upg + c) * (ng + 1) + g2];
+      for (int r = 0; r < p.csize; ++r) {
+        if (g2 == ng)
+          cluster.map_shared_rank(num, r)[buf * ng + g] = t;
+        else
+          cluster.map_shared_rank(Am, r)[((size_t)buf * ng + g2) * ng + g] = t;
+      }
     }
-    __syncthreads();
-    // ---- the scalar chain over the row's groups ----
+    cluster.sync();
+    // ---- the scalar chain over the row's groups (every CTA runs it) ----
     if (warp == 0) {
+      double* nm = num + buf * ng;
+      const double* A = Am + (size_t)buf * ng * ng;
       for (int g2 = 0; g2 < ng; ++g2) {
-        const double den = Am[(size_t)g2 * ng + g2] * hjj;
-        const double dl = (den == 0.0) ? 0.0 : -num[g2] / den;
+        const double den = A[(size_t)g2 * ng + g2] * hjj;
+        const double dl = (den == 0.0) ? 0.0 : -nm[g2] / den;
         if (lane == 0) delta[g2] = dl;
-        for (int g = g2 + 1 + lane; g < ng; g += 32) num[g] = fma(hjj * dl, Am[(size_t)g2 * ng + g], num[g]);
+        for (int g = g2 + 1 + lane; g < ng; g += 32) nm[g] = fma(hjj * dl, A[(size_t)g2 * ng + g], nm[g]);
         __syncwarp();
       }
     }
     __syncthreads();
-    // ---- u_j and the scales ----
+    // ---- u_j on this CTA's columns, and the scales ----
     double* ur = p.Uacc + row * d;
-    for (int col = tid; col < d; col += CDH_THREADS) {
-      double acc = 0.0;
-      for (int g2 = 0; g2 < ng; ++g2) acc = fma(delta[g2], Yr[(long long)g2 * d + col], acc);
-      ur[col] = acc;
+    for (int c0 = tid; c0 < c_cnt; c0 += 4 * CDH_THREADS) {
+      double acc[4] = {0.0, 0.0, 0.0, 0.0};
+      for (int g2 = 0; g2 < ng; ++g2) {
+        const double dl = delta[g2];
+        const double* y = Yr + (long long)g2 * d + c_lo + c0;
+#pragma unroll
+        for (int t = 0; t < 4; ++t)
+          if (c0 + t * CDH_THREADS < c_cnt) acc[t] = fma(dl, y[t * CDH_THREADS], acc[t]);
+      }
+#pragma unroll
+      for (int t = 0; t < 4; ++t)
+        if (c0 + t * CDH_THREADS < c_cnt) ur[c_lo + c0 + t * CDH_THREADS] = acc[t];
     }
-    for (int g = tid; g < ng; g += CDH_THREADS) p.sD[row * ng + g] += delta[g];
+    if (rank == 0)
+      for (int g = tid; g < ng; g += CDH_THREADS) p.sD[row * ng + g] += delta[g];
     __syncthreads();
     // ---- end of a block: fold its vectors into the rows of G still to come ----
-    if (((j + 1) % CDH_BLOCK == 0 || j + 1 == dh) && j + 1 < dh) {
-      const int nb = j + 1 - blk0;
-      for (int col = tid; col < d; col += CDH_THREADS) {
-        double u[CDH_BLOCK];
+    if ((j + 1) % CDH_BLOCK == 0 && j + 1 < dh) {
+      for (int c = tid; c < c_cnt; c += CDH_THREADS) {
+        const int col = c_lo + c;
+        double u16[CDH_BLOCK];
 #pragma unroll
-        for (int i = 0; i < CDH_BLOCK; ++i) u[i] = (i < nb) ? p.Uacc[(row0 + blk0 + i) * d + col] : 0.0;
+        for (int i = 0; i < CDH_BLOCK; ++i) u16[i] = p.Uacc[(row0 + blk0 + i) * d + col];
         for (int jj = j + 1; jj < dh; ++jj) {
           const float* hr = Ho + (long long)jj * dh + blk0;
-          double gv = p.G[(row0 + jj) * d + col];
+          double gvv = p.G[(row0 + jj) * d + col];
 #pragma unroll
-          for (int i = 0; i < CDH_BLOCK; ++i)
-            if (i < nb) gv = fma((double)hr[i], u[i], gv);
-          p.G[(row0 + jj) * d + col] = gv;
+          for (int i = 0; i < CDH_BLOCK; ++i) gvv = fma((double)hr[i], u16[i], gvv);
+          p.G[(row0 + jj) * d + col] = gvv;
         }
       }
       __syncthreads();
     }
   }
+  cluster.sync();  // no CTA may exit while another can still store into its shared memory
 }
 
 // Dm += Uacc (the effect of one pass on (Q - W) H_in + W R)
@@ -1533,7 +1599,14 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
         hp.seg = p.seg;
         hp.ng = p.ng;
         hp.dh = p.dh;
-        const size_t sm_head = ((size_t)(d / 32) * (p.ng + 1) + (size_t)p.ng * p.ng + 2 * (size_t)p.ng) * sizeof(double);
+        hp.uw = (p.seg % 128 == 0) ? 128 : (p.seg <= 128 ? p.seg : 32);
+        // CTAs per head: whole groups per CTA, and no more CTAs than the GPU holds at once
+        int csize = 8;
+        while (csize > 1 && ((p.ng % csize) || (long long)heads_b * csize > 148)) csize >>= 1;
+        hp.csize = csize;
+        const int n_units = (p.ng / csize) * (p.seg / hp.uw);
+        const size_t sm_head =
+            ((size_t)n_units * (p.ng + 1) + 2 * (size_t)p.ng * p.ng + 3 * (size_t)p.ng) * sizeof(double);
         if (sm_head > 200 * 1024) return TB_ERR_UNSUPPORTED;
         static bool conf_head[64] = {false};
         TB_TRY(allow_smem(k_cd_head, 200 * 1024, conf_head));
@@ -1555,7 +1628,19 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
           g.K = p.dh;
           g.n_batch = heads_b;
           TB_TRY((gemm_launch<float, double, double, double, false, true>(g, st)));
-          k_cd_head<<<heads_b, CDH_THREADS, sm_head, st>>>(hp);
+          cudaLaunchConfig_t cfg = {};
+          cfg.gridDim = dim3((unsigned)(heads_b * csize));
+          cfg.blockDim = dim3(CDH_THREADS);
+          cfg.dynamicSmemBytes = sm_head;
+          cfg.stream = st;
+          cudaLaunchAttribute attr[1];
+          attr[0].id = cudaLaunchAttributeClusterDimension;
+          attr[0].val.clusterDim.x = (unsigned)csize;
+          attr[0].val.clusterDim.y = 1;
+          attr[0].val.clusterDim.z = 1;
+          cfg.attrs = attr;
+          cfg.numAttrs = 1;
+          TB_CUDA_CHECK(cudaLaunchKernelEx(&cfg, k_cd_head, hp));
           TB_LAUNCH_CHECK();
           k_axpy<<<ew_blocks(nb_el), 256, 0, st>>>(p.Dm + r0 * d, hp.Uacc, nb_el);
           TB_LAUNCH_CHECK();
