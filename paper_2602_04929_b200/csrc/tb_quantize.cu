@@ -1728,7 +1728,10 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
     g.n_batch = units;
     g.a_batch = g.c_batch = (long long)g.M * d;
     g.b_batch = (units > 1) ? dd : 0;
-    TB_TRY((gemm_launch<double, float, double, double, false, true>(g, st)));
+    // Z = dW H_in (+ 2 W R).  After the scale refinement without R the buffer Dm already holds
+    // dW H_in for the final scales (it was kept current through the pass), so the product is skipped.
+    const bool dm_is_current = p.cd && !with_r;
+    if (!dm_is_current) TB_TRY((gemm_launch<double, float, double, double, false, true>(g, st)));
     if (with_r) {
       GemmP h = g;
       h.A = W;
