@@ -3,7 +3,7 @@
 // Per step i (a group of g = out_block rows of every head, M = n_heads * g
 // rows in all, heads being independent):
 //   grid     k_grid           Algorithm 1 line 9    candidate search per (row, column group)
-//   sweep    k_sweep_block    Algorithm 2 / Eq. 2   one launch per 128-column block
+//   sweep    k_sweep_rows     Algorithm 2 / Eq. 2   one launch, 8 rows per CTA for the whole sweep
 //   residual k_residual       E = W0 - Q_B          (Proposition 3.1)
 //            GEMM             E -= W0 C             (Proposition 3.2, only with R)
 //   update   GEMM             W~[rem] -= T_i E      (Algorithm 1 line 11)
@@ -239,249 +239,35 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) k_grid(GridP p) {
 }
 
 // ---------------------------------------------------------------------------
-// Column sweep (Algorithm 2; Eq. 2), one launch per 128-column block `blk`.
-//
-// Panel CTAs (8 warps, one active row per warp) finish block `blk`: they apply
-// the previous block's errors to the block's columns, then walk its 128
-// columns in order -- quantize, form the normalised error, feed it back into
-// the columns to the right -- in four 32-column sub-blocks with one lane per
-// column; after a sub-block its 32 errors update the rest of the block.
-// Trailing CTAs apply the previous block's errors (a rank-128 update, rank-256
-// with the P term) to every column block right of `blk`, as GEMM tiles.  Both
-// read Err(blk-1); the panel writes Err(blk).  Stream order between launches
-// is the only synchronisation.
-// ---------------------------------------------------------------------------
-struct SweepP {
-  double* Wk;            // [M][d] working rows
-  const float* U;        // [n_hin][d][d]
-  const float* P;        // [n_hin][d][d] or nullptr
-  double* Err;           // [2][M][128] normalised errors of a block
-  double* Warr;          // [2][M][128] arrival values of a block (P term) or nullptr
-  unsigned char* codes;  // [d_out][d]
-  const double* sD;      // [d_out][ng]
-  const int* z;          // [d_out][ng]
-  tb_stats* stats;       // or nullptr
-  RowMap rm;
-  int M, d, seg, ng, maxq, blk, nblk;
-  int units, rows_per_unit;
-  int panel_ctas_per_unit, n_panel_ctas;
-  int trail_mtiles_per_unit, trail_ntiles;
-};
-
-__device__ __forceinline__ void sweep_panel(const SweepP& p, int pc, unsigned char* smem_raw) {
-  float* sU = reinterpret_cast<float*>(smem_raw);  // [128][128] diagonal block of U
-  float* sP = sU + 128 * 128;                      // [128][128] diagonal block of P (if any)
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int unit = pc / p.panel_ctas_per_unit;
-  const int rloc = (pc % p.panel_ctas_per_unit) * 8 + warp;
-  const int d = p.d, c0 = p.blk * 128;
-  const bool withP = (p.P != nullptr);
-  const float* U = p.U + (long long)unit * d * d * (p.units > 1 ? 1 : 0);
-  const float* Pm = withP ? p.P + (long long)unit * d * d * (p.units > 1 ? 1 : 0) : nullptr;
-
-  // stage the diagonal blocks (float4; rows c0+j, columns c0..c0+127)
-  for (int idx = tid; idx < 128 * 32; idx += GEMM_THREADS) {
-    const int j = idx >> 5, c4 = (idx & 31) * 4;
-    const float4 v = *reinterpret_cast<const float4*>(U + (long long)(c0 + j) * d + c0 + c4);
-    *reinterpret_cast<float4*>(sU + j * 128 + c4) = v;
-    if (withP) {
-      const float4 q = *reinterpret_cast<const float4*>(Pm + (long long)(c0 + j) * d + c0 + c4);
-      *reinterpret_cast<float4*>(sP + j * 128 + c4) = q;
-    }
-  }
-  __syncthreads();
-  if (rloc >= p.rows_per_unit) return;
-
-  const int m = unit * p.rows_per_unit + rloc;
-  const long long grow = p.rm.row(m);
-  const double maxq = (double)p.maxq;
-
-  double w[4];
-  const double* wrow = p.Wk + (long long)m * d + c0;
-#pragma unroll
-  for (int sb = 0; sb < 4; ++sb) w[sb] = wrow[sb * 32 + lane];
-
-  if (p.blk > 0) {
-    const long long eoff = ((long long)((p.blk - 1) & 1) * p.M + m) * 128;
-    const double* Ep = p.Err + eoff;
-    const float* Up = U + (long long)(c0 - 128) * d + c0 + lane;
-#pragma unroll 4
-    for (int j = 0; j < 128; ++j) {
-      const double ej = Ep[j];
-      const float* ur = Up + (long long)j * d;
-      w[0] = fma(-ej, (double)ur[0], w[0]);
-      w[1] = fma(-ej, (double)ur[32], w[1]);
-      w[2] = fma(-ej, (double)ur[64], w[2]);
-      w[3] = fma(-ej, (double)ur[96], w[3]);
-    }
-    if (withP) {
-      const double* Ap = p.Warr + eoff;
-      const float* Pp = Pm + (long long)(c0 - 128) * d + c0 + lane;
-#pragma unroll 4
-      for (int j = 0; j < 128; ++j) {
-        const double aj = Ap[j];
-        const float* pr = Pp + (long long)j * d;
-        w[0] = fma(-aj, (double)pr[0], w[0]);
-        w[1] = fma(-aj, (double)pr[32], w[1]);
-        w[2] = fma(-aj, (double)pr[64], w[2]);
-        w[3] = fma(-aj, (double)pr[96], w[3]);
-      }
-    }
-  }
-
-  unsigned int n_near = 0, n_clamp = 0;
-  const long long cur = ((long long)(p.blk & 1) * p.M + m) * 128;
-#pragma unroll
-  for (int sb = 0; sb < 4; ++sb) {
-    const int cl = sb * 32 + lane;  // column inside the block
-    const int col = c0 + cl;
-    const long long so = grow * p.ng + col / p.seg;
-    const double s_l = p.sD[so], z_l = (double)p.z[so];
-    const double rs_l = 1.0 / s_l;
-    const double rd_l = 1.0 / (double)sU[cl * 128 + cl];
-    const double srd_l = s_l * rd_l;
-    double u[32];
-#pragma unroll
-    for (int j = 0; j < 32; ++j) u[j] = (double)sU[(sb * 32 + j) * 128 + cl];
-
-    double v = w[sb];
-    if (!withP) {
-#pragma unroll
-      for (int j = 0; j < 32; ++j) {
-        // e = (v - s (q - z)) / U_jj, arranged so that the rounding is the only
-        // long dependency: e = (v + s z) / U_jj - (s / U_jj) q
-        const double ard = fma(s_l, z_l, v) * rd_l;
-        double q = rne(fma(v, rs_l, z_l));
-        q = fmin(fmax(q, 0.0), maxq);
-        const double e = fma(-srd_l, q, ard);
-        const double ej = shfl_d(e, j);
-        if (lane > j) v = fma(-ej, u[j], v);
-      }
-    } else {
-      double pu[32];
-#pragma unroll
-      for (int j = 0; j < 32; ++j) pu[j] = (double)sP[(sb * 32 + j) * 128 + cl];
-#pragma unroll
-      for (int j = 0; j < 32; ++j) {
-        const double ard = fma(s_l, z_l, v) * rd_l;
-        double q = rne(fma(v, rs_l, z_l));
-        q = fmin(fmax(q, 0.0), maxq);
-        const double e = fma(-srd_l, q, ard);
-        const double ej = shfl_d(e, j);
-        const double vj = shfl_d(v, j);  // value of column j on arrival
-        if (lane > j) v = fma(-vj, pu[j], fma(-ej, u[j], v));
-      }
-    }
-    // v is now this lane's value on arrival at its own column
-    const double x = fma(v, rs_l, z_l);
-    const double xr = rne(x);
-    const double q = fmin(fmax(xr, 0.0), maxq);
-    const double e_mine = fma(-srd_l, q, fma(s_l, z_l, v) * rd_l);
-    p.codes[grow * d + col] = (unsigned char)(int)q;
-    p.Err[cur + cl] = e_mine;
-    if (withP) p.Warr[cur + cl] = v;
-    {
-      const double fl = floor(x);
-      const double a0 = fmin(fmax(fl, 0.0), maxq), a1 = fmin(fmax(fl + 1.0, 0.0), maxq);
-      if (fabs(x - (fl + 0.5)) < 1e-6 && a0 != a1) ++n_near;
-      if (xr != q) ++n_clamp;
-    }
-    // the sub-block's errors update the later sub-blocks of this block
-    if (sb < 3) {
-#pragma unroll 8
-      for (int j = 0; j < 32; ++j) {
-        const double ej = shfl_d(e_mine, j);
-        const float* ur = sU + (sb * 32 + j) * 128 + lane;
-#pragma unroll
-        for (int sb2 = sb + 1; sb2 < 4; ++sb2) w[sb2] = fma(-ej, (double)ur[sb2 * 32], w[sb2]);
-        if (withP) {
-          const double vj = shfl_d(v, j);
-          const float* pr = sP + (sb * 32 + j) * 128 + lane;
-#pragma unroll
-          for (int sb2 = sb + 1; sb2 < 4; ++sb2) w[sb2] = fma(-vj, (double)pr[sb2 * 32], w[sb2]);
-        }
-      }
-    }
-  }
-  if (p.stats) {
-    n_near = __reduce_add_sync(0xffffffffu, n_near);
-    n_clamp = __reduce_add_sync(0xffffffffu, n_clamp);
-    if (lane == 0) {
-      if (n_near) atomicAdd(&p.stats->near_tie_codes, (unsigned long long)n_near);
-      if (n_clamp) atomicAdd(&p.stats->clamped_codes, (unsigned long long)n_clamp);
-      if (pc == 0 && warp == 0) atomicAdd(&p.stats->column_steps, 128ull);
-    }
-  }
-}
-
-__global__ void __launch_bounds__(GEMM_THREADS, 1) k_sweep_block(SweepP p) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  const int bid = blockIdx.x;
-  if (bid < p.n_panel_ctas) {
-    sweep_panel(p, bid, smem_raw);
-    return;
-  }
-  // trailing tile: Wk[:, cols] -= Err(blk-1) U[blk-1 rows, cols]  (- Warr(blk-1) P[...])
-  const int t = bid - p.n_panel_ctas;
-  const int per_unit = p.trail_mtiles_per_unit * p.trail_ntiles;
-  const int unit = t / per_unit;
-  const int mt = (t % per_unit) / p.trail_ntiles, nt = (t % per_unit) % p.trail_ntiles;
-  const int d = p.d, prev = p.blk - 1;
-  const long long uoff = (long long)unit * d * d * (p.units > 1 ? 1 : 0);
-  GemmP g;
-  g.A = p.Err + ((long long)(prev & 1) * p.M + (long long)unit * p.rows_per_unit) * 128;
-  g.a_m = 128;
-  g.a_k = 1;
-  g.B = p.U + uoff + (long long)prev * 128 * d;
-  g.b_k = d;
-  g.b_n = 1;
-  g.C = p.Wk + (long long)unit * p.rows_per_unit * d;
-  g.ldc = d;
-  g.a_batch = g.b_batch = g.c_batch = 0;
-  g.M = p.rows_per_unit;
-  g.N = d;
-  g.K = 128;
-  g.n_batch = 1;
-  g.alpha = -1.0;
-  g.beta = 1.0;
-  g.flags = 0;
-  g.btrim = g.boff = g.atrim = g.aoff = 0;
-  const int m0 = mt * GEMM_BM, n0 = (p.blk + 1 + nt) * GEMM_BN;
-  gemm_tile<double, float, double, double, false, true>(g, m0, n0, 0, smem_raw);
-  if (p.P) {
-    g.A = p.Warr + ((long long)(prev & 1) * p.M + (long long)unit * p.rows_per_unit) * 128;
-    g.B = p.P + uoff + (long long)prev * 128 * d;
-    gemm_tile<double, float, double, double, false, true>(g, m0, n0, 0, smem_raw);
-  }
-}
-
-// ---------------------------------------------------------------------------
-// Column sweep without the propagated-error term, one launch per step
-// (Algorithm 2 with P = 0; Eq. 2).  Rows never interact inside the sweep, so a
-// CTA keeps 8 active rows for the whole sweep and no CTA ever waits for another.
+// Column sweep (Algorithm 2; Eq. 2), one launch per step.  Rows never interact
+// inside the sweep, so a CTA keeps 8 active rows for the whole sweep and no CTA
+// ever waits for another.
 //
 // Left-looking form: the values of block b on arrival are
-//   w[:, b] = W0[:, b] - Err[:, 0 : 128 b] U[0 : 128 b, b],
-// where Err holds the normalised errors of the columns already quantized.
-// 16 warps: warps 0-7 are the panel warps (one row each, one lane per column,
-// the 128 columns of a block strictly in order); warps 8-15 are the update
-// warps (two 8-column fragments each, on the FP64 tensor pipe).  While the
-// panel warps walk block b, the update warps form the part of block b+1's sum
-// that needs only blocks < b: 64-row chunks of U and of the error history
-// arrive by TMA (one box each, 8 spare columns per row so that fragment loads
-// are free of bank conflicts) in a 3-stage ring guarded by full / empty
-// mbarriers; when the panel is done they add the last 128 terms (errors of
-// block b straight from shared memory) and hand block b+1 over.  The two warp
-// groups meet at hardware barriers with fixed participant counts; every trip
-// count depends on the block index alone.  mbarrier waits are bounded: when a
-// bound runs out the kernel raises a device error word and stops computing, but
-// still passes every barrier, so it always terminates.
+//   w[:, b] = W0[:, b] - Err[:, 0 : 128 b] U[0 : 128 b, b]  (- Arr[:, 0 : 128 b] P[0 : 128 b, b]),
+// where Err holds the normalised errors and Arr the arrival values of the
+// columns already quantized (the second product only with the propagated-error
+// term, WITH_P).  16 warps: warps 0-7 are the panel warps (one row each, one
+// lane per column, the 128 columns of a block strictly in order); warps 8-15
+// are the update warps (two 8-column fragments each, on the FP64 tensor pipe).
+// While the panel warps walk block b, the update warps form the part of block
+// b+1's sum that needs only blocks < b: 64-row chunks of U (and P) and of the
+// histories arrive by TMA (one box each, 8 spare columns per row so that
+// fragment loads are free of bank conflicts) in a ring guarded by full / empty
+// mbarriers; when the panel is done they add the last 128 terms (block b's
+// errors and arrival values straight from shared memory) and hand block b+1
+// over.  The two warp groups meet at hardware barriers with fixed participant
+// counts; every trip count depends on the block index alone.  mbarrier waits
+// are bounded: when a bound runs out the kernel raises a device error word and
+// stops computing, but still passes every barrier, so it always terminates.
 // ---------------------------------------------------------------------------
-enum { RS_THREADS = 512, RS_STAGES = 3, RS_LDB = 136, RS_LDE = 68, RS_CHUNK = 64, RS_LDW = 132 };
+enum { RS_THREADS = 512, RS_LDB = 136, RS_LDE = 68, RS_CHUNK = 64, RS_LDW = 132, RS_TRI = 10240 };
 struct RowSweepP {
   const double* Wt;      // [d_out][d] current W~ (rows of the step are read, never written)
   const float* U;        // [n_hin][d][d]
+  const float* P;        // [n_hin][d][d] (WITH_P)
   double* ErrG;          // [M][d] normalised errors of the step's rows
+  double* ArrG;          // [M][d] arrival values of the step's rows (WITH_P)
   unsigned char* codes;  // [d_out][d]
   const double* sD;      // [d_out][ng]
   const int* z;          // [d_out][ng]
@@ -491,15 +277,22 @@ struct RowSweepP {
   int units, rows_per_unit, ctas_per_unit;
 };
 struct RowSweepStage {
-  float Ub[RS_CHUNK][RS_LDB];   // 64 rows of U: 128 columns of the target block + 8 spare
-  double Eb[8][RS_LDE];         // the same 64 columns of the error history (+ 4 spare), 8 rows
+  float Ub[RS_CHUNK][RS_LDB];   // 64 rows of U or P: 128 columns of the target block + 8 spare
+  double Eb[8][RS_LDE];         // the same 64 columns of a history (+ 4 spare), 8 rows
 };
+// The panel only touches the upper triangle of a diagonal block: rows of sub-block sb
+// (32 rows) are stored from column 32 sb on, 128 - 32 sb wide.
+__host__ __device__ constexpr int tri_base(int sb) { return sb * 4096 - 512 * sb * (sb - 1); }
+template <bool WITH_P>
 struct RowSweepSmem {
-  float sU[128 * 128];          // diagonal block of U
-  RowSweepStage ring[RS_STAGES];
-  double wblk[8][RS_LDW];       // arrival values of the current block
+  static constexpr int STAGES = WITH_P ? 3 : 4;
+  float sU[RS_TRI];             // diagonal block of U, upper part
+  float sP[WITH_P ? RS_TRI : 4];
+  alignas(128) RowSweepStage ring[STAGES];  // TMA destinations
+  double wblk[8][128];          // arrival values of the current block before its own feedback
   double Es[8][RS_LDW];         // normalised errors of the current block
-  unsigned long long full_bar[RS_STAGES], empty_bar[RS_STAGES];
+  double As[WITH_P ? 8 : 1][RS_LDW];  // arrival values of the current block
+  unsigned long long full_bar[STAGES], empty_bar[STAGES];
   int abort_flag;
 };
 __device__ int g_sweep_error = 0;
@@ -511,26 +304,33 @@ __device__ __forceinline__ void mma_f64(double (&c)[2], double a, double b) {
 }
 __device__ __forceinline__ void bar_all() { asm volatile("bar.sync 3, 512;" ::: "memory"); }
 
+template <bool WITH_P>
 __global__ void __launch_bounds__(RS_THREADS, 1)
-    k_sweep_rows(RowSweepP p, const __grid_constant__ CUtensorMap map_u, const __grid_constant__ CUtensorMap map_e) {
+    k_sweep_rows(RowSweepP p, const __grid_constant__ CUtensorMap map_u, const __grid_constant__ CUtensorMap map_e,
+                 const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_a) {
   extern __shared__ __align__(128) unsigned char rs_raw[];
-  RowSweepSmem& sm = *reinterpret_cast<RowSweepSmem*>(rs_raw);
+  using Smem = RowSweepSmem<WITH_P>;
+  constexpr int STAGES = Smem::STAGES;
+  constexpr int NOP = WITH_P ? 2 : 1;  // operand pairs per 64-row chunk: (Err, U) and (Arr, P)
+  Smem& sm = *reinterpret_cast<Smem*>(rs_raw);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int unit = blockIdx.x / p.ctas_per_unit;
   const int r_first = (blockIdx.x % p.ctas_per_unit) * 8;  // first row of this CTA inside its unit
   const int d = p.d;
-  const float* U = p.U + (long long)unit * d * d * (p.units > 1 ? 1 : 0);
+  const long long uoff = (long long)unit * d * d * (p.units > 1 ? 1 : 0);
+  const float* U = p.U + uoff;
+  const float* Pm = WITH_P ? p.P + uoff : nullptr;
   const double maxq = (double)p.maxq;
   const int m_base = unit * p.rows_per_unit + r_first;
   const int rows_here = min(8, p.rows_per_unit - r_first);
 
-  // block 0 arrives unchanged; error rows of absent rows stay zero in every ring stage
+  // block 0 arrives unchanged
   for (int idx = tid; idx < 8 * 128; idx += RS_THREADS) {
     const int r = idx >> 7, c = idx & 127;
     sm.wblk[r][c] = (r < rows_here) ? p.Wt[p.rm.row(m_base + r) * d + c] : 0.0;
   }
   if (tid == 0) {
-    for (int s = 0; s < RS_STAGES; ++s) {
+    for (int s = 0; s < STAGES; ++s) {
       mbar_init(smem_u32(&sm.full_bar[s]), 1);
       mbar_init(smem_u32(&sm.empty_bar[s]), 8);  // one arrival per update warp
     }
@@ -555,10 +355,17 @@ __global__ void __launch_bounds__(RS_THREADS, 1)
         s4[sb] = valid ? p.sD[so] : 1.0;
         z4[sb] = valid ? (double)p.z[so] : 0.0;
       }
+      // upper part of the diagonal block(s): row r of sub-block sb from column 32 sb on
       for (int idx = tid; idx < 128 * 32; idx += 256) {
-        const int j = idx >> 5, c4 = (idx & 31) * 4;
-        *reinterpret_cast<float4*>(sm.sU + j * 128 + c4) =
-            *reinterpret_cast<const float4*>(U + (long long)(c0 + j) * d + c0 + c4);
+        const int r = idx >> 5, c4 = (idx & 31) * 4, sb = r >> 5;
+        if (c4 >= 32 * sb) {
+          const int o = tri_base(sb) + (r - 32 * sb) * (128 - 32 * sb) + (c4 - 32 * sb);
+          *reinterpret_cast<float4*>(sm.sU + o) =
+              *reinterpret_cast<const float4*>(U + (long long)(c0 + r) * d + c0 + c4);
+          if (WITH_P)
+            *reinterpret_cast<float4*>(sm.sP + o) =
+                *reinterpret_cast<const float4*>(Pm + (long long)(c0 + r) * d + c0 + c4);
+        }
       }
       asm volatile("bar.sync 2, 256;" ::: "memory");
       double w[4], rs4[4], rd4[4];
@@ -566,11 +373,14 @@ __global__ void __launch_bounds__(RS_THREADS, 1)
       for (int sb = 0; sb < 4; ++sb) {
         w[sb] = sm.wblk[warp][sb * 32 + lane];
         rs4[sb] = 1.0 / s4[sb];
-        rd4[sb] = 1.0 / (double)sm.sU[(sb * 32 + lane) * 129];
+        rd4[sb] = 1.0 / (double)sm.sU[tri_base(sb) + lane * (128 - 32 * sb) + lane];
       }
 #pragma unroll 1
       for (int sb = 0; sb < 4; ++sb) {
         const int cl = sb * 32 + lane, col = c0 + cl;
+        const int wd = 128 - 32 * sb;                 // width of this sub-block's stored rows
+        const float* ub = sm.sU + tri_base(sb) + lane;  // element (32 sb + j, 32 sb + lane + 32 t) at ub[j * wd + 32 t]
+        const float* pb = sm.sP + (WITH_P ? tri_base(sb) + lane : 0);
         const double s_l = (sb == 0) ? s4[0] : (sb == 1) ? s4[1] : (sb == 2) ? s4[2] : s4[3];
         const double z_l = (sb == 0) ? z4[0] : (sb == 1) ? z4[1] : (sb == 2) ? z4[2] : z4[3];
         const double rs_l = (sb == 0) ? rs4[0] : (sb == 1) ? rs4[1] : (sb == 2) ? rs4[2] : rs4[3];
@@ -580,7 +390,7 @@ __global__ void __launch_bounds__(RS_THREADS, 1)
         const double zm_l = z_l + magic;
         float u[32];
 #pragma unroll
-        for (int j = 0; j < 32; ++j) u[j] = sm.sU[(sb * 32 + j) * 128 + cl];
+        for (int j = 0; j < 32; ++j) u[j] = ub[j * wd];
         double v = (sb == 0) ? w[0] : (sb == 1) ? w[1] : (sb == 2) ? w[2] : w[3];
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
@@ -594,24 +404,30 @@ __global__ void __launch_bounds__(RS_THREADS, 1)
           const double q = __hiloint2double(0x43380000, n) - magic;
           const double e = fma(-srd_l, q, ard);
           const double ej = shfl_d(e, j);
-          if (lane > j) v = fma(-ej, (double)u[j], v);
+          if (WITH_P) {
+            const double vj = shfl_d(v, j);  // value of column j on arrival
+            if (lane > j) v = fma(-vj, (double)pb[j * wd], fma(-ej, (double)u[j], v));
+          } else {
+            if (lane > j) v = fma(-ej, (double)u[j], v);
+          }
         }
         const double x = fma(v, rs_l, z_l);
         const double xr = fma(v, rs_l, zm_l) - magic;
         const double q = fmin(fmax(xr, 0.0), maxq);
         const double e_mine = fma(-srd_l, q, fma(v, rd_l, szrd_l));  // the value broadcast at step `lane`
         sm.Es[warp][cl] = valid ? e_mine : 0.0;
+        if (WITH_P) sm.As[warp][cl] = valid ? v : 0.0;
         if (valid) {
           p.codes[grow * d + col] = (unsigned char)(int)q;
           p.ErrG[(long long)(m_base + warp) * d + col] = e_mine;
+          if (WITH_P) p.ArrG[(long long)(m_base + warp) * d + col] = v;
           const double fl = floor(x);
           const double a0 = fmin(fmax(fl, 0.0), maxq), a1 = fmin(fmax(fl + 1.0, 0.0), maxq);
           if (fabs(x - (fl + 0.5)) < 1e-6 && a0 != a1) ++n_near;
           if (xr != q) ++n_clamp;
         }
-        // the sub-block's errors update the later sub-blocks of this block (one branch-free loop
-        // per case, so that shuffles, loads and multiply-adds of different j overlap)
-        const float* ub = sm.sU + (sb * 32) * 128 + lane;
+        // the sub-block's errors (and arrival values) update the later sub-blocks of this block:
+        // one branch-free loop per case, so that shuffles, loads and multiply-adds of different j overlap
         if (sb == 0) {
 #pragma unroll 8
           for (int j = 0; j < 32; ++j) {
@@ -619,23 +435,38 @@ __global__ void __launch_bounds__(RS_THREADS, 1)
             w[1] = fma(-ej, (double)ub[j * 128 + 32], w[1]);
             w[2] = fma(-ej, (double)ub[j * 128 + 64], w[2]);
             w[3] = fma(-ej, (double)ub[j * 128 + 96], w[3]);
+            if (WITH_P) {
+              const double vj = shfl_d(v, j);
+              w[1] = fma(-vj, (double)pb[j * 128 + 32], w[1]);
+              w[2] = fma(-vj, (double)pb[j * 128 + 64], w[2]);
+              w[3] = fma(-vj, (double)pb[j * 128 + 96], w[3]);
+            }
           }
         } else if (sb == 1) {
 #pragma unroll 8
           for (int j = 0; j < 32; ++j) {
             const double ej = shfl_d(e_mine, j);
-            w[2] = fma(-ej, (double)ub[j * 128 + 64], w[2]);
-            w[3] = fma(-ej, (double)ub[j * 128 + 96], w[3]);
+            w[2] = fma(-ej, (double)ub[j * 96 + 32], w[2]);
+            w[3] = fma(-ej, (double)ub[j * 96 + 64], w[3]);
+            if (WITH_P) {
+              const double vj = shfl_d(v, j);
+              w[2] = fma(-vj, (double)pb[j * 96 + 32], w[2]);
+              w[3] = fma(-vj, (double)pb[j * 96 + 64], w[3]);
+            }
           }
         } else if (sb == 2) {
 #pragma unroll 8
           for (int j = 0; j < 32; ++j) {
             const double ej = shfl_d(e_mine, j);
-            w[3] = fma(-ej, (double)ub[j * 128 + 96], w[3]);
+            w[3] = fma(-ej, (double)ub[j * 64 + 32], w[3]);
+            if (WITH_P) {
+              const double vj = shfl_d(v, j);
+              w[3] = fma(-vj, (double)pb[j * 64 + 32], w[3]);
+            }
           }
         }
       }
-      // the error history is read back by TMA (async proxy): order these stores before it
+      // the histories are read back by TMA (async proxy): order these stores before it
       asm volatile("fence.proxy.async;" ::: "memory");
       bar_all();  // block b is quantized: its errors are in Es and in the history
       bar_all();  // block b+1 has been handed over in wblk
@@ -673,8 +504,8 @@ __global__ void __launch_bounds__(RS_THREADS, 1)
       break;
     }
     const int cn = (b + 1) * 128;            // first column of the target block
-    const int n_hist = 2 * b;                // chunks whose errors come from the history (blocks < b)
-    const int n_all = n_hist + 2;            // plus the two chunks of block b itself
+    const int n_hist = 2 * b * NOP;          // steps whose left operand comes from a history (blocks < b)
+    const int n_all = n_hist + 2 * NOP;      // plus the two chunks of block b itself
     double acc[2][2][2];
 #pragma unroll
     for (int i = 0; i < 8; ++i) (&acc[0][0][0])[i] = 0.0;
@@ -686,32 +517,40 @@ __global__ void __launch_bounds__(RS_THREADS, 1)
       for (int e = 0; e < 2; ++e)
         w0[t][e] = fr_valid ? p.Wt[fr_grow * d + cn + n_lo + 2 * (2 * fk + e) + t] : 0.0;
 
+    // step c: 64-row chunk c / NOP of the contraction, operand pair c % NOP
     auto produce = [&](int c) {   // producer thread only
       if (c < n_all) {
         RowSweepStage& st = sm.ring[p_slot];
         const uint32_t fb = smem_u32(&sm.full_bar[p_slot]);
         if (mbar_wait(smem_u32(&sm.empty_bar[p_slot]), p_phase ^ 1u, abort_flag, &g_sweep_error)) {
           const bool hist = c < n_hist;
+          const bool second = WITH_P && (c & 1);
+          const int kc = c / NOP;
           mbar_expect_tx(fb, (uint32_t)(sizeof(st.Ub) + (hist ? sizeof(st.Eb) : 0)));
-          tma_load_2d(smem_u32(&st.Ub[0][0]), &map_u, cn, u_row0 + c * RS_CHUNK, fb);
-          if (hist) tma_load_2d(smem_u32(&st.Eb[0][0]), &map_e, c * RS_CHUNK, m_base, fb);
+          tma_load_2d(smem_u32(&st.Ub[0][0]), second ? &map_p : &map_u, cn, u_row0 + kc * RS_CHUNK, fb);
+          if (hist) tma_load_2d(smem_u32(&st.Eb[0][0]), second ? &map_a : &map_e, kc * RS_CHUNK, m_base, fb);
         }
-        if (++p_slot == RS_STAGES) {
+        if (++p_slot == STAGES) {
           p_slot = 0;
           p_phase ^= 1u;
         }
       }
     };
-    if (producer) {
-      produce(0);
-      produce(1);
-    }
+    if (producer)
+      for (int c = 0; c < STAGES - 1; ++c) produce(c);
     for (int c = 0; c < n_all; ++c) {
-      if (c == n_hist) bar_all();  // the panel warps have finished block b: Es is complete
+      if (c == n_hist) bar_all();  // the panel warps have finished block b: Es (and As) are complete
       const RowSweepStage& st = sm.ring[c_slot];
       const bool ok = mbar_wait(smem_u32(&sm.full_bar[c_slot]), c_phase, abort_flag, &g_sweep_error);
       if (ok) {
-        const double* ap = (c < n_hist) ? &st.Eb[fr][fk] : &sm.Es[fr][(c - n_hist) * RS_CHUNK + fk];
+        const int own = (c - n_hist) / NOP;  // which of block b's two chunks (when c >= n_hist)
+        const double* ap;
+        if (c < n_hist)
+          ap = &st.Eb[fr][fk];
+        else if (WITH_P && (c & 1))
+          ap = &sm.As[fr][own * RS_CHUNK + fk];
+        else
+          ap = &sm.Es[fr][own * RS_CHUNK + fk];
         const float* bp = &st.Ub[fk][n_lo + 2 * fr];
 #pragma unroll
         for (int q = 0; q < 16; ++q) {
@@ -723,11 +562,11 @@ __global__ void __launch_bounds__(RS_THREADS, 1)
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&sm.empty_bar[c_slot]));  // this warp is done with the stage
-      if (++c_slot == RS_STAGES) {
+      if (++c_slot == STAGES) {
         c_slot = 0;
         c_phase ^= 1u;
       }
-      if (producer) produce(c + 2);
+      if (producer) produce(c + STAGES - 1);
     }
 #pragma unroll
     for (int t = 0; t < 2; ++t)
@@ -1155,7 +994,7 @@ struct Plan {
   int Mmax;
   long long cd_rows;  // rows per coordinate-descent batch
   // workspace
-  double *Wt, *Wk, *W0c, *E, *Err, *Warr, *sD, *T, *Dq, *Dm, *Yw, *n0, *Amat, *G2;
+  double *Wt, *Wk, *W0c, *E, *sD, *T, *Dq, *Dm, *Yw, *n0, *Amat, *G2;
   float* Wb;
   size_t ws_total;
 };
@@ -1210,8 +1049,6 @@ static tb_status make_plan(const tb_layer_desc* D, bool has_hout, bool with_r, b
   p.Wk = b.take<double>((size_t)p.Mmax * dd);
   p.E = b.take<double>((size_t)p.Mmax * dd);
   p.W0c = with_r ? b.take<double>((size_t)p.Mmax * dd) : nullptr;
-  p.Err = b.take<double>((size_t)2 * p.Mmax * 128);
-  p.Warr = with_r ? b.take<double>((size_t)2 * p.Mmax * 128) : nullptr;
   p.sD = b.take<double>((size_t)p.d_out * p.ng);
   p.T = (has_hout && p.S > 1) ? b.take<double>((size_t)p.H * p.S * p.dh * p.g) : nullptr;
   p.Dq = p.Dm = p.Yw = p.n0 = p.Amat = p.G2 = nullptr;
@@ -1314,12 +1151,26 @@ static tb_status run_grid(const Plan& p, const float* H_in, float* scales, int* 
   return TB_OK;
 }
 
-static tb_status run_sweep_rows(const Plan& p, const float* U_in, unsigned char* codes,
+template <bool WITH_P>
+static tb_status launch_sweep_rows(const RowSweepP& sp, const CUtensorMap& mu, const CUtensorMap& me,
+                                   const CUtensorMap& mp, const CUtensorMap& ma, cudaStream_t st) {
+  auto kern = k_sweep_rows<WITH_P>;
+  static bool configured[64] = {false};
+  TB_TRY(allow_smem(kern, sizeof(RowSweepSmem<WITH_P>), configured));
+  const long long ctas = (long long)sp.ctas_per_unit * sp.units;
+  kern<<<(unsigned)ctas, RS_THREADS, sizeof(RowSweepSmem<WITH_P>), st>>>(sp, mu, me, mp, ma);
+  TB_LAUNCH_CHECK();
+  return TB_OK;
+}
+
+static tb_status run_sweep_rows(const Plan& p, const float* U_in, const float* P, unsigned char* codes,
                                 const int* zeros, tb_stats* stats, RowMap rm, int M, cudaStream_t st) {
   RowSweepP sp;
   sp.Wt = p.Wt;
   sp.U = U_in;
-  sp.ErrG = p.Wk;  // the working-row buffer of the multi-launch sweep doubles as the error history
+  sp.P = P;
+  sp.ErrG = p.Wk;  // error history of the step's rows
+  sp.ArrG = p.E;   // arrival values; E itself is formed after the sweep
   sp.codes = codes;
   sp.sD = p.sD;
   sp.z = zeros;
@@ -1334,56 +1185,19 @@ static tb_status run_sweep_rows(const Plan& p, const float* U_in, unsigned char*
   sp.units = (p.n_hin == 1) ? 1 : p.H;
   sp.rows_per_unit = M / sp.units;
   sp.ctas_per_unit = (sp.rows_per_unit + 7) / 8;
-  static bool configured[64] = {false};
-  TB_TRY(allow_smem(k_sweep_rows, sizeof(RowSweepSmem), configured));
-  CUtensorMap map_u, map_e;
+  CUtensorMap map_u, map_e, map_p, map_a;
   const unsigned box_u = (unsigned)((p.d >= RS_LDB) ? RS_LDB : p.d), box_e = (unsigned)((p.d >= RS_LDE) ? RS_LDE : p.d);
-  TB_TRY(make_map_2d(&map_u, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, sizeof(float), U_in, (unsigned long long)p.d,
-                     (unsigned long long)p.d * sp.units, box_u, RS_CHUNK, CU_TENSOR_MAP_SWIZZLE_NONE));
+  const unsigned long long mat_rows = (unsigned long long)p.d * sp.units;
+  TB_TRY(make_map_2d(&map_u, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, sizeof(float), U_in, (unsigned long long)p.d, mat_rows,
+                     box_u, RS_CHUNK, CU_TENSOR_MAP_SWIZZLE_NONE));
   TB_TRY(make_map_2d(&map_e, CU_TENSOR_MAP_DATA_TYPE_FLOAT64, sizeof(double), sp.ErrG, (unsigned long long)p.d,
                      (unsigned long long)M, box_e, 8, CU_TENSOR_MAP_SWIZZLE_NONE));
-  const long long ctas = (long long)sp.ctas_per_unit * sp.units;
-  k_sweep_rows<<<(unsigned)ctas, RS_THREADS, sizeof(RowSweepSmem), st>>>(sp, map_u, map_e);
-  TB_LAUNCH_CHECK();
-  return TB_OK;
-}
-
-static tb_status run_sweep(const Plan& p, const float* U_in, const float* P, unsigned char* codes,
-                           const int* zeros, tb_stats* stats, RowMap rm, int M, cudaStream_t st) {
-  SweepP sp;
-  sp.Wk = p.Wk;
-  sp.U = U_in;
-  sp.P = P;
-  sp.Err = p.Err;
-  sp.Warr = p.Warr;
-  sp.codes = codes;
-  sp.sD = p.sD;
-  sp.z = zeros;
-  sp.stats = stats;
-  sp.rm = rm;
-  sp.M = M;
-  sp.d = p.d;
-  sp.seg = p.seg;
-  sp.ng = p.ng;
-  sp.maxq = p.maxq;
-  sp.nblk = p.d / 128;
-  sp.units = (p.n_hin == 1) ? 1 : p.H;
-  sp.rows_per_unit = M / sp.units;
-  sp.panel_ctas_per_unit = (sp.rows_per_unit + 7) / 8;
-  sp.n_panel_ctas = sp.panel_ctas_per_unit * sp.units;
-  sp.trail_mtiles_per_unit = (sp.rows_per_unit + GEMM_BM - 1) / GEMM_BM;
-  const size_t smem = P ? (size_t)2 * 128 * 128 * sizeof(float) : GemmSmem<double>::bytes;
-  static bool configured[64] = {false};
-  TB_TRY(allow_smem(k_sweep_block, (size_t)2 * 128 * 128 * sizeof(float), configured));
-  for (int blk = 0; blk < sp.nblk; ++blk) {
-    sp.blk = blk;
-    sp.trail_ntiles = (blk > 0) ? (sp.nblk - blk - 1) : 0;
-    const long long ctas =
-        sp.n_panel_ctas + (long long)sp.units * sp.trail_mtiles_per_unit * sp.trail_ntiles;
-    k_sweep_block<<<(unsigned)ctas, GEMM_THREADS, smem, st>>>(sp);
-    TB_LAUNCH_CHECK();
-  }
-  return TB_OK;
+  if (!P) return launch_sweep_rows<false>(sp, map_u, map_e, map_u, map_e, st);
+  TB_TRY(make_map_2d(&map_p, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, sizeof(float), P, (unsigned long long)p.d, mat_rows,
+                     box_u, RS_CHUNK, CU_TENSOR_MAP_SWIZZLE_NONE));
+  TB_TRY(make_map_2d(&map_a, CU_TENSOR_MAP_DATA_TYPE_FLOAT64, sizeof(double), sp.ArrG, (unsigned long long)p.d,
+                     (unsigned long long)M, box_e, 8, CU_TENSOR_MAP_SWIZZLE_NONE));
+  return launch_sweep_rows<true>(sp, map_u, map_e, map_p, map_a, st);
 }
 
 }  // namespace tb
@@ -1469,14 +1283,11 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
     }
     {
       PhaseScope ph(PH_SWEEP, st);
-      if (with_r) {
-        // with the propagated-error term: one launch per column block
-        k_gather<<<ew_blocks((long long)M * d), 256, 0, st>>>(p.Wt, p.Wk, p.W0c, rm, M, d);
+      if (with_r) {  // the snapshot W0 as a contiguous GEMM operand of the propagated-error term
+        k_gather<<<ew_blocks((long long)M * d), 256, 0, st>>>(p.Wt, p.W0c, nullptr, rm, M, d);
         TB_LAUNCH_CHECK();
-        TB_TRY(run_sweep(p, U_in, P, codes, zeros, stats, rm, M, st));
-      } else {
-        TB_TRY(run_sweep_rows(p, U_in, codes, zeros, stats, rm, M, st));
       }
+      TB_TRY(run_sweep_rows(p, U_in, P, codes, zeros, stats, rm, M, st));
     }
     const int nrem = p.dh - i0 - p.g;
     if (!p.has_hout || nrem <= 0) continue;
