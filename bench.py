@@ -193,8 +193,111 @@ def cpu_baseline(cfg, proj, budget_s: float = 20.0):
                       f"{dt:.1f} s; Hessian accumulation and factorisation not included"}
 
 
+def report_configs(args):
+    """Times tb_quantize_layer on every projection of the five configurations (device-resident
+    inputs; Hessians from 16384 synthetic tokens, which changes no shape) and prints one JSON
+    line per projection: seconds per layer, out-channels/s of the whole call and of the group
+    loop (grid + sweep + compensation), and the loop's fraction of the FP64 peak."""
+    import torch
+    import paper_2602_04929_b200 as tb
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    n_tok = args.tokens or 16384
+    only = set(args.only.split(",")) if args.only else None
+    for name, cfg in tb_inputs.CONFIGS.items():
+        if only and name not in only:
+            continue
+        d = cfg.d_model
+        cache = {}
+
+        def hessian(tag, with_r):
+            if tag in cache:
+                return cache[tag]
+            rec = tb_inputs.HeavyTailRecipe(d, seed=0, tid_shift=0 if tag == "attn" else 1)
+            if name == "tiny":
+                X = torch.from_numpy(tb_inputs.activations_gaussian(0, cfg.n_tok, d)).to(dev)
+                Xfp = None
+            elif with_r:
+                xs, xf = tb_inputs.DeviationRecipe(rec).chunk(0, n_tok)
+                X = torch.from_numpy(xs).to(dev).to(torch.bfloat16)
+                Xfp = torch.from_numpy(xf).to(dev).to(torch.bfloat16)
+            else:
+                X = torch.from_numpy(rec.chunk(0, n_tok)).to(dev).to(torch.bfloat16)
+                Xfp = None
+            H = torch.zeros((d, d), dtype=torch.float32, device=dev)
+            tb.tb_accumulate_hessian(H, X)
+            R = None
+            if Xfp is not None:
+                R = torch.zeros((d, d), dtype=torch.float32, device=dev)
+                tb.tb_accumulate_cross(R, X, Xfp, cfg.alpha)
+            Hsum = torch.empty_like(H)
+            tb.tb_finalize_hessian(H, R, X.shape[0], cfg.damp, Hsum_out=Hsum)
+            U, info = tb.tb_factor(H)
+            assert int(info.max().item()) == 0
+            P = C = None
+            if R is not None:
+                P, C = tb.tb_prepare_correction(R, U)
+            cache[tag] = (H, Hsum, U, R, P, C)
+            return cache[tag]
+
+        for proj in cfg.projections:
+            H, Hsum, U, R, P, C = hessian("o" if proj.name == "o" else "attn", cfg.with_r)
+            W = torch.from_numpy(tb_inputs.weight(0, proj.d_out, proj.d_in, tid=tb_inputs.T_W + (hash(proj.name) % 3))).to(dev)
+            Hout = Uout = None
+            if name == "tiny":
+                Hout = torch.from_numpy(tb_inputs.spd_matrix(0, proj.d_head)[None]).to(dev)
+            elif proj.partner in ("k", "q"):
+                gh = cfg.n_kv_heads if proj.partner == "k" else cfg.n_q_heads
+                G = torch.from_numpy(tb_inputs.weight(0, gh * cfg.d_head, d, tid=tb_inputs.T_WPARTNER)).to(dev)
+                Hout = tb.tb_build_hout(G, Hsum, proj.n_heads, proj.d_head, cfg.damp)
+            elif proj.partner == "o":
+                G = torch.from_numpy(tb_inputs.weight(0, cfg.n_q_heads * cfg.d_head, d, tid=tb_inputs.T_WOUT)).to(dev)
+                Hout = tb.tb_build_hout(G, None, proj.n_heads, proj.d_head, cfg.damp)
+            if Hout is not None:
+                Uout, info = tb.tb_factor(Hout)
+                assert int(info.max().item()) == 0
+            blocks = [cfg.out_block] if name != "l2_70b_block" or proj.name != "q" else [1, 8, 32, 64, 128]
+            for g in blocks:
+                flags = (FLAGS_ADAPT if cfg.adaptive else 0) | (FLAGS_CD if cfg.cd else 0)
+                desc = tb.layer_desc(proj.d_out, proj.d_in, proj.n_heads, proj.d_head, cfg.bits, cfg.quant_group,
+                                     g if Hout is not None else proj.d_head, flags=flags)
+                ws = torch.empty(tb.tb_quantize_layer_workspace(desc, R is not None, True), dtype=torch.uint8, device=dev)
+                res = None
+                for rep in range(3):
+                    if rep == 1:
+                        tb.tb_profile_enable(True)
+                        torch.cuda.synchronize()
+                        t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+                        t0.record()
+                    res = tb.tb_quantize_layer(desc, W, H, U, Hout, Uout, R, P, C, ws=ws, out=res)
+                t1.record()
+                torch.cuda.synchronize()
+                ms = t0.elapsed_time(t1) / 2
+                q = {k: v / 2 for k, v in tb.tb_profile_read().items()}
+                tb.tb_profile_enable(False)
+                loop_ms = q["grid"] + q["sweep"] + q["compensation"]
+                seg = cfg.quant_group or proj.d_in
+                S = proj.d_head // g if Hout is not None else 1
+                fl = (1 + (R is not None)) * proj.d_out * proj.d_in ** 2 + 2.0 * 16 * proj.d_out * proj.d_in * seg * \
+                    (1 if cfg.adaptive else 1) + (2.0 * (1 + (R is not None)) * proj.d_out * proj.d_in ** 2 if (R is not None and S > 1) else 0)
+                print(json.dumps({"config": name, "projection": proj.name, "shape": [proj.d_out, proj.d_in],
+                                  "heads": proj.n_heads, "out_block": g, "bits": cfg.bits, "with_r": R is not None,
+                                  "adaptive": cfg.adaptive, "cd": cfg.cd, "ms_per_layer": ms,
+                                  "out_channels_per_s": proj.d_out / (ms * 1e-3), "phases_ms": q, "loop_ms": loop_ms,
+                                  "loop_out_channels_per_s": proj.d_out / (loop_ms * 1e-3),
+                                  "loop_tflops": fl / (loop_ms * 1e-3) / 1e12,
+                                  "loop_frac_of_fp64_peak": fl / (loop_ms * 1e-3) / 1e12 / FP64_ALU_PEAK_TFLOPS,
+                                  "device_error_flag": tb.tb_device_error_flag()}), flush=True)
+                del ws
+        del cache
+        torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--report-configs", action="store_true",
+                    help="time tb_quantize_layer on every projection of the five configurations")
+    ap.add_argument("--only", default="", help="comma-separated config names for --report-configs")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
@@ -208,6 +311,9 @@ def main():
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
+    if args.report_configs:
+        report_configs(args)
+        return
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

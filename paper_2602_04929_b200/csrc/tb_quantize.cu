@@ -965,14 +965,16 @@ __global__ void __launch_bounds__(256) k_loss_hout(const float* __restrict__ Hou
   }
 }
 
-// H_out = I: loss[h] = sum over the head's rows of <Z[r,:], dW[r,:]>
-__global__ void __launch_bounds__(256) k_loss_identity(const double* __restrict__ Z,
-                                                       const double* __restrict__ Dq,
-                                                       double* __restrict__ loss,
-                                                       long long rows_per_head, int d) {
+// H_out = I: loss[h] = sum over the head's rows of <Z[r,:], dW[r,:]>, in two steps with a
+// fixed order: one partial sum per block of 32 rows, then the partial sums of a head.
+__global__ void __launch_bounds__(256) k_loss_identity_partial(const double* __restrict__ Z,
+                                                               const double* __restrict__ Dq,
+                                                               double* __restrict__ partial,
+                                                               long long rows_per_head, int d, int chunks) {
   __shared__ double part[8];
-  const int h = blockIdx.x;
-  const long long base = (long long)h * rows_per_head * d, n = rows_per_head * d;
+  const int h = blockIdx.y, c = blockIdx.x;
+  const long long r0 = (long long)c * 32, r1 = (r0 + 32 < rows_per_head) ? r0 + 32 : rows_per_head;
+  const long long base = ((long long)h * rows_per_head + r0) * d, n = (r1 - r0) * d;
   double acc = 0.0;
   for (long long i = threadIdx.x; i < n; i += blockDim.x) acc = fma(Z[base + i], Dq[base + i], acc);
   acc = warp_sum(acc);
@@ -981,7 +983,14 @@ __global__ void __launch_bounds__(256) k_loss_identity(const double* __restrict_
   if (threadIdx.x == 0) {
     double t = 0.0;
     for (int i = 0; i < 8; ++i) t += part[i];
-    loss[h] = t;
+    partial[(long long)h * chunks + c] = t;
+  }
+}
+__global__ void k_loss_identity_final(const double* __restrict__ partial, double* __restrict__ loss, int chunks) {
+  if (threadIdx.x == 0) {
+    double t = 0.0;
+    for (int c = 0; c < chunks; ++c) t += partial[(long long)blockIdx.x * chunks + c];
+    loss[blockIdx.x] = t;
   }
 }
 
@@ -1075,7 +1084,7 @@ static tb_status make_plan(const tb_layer_desc* D, bool has_hout, bool with_r, b
     p.n0 = b.take<double>((size_t)lines * p.ng);
     p.Amat = b.take<double>((size_t)lines * p.ng * p.ng);
   }
-  if (with_loss && has_hout) p.G2 = b.take<double>((size_t)p.H * p.dh * p.dh);
+  if (with_loss) p.G2 = b.take<double>((size_t)p.H * p.dh * (has_hout ? p.dh : 1));  // Z dW^T, or partial sums
   p.ws_total = b.total();
   return TB_OK;
 }
@@ -1571,7 +1580,10 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
       TB_TRY((gemm_launch<double, double, double, double, false, false>(q, st)));
       k_loss_hout<<<p.H, 256, 0, st>>>(H_out, p.G2, loss, p.dh);
     } else {
-      k_loss_identity<<<p.H, 256, 0, st>>>(p.Dm, p.Dq, loss, p.dh, d);
+      const int chunks = (p.dh + 31) / 32;
+      k_loss_identity_partial<<<dim3(chunks, p.H), 256, 0, st>>>(p.Dm, p.Dq, p.G2, p.dh, d, chunks);
+      TB_LAUNCH_CHECK();
+      k_loss_identity_final<<<p.H, 32, 0, st>>>(p.G2, loss, chunks);
     }
     TB_LAUNCH_CHECK();
   }

@@ -102,3 +102,34 @@ def test_llama7b_q_proj_shape_sampled_heads():
     gpu = run_gpu(prob, 2, 128, 32, ADAPT | CD)
     rep = compare(prob, gpu, 2, 128, 32, ADAPT | CD, heads=[0, 21], label="7b-q sampled heads")
     assert rep["gpu_stats"]["column_steps"] == 4 * 4096
+
+
+def test_llama7b_q_proj_with_propagated_error_sampled_head():
+    """Config 3's q_proj: 4096 x 4096, 32 heads, INT2, group 128, g = 32, adaptive grid + CD, with the
+    propagated-error operands R, P, C (alpha = 0.25) from a synthetic input deviation."""
+    prob = make_problem(0, 4096, 32, 128, 8192, with_r=True)
+    gpu = run_gpu(prob, 2, 128, 32, ADAPT | CD)
+    compare(prob, gpu, 2, 128, 32, ADAPT | CD, heads=[9], label="7b-q with R, sampled head")
+
+
+def test_llama3_gqa_k_proj_shape_sampled_head():
+    """Config 4's k_proj: 1024 x 4096, 8 key/value heads whose H_out sums 4 query heads each, INT3, g = 64."""
+    prob = make_problem(1, 4096, 8, 128, 8192, g_heads=32)
+    gpu = run_gpu(prob, 3, 128, 64, ADAPT | CD)
+    compare(prob, gpu, 3, 128, 64, ADAPT | CD, heads=[5], label="8b-k GQA, sampled head")
+
+
+def test_o_proj_identity_hout_sampled_rows():
+    """o_proj of the block configs: H_out = NULL (all 4096 rows at once); the oracle recomputes 128 of them."""
+    prob = make_problem(2, 4096, 32, 128, 8192, hout=None)
+    gpu = run_gpu(prob, 2, 128, 32, ADAPT | CD)
+    compare(prob, gpu, 2, 128, 32, ADAPT | CD, heads=[3], label="o_proj GPTQ mode, sampled rows")
+
+
+@pytest.mark.parametrize("g", [32, 1])
+def test_llama70b_q_proj_shape_sampled_head(g):
+    """Config 5's q_proj: 8192 x 8192, 64 heads x 128, INT2, group 128, fixed grid, no CD (the paper's
+    'BoA + joint quantization' setting), at g = 32 and at g = 1 (BoA's sequential rule)."""
+    prob = make_problem(3, 8192, 64, 128, 8192)
+    gpu = run_gpu(prob, 2, 128, g, 0)
+    compare(prob, gpu, 2, 128, g, 0, heads=[37], label=f"70b-q g={g}, sampled head")
