@@ -114,28 +114,31 @@ class ClockSampler:
 
 
 def count_launches(cfg, proj, n_tok: int, with_loss=True) -> int:
-    """Kernel launches of one step, counted from the launch loops of the library."""
+    """Kernel launches of one step of this library (torch's own fill / reduce kernels not counted),
+    from the launch loops of the library for a shared H_in without the propagated-error term."""
     d, dh, H = proj.d_in, proj.d_head, proj.n_heads
-    g = cfg.out_block if proj.partner else dh
+    has_hout = bool(proj.partner)
+    g = cfg.out_block if has_hout else dh
     S = dh // g
-    nblk = d // 128
-    n = 0
-    n += -(-n_tok // 4096) + 1 + 2                      # accumulate launches, mirror, finalize (2)
-    if proj.partner:
-        n += 3                                          # G Hsum, per-head Gram, combine
-    for (dd, nb) in ((d, 1),) + (((dh, H),) if proj.partner else ()):
+
+    def factor(dd):
         blocks = -(-dd // 64)
-        levels = max(0, (blocks - 1).bit_length())
-        n += 1 + blocks + (blocks - 1) + 1 + 2 * levels * (nb if blocks > 2 and nb > 1 else 1) + 1   # reverse, panels, trailing updates, block inverses, doubling levels, reverse
-    n += 1 + (1 if S > 1 else 0)                        # widen, compensation matrices
-    n += (S if cfg.adaptive else 1)                     # grid
-    n += S * (1 + nblk)                                 # gather + one launch per column block
-    n += (S - 1) * 2 if proj.partner else 0             # residual + compensation GEMM
+        dp_blocks = 1 << max(0, (blocks - 1).bit_length())
+        levels = dp_blocks.bit_length() - 1
+        return 1 + blocks + (blocks - 1) + 1 + 2 * levels + 1   # reverse, panels, trailing, block inverses, doubling, reverse
+
+    n = 1 + 1 + 2                                       # tensor-core accumulate, mirror, finalize (2)
+    if has_hout:
+        n += 3                                          # G Hsum, per-head Gram, combine
+    n += factor(d) + (factor(dh) if has_hout else 0)
+    n += 1 + (1 if has_hout and S > 1 else 0)           # widen, compensation matrices
+    n += (S if cfg.adaptive else 1) + S                 # grid search, one sweep launch per step
+    n += 2 * (S - 1) if has_hout else 0                 # residual + compensation GEMM
     if cfg.cd:
-        n += 1 + 2 + 2 * (dh if proj.partner else 1)    # prep, Dm and Yw products, two kernels per row step
+        n += 3 + (3 if has_hout else 2)                 # prep, Dm, Yw; then G, cluster pass, refresh (or two row kernels)
     n += 1                                              # dequant
     if with_loss:
-        n += 2 + (2 if proj.partner else 1)
+        n += 1 + (0 if cfg.cd else 1) + 2               # prep, (Z product), Z dW^T / partial sums, reduction
     return n
 
 
