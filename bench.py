@@ -41,6 +41,13 @@ FLAGS_ADAPT, FLAGS_CD = 1, 2
 FP64_ALU_PEAK_TFLOPS = 148 * 64 * 2 * 1.965e9 / 1e12
 # FP32 FMA peak: 148 SMs x 128 lanes x 2 x 1.965 GHz
 FP32_ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under
+# profiles/ (full-size workload, one launch each); filled in when a capture of the current kernel exists
+NCU_TRAFFIC = {
+    ("l2_7b_q", "k_sweep_rows"): 78.0e6,   # 69.4 MB read + 8.6 MB written per launch (4 launches per layer)
+    ("l2_7b_q", "k_grid"): 35.7e6,         # per launch (4 launches per layer)
+    ("l2_7b_q", "k_syrk_tc"): 6.667e9,     # one launch per layer; X itself is 2.15 GB
+}
 
 
 def workload(name: str):
@@ -474,32 +481,54 @@ def main():
         return
 
     # ---- rooflines (algorithmic work / measured phase time) ----
-    S = dh // (cfg.out_block if G is not None else dh)
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except OSError:
+        pass
+    bf16_peak = float(peaks.get("bf16_tflops", 1590.0))
+    bf16_kind = "measured cuBLAS bf16 burst (MEASURED_PEAKS.json)" if peaks else "fallback 1.59 PFLOP/s"
     seg = cfg.quant_group or d
+    has_hout = G is not None
+    # issued tensor-core work of the Hessian: 128 x 256 tiles on or below the diagonal
+    m_blocks = -(-d // 128)
+    syrk_tiles = sum(mi // 2 + 1 for mi in range(m_blocks))
     fl = {
-        "hessian": 2.0 * n_tok * d * d,                           # X^T X (the symmetric half is skipped)
+        "hessian": 2.0 * 128 * 256 * n_tok * syrk_tiles,
+        "gemm": 2.0 * d_out * d * d + 2.0 * d_out * dh * d,     # G Hsum, then the per-head Grams
         "sweep": 1.0 * d_out * d * d,                             # d_in^2 flop per out-channel
-        "grid": 2.0 * 16 * d_out * d * seg * (1 if cfg.adaptive else 1),
-        "cd": (4.0 * d_out * d * d) if cfg.cd else 0.0,           # (Q-W) H_in and the blockwise Wbar H_in
+        "grid": 2.0 * 16 * d_out * d * seg,
+        "cd": (4.0 * d_out * d * d + 2.0 * d_out * dh * d + 3.0 * d_out * d * (d // seg)) if cfg.cd else 0.0,
     }
+    fp64_kind = "FP64 FMA / FP64 tensor pipe, 148 SM x 64 lanes x 2 x 1.965 GHz"
     roof_all = {}
     if phases.get("hessian"):
         t = phases["hessian"] * 1e-3
-        roof_all["hessian"] = {"bound": "alu", "achieved": fl["hessian"] / t / 1e12, "peak": FP32_ALU_PEAK_TFLOPS,
-                               "unit": "TFLOP/s", "peak_kind": "FP32 FMA, 148 SM x 128 lanes x 2 x 1.965 GHz"}
+        roof_all["hessian"] = {"kernel": "k_syrk_tc (+ zero, mirror, finalize)", "bound": "tensor",
+                               "achieved": fl["hessian"] / t / 1e12, "peak": bf16_peak, "unit": "TFLOP/s",
+                               "peak_kind": bf16_kind}
+    if has_hout and phases.get("hout"):
+        t = phases["hout"] * 1e-3
+        roof_all["gemm"] = {"kernel": "gemm_kernel<float,float,double,double> (timed through tb_build_hout)",
+                            "bound": "alu", "achieved": fl["gemm"] / t / 1e12, "peak": FP64_ALU_PEAK_TFLOPS,
+                            "unit": "TFLOP/s", "peak_kind": fp64_kind}
+    names = {"sweep": "k_sweep_rows", "grid": "k_grid", "cd": "scale refinement (3 GEMMs + k_cd_head)"}
     for nm in ("sweep", "grid", "cd"):
         if q_ms.get(nm) and fl[nm]:
             t = q_ms[nm] * 1e-3
-            roof_all[nm] = {"bound": "alu", "achieved": fl[nm] / t / 1e12, "peak": FP64_ALU_PEAK_TFLOPS,
-                            "unit": "TFLOP/s", "peak_kind": "FP64 FMA, 148 SM x 64 lanes x 2 x 1.965 GHz"}
-    for v in roof_all.values():
+            roof_all[nm] = {"kernel": names[nm], "bound": "alu", "achieved": fl[nm] / t / 1e12,
+                            "peak": FP64_ALU_PEAK_TFLOPS, "unit": "TFLOP/s", "peak_kind": fp64_kind}
+    # DRAM traffic per launch from the committed ncu captures (profiles/), bytes; None where no capture applies
+    traffic = {"sweep": NCU_TRAFFIC.get((cfg.name, "k_sweep_rows")), "grid": NCU_TRAFFIC.get((cfg.name, "k_grid")),
+               "gemm": NCU_TRAFFIC.get((cfg.name, "gemm_hout")), "hessian": NCU_TRAFFIC.get((cfg.name, "k_syrk_tc"))}
+    for k, v in roof_all.items():
         v["frac"] = v["achieved"] / v["peak"]
-        v["traffic"] = None
-    times = {"hessian": phases.get("hessian", 0.0), "sweep": q_ms.get("sweep", 0.0), "grid": q_ms.get("grid", 0.0),
-             "cd": q_ms.get("cd", 0.0)}
-    dominant = max(times, key=times.get)
-    roofline = dict(roof_all.get(dominant, {}), kernel=dominant)
+        v["traffic"] = traffic.get(k) if not args.heads and not args.tokens else None
+    # the kernel with the largest share of the step: the FP64 GEMM engine (H_out build, Dm, Yw, factor updates)
+    dominant = "gemm" if "gemm" in roof_all else "sweep"
+    roofline = dict(roof_all.get(dominant, {}))
     loop_ms = q_ms.get("grid", 0.0) + q_ms.get("sweep", 0.0) + q_ms.get("compensation", 0.0)
+    loop_fl = fl["sweep"] + fl["grid"] + (1.0 * d_out * d * (dh - cfg.out_block) if has_hout else 0.0)
 
     line = {
         "metric": METRIC, "value": d_out * world / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world,
@@ -513,6 +542,9 @@ def main():
         "phases_ms": dict(phases, **{"quantize/" + k: v for k, v in q_ms.items()}),
         "loop_ms": loop_ms,
         "loop_out_channels_per_s": d_out / (loop_ms * 1e-3) if loop_ms else None,
+        "loop_roofline": {"bound": "alu", "achieved": loop_fl / (loop_ms * 1e-3) / 1e12 if loop_ms else None,
+                          "peak": FP64_ALU_PEAK_TFLOPS, "unit": "TFLOP/s",
+                          "frac": loop_fl / (loop_ms * 1e-3) / 1e12 / FP64_ALU_PEAK_TFLOPS if loop_ms else None},
         "clocks": clocks, "gpu_launches": count_launches(cfg, proj, n_tok) * args.steps,
         "roofline": roofline, "rooflines": roof_all,
     }
