@@ -1,0 +1,267 @@
+// Blockwise product Yw[r][g][:] = Wbar[r, G_g] H_in[G_g, :] of the scale refinement
+// (Algorithm 3: one row of products per scale) on the 5th-generation tensor cores.
+//
+// Wbar = W_int - z holds small integers, exact in bf16.  H_in (float) is split
+// exactly into three bf16 pieces, H = H1 + H2 + H3 (8 + 8 + 8 mantissa bits), so
+// every product Wbar * H_p is exact in float and the only rounding is the float
+// accumulation of 3 * |G_g| terms per output in tensor memory.  The result is
+// stored in float: it feeds coefficients and small corrections of the
+// refinement, where a relative error of a few 1e-7 is three orders of magnitude
+// below the tolerance on the scales.
+//
+// Both operands are MN-major (the contraction index is the strided one): Wbar is
+// written transposed, [d_in][rows], by the preparation kernel, H_in's pieces are
+// [d_in][d_in] row-major.  Same machinery as the Hessian kernel: TMA boxes of
+// 64 x 64 with the 128-byte swizzle, mbarrier ring, tcgen05.mma kind::f16 with
+// accumulators in TMEM, two accumulator buffers so that the epilogue of one tile
+// overlaps the MMAs of the next.  Warps 0-7 epilogue, warp 8 TMA producer, warp 9
+// MMA issuer.  Every mbarrier wait is bounded.
+#include "tb_common.cuh"
+#include "tb_tma.cuh"
+
+namespace tb {
+
+enum {
+  YT_BM = 128,
+  YT_BN = 128,
+  YT_BK = 64,
+  YT_STAGES = 3,
+  YT_BOX = 64 * 64 * 2,
+  YT_A_BYTES = 2 * YT_BOX,            // Wbar^T: 64 k x 128 rows
+  YT_B_BYTES = 3 * 2 * YT_BOX,        // three pieces of H_in: 64 k x 128 columns each
+  YT_STAGE_BYTES = YT_A_BYTES + YT_B_BYTES,
+  YT_THREADS = 320,
+  YT_SMEM = YT_STAGES * YT_STAGE_BYTES + 1024 + 256
+};
+
+__device__ int g_yt_error = 0;
+
+// H (float) -> three bf16 pieces with H = p1 + p2 + p3 exactly (for finite normal values)
+__global__ void k_split3(const float* __restrict__ H, __nv_bfloat16* __restrict__ out, long long n) {
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n;
+       i += (long long)gridDim.x * blockDim.x) {
+    const float x = H[i];
+    const __nv_bfloat16 p1 = __float2bfloat16_rn(x);
+    const float r1 = x - __bfloat162float(p1);
+    const __nv_bfloat16 p2 = __float2bfloat16_rn(r1);
+    const float r2 = r1 - __bfloat162float(p2);
+    out[i] = p1;
+    out[n + i] = p2;
+    out[2 * n + i] = __float2bfloat16_rn(r2);
+  }
+}
+
+// WbT[k][r] = code[r][k] - z[r][group(k)] as bf16 (exact), tiled transpose
+__global__ void k_wbar_transpose(const unsigned char* __restrict__ codes, const int* __restrict__ z,
+                                 __nv_bfloat16* __restrict__ WbT, long long rows, int d, int seg, int ng) {
+  __shared__ float tile[32][33];
+  const long long r0 = (long long)blockIdx.y * 32;
+  const int k0 = blockIdx.x * 32;
+  for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+    const long long r = r0 + i;
+    const int k = k0 + threadIdx.x;
+    tile[i][threadIdx.x] = (r < rows) ? (float)((int)codes[r * d + k] - z[r * ng + k / seg]) : 0.0f;
+  }
+  __syncthreads();
+  for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+    const int k = k0 + i;
+    const long long r = r0 + threadIdx.x;
+    if (r < rows) WbT[(long long)k * rows + r] = __float2bfloat16_rn(tile[threadIdx.x][i]);
+  }
+}
+
+__global__ void __launch_bounds__(YT_THREADS, 1)
+    k_yw_tc(float* __restrict__ Yw, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+            int rows, int d, int seg, int ng, int n_tiles) {
+  extern __shared__ unsigned char yt_raw[];
+  const uint32_t raw = smem_u32(yt_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  unsigned char* gen_base = yt_raw + (base - raw);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(gen_base + YT_STAGES * YT_STAGE_BYTES);
+  // bars[0..2] full, [3..5] empty, [6..7] acc_full, [8..9] acc_empty; then tmem slot, abort flag
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 10);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const uint32_t bar0 = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (3 + s); };
+  auto accf_bar = [&](int b) { return bar0 + 8u * (6 + b); };
+  auto acce_bar = [&](int b) { return bar0 + 8u * (8 + b); };
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < YT_STAGES; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(accf_bar(b), 1);
+      mbar_init(acce_bar(b), 8);
+    }
+    *abort_flag = 0;
+    mbar_fence_init();
+  }
+  if (warp == 8) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(256u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int n_stages = seg / YT_BK;                       // stages per tile
+  const int m_tiles = (rows + YT_BM - 1) / YT_BM, n_tilesN = (d + YT_BN - 1) / YT_BN;
+  // tile t -> (group g, row tile mi, column tile nj), column tiles innermost
+  auto tile_of = [&](int t, int& g, int& mi, int& nj) {
+    nj = t % n_tilesN;
+    mi = (t / n_tilesN) % m_tiles;
+    g = t / (n_tilesN * m_tiles);
+  };
+
+  if (warp == 8) {
+    if (lane == 0) {
+      uint32_t it = 0;
+      for (int t = blockIdx.x; t < n_tiles && !*abort_flag; t += gridDim.x) {
+        int g, mi, nj;
+        tile_of(t, g, mi, nj);
+        const int m0 = mi * YT_BM, n0 = nj * YT_BN, k00 = g * seg;
+        for (int st = 0; st < n_stages; ++st, ++it) {
+          const int s = it % YT_STAGES;
+          const uint32_t ph = (it / YT_STAGES) & 1u;
+          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, &g_yt_error)) break;
+          mbar_expect_tx(full_bar(s), YT_STAGE_BYTES);
+          const uint32_t sa = base + s * YT_STAGE_BYTES, sb = sa + YT_A_BYTES;
+          const int k0 = k00 + st * YT_BK;
+#pragma unroll
+          for (int j = 0; j < 2; ++j) tma_load_2d(sa + j * YT_BOX, &map_a, m0 + 64 * j, k0, full_bar(s));
+#pragma unroll
+          for (int pc = 0; pc < 3; ++pc)
+#pragma unroll
+            for (int j = 0; j < 2; ++j)
+              tma_load_2d(sb + (pc * 2 + j) * YT_BOX, &map_b, n0 + 64 * j, pc * d + k0, full_bar(s));
+        }
+      }
+    }
+  } else if (warp == 9) {
+    if (lane == 0) {
+      const uint32_t idesc = idesc_bf16_mn(YT_BM, YT_BN);
+      uint32_t it = 0, tile_it = 0;
+      for (int t = blockIdx.x; t < n_tiles && !*abort_flag; t += gridDim.x, ++tile_it) {
+        const int b = tile_it & 1;
+        if (!mbar_wait(acce_bar(b), ((tile_it >> 1) & 1u) ^ 1u, abort_flag, &g_yt_error)) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t tmem_d = tmem_base + (uint32_t)b * YT_BN;
+        bool ok = true;
+        for (int st = 0; st < n_stages; ++st, ++it) {
+          const int s = it % YT_STAGES;
+          const uint32_t ph = (it / YT_STAGES) & 1u;
+          if (!mbar_wait(full_bar(s), ph, abort_flag, &g_yt_error)) {
+            ok = false;
+            break;
+          }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t sa = base + s * YT_STAGE_BYTES, sb = sa + YT_A_BYTES;
+#pragma unroll
+          for (int kk = 0; kk < YT_BK / 16; ++kk) {
+            const uint64_t adesc = smem_desc_mn_sw128(sa + kk * 2048);
+#pragma unroll
+            for (int pc = 0; pc < 3; ++pc) {
+              const uint64_t bdesc = smem_desc_mn_sw128(sb + pc * 2 * YT_BOX + kk * 2048);
+              umma_bf16(tmem_d, adesc, bdesc, idesc, (st > 0 || kk > 0 || pc > 0) ? 1u : 0u);
+            }
+          }
+          umma_commit(empty_bar(s));
+        }
+        if (!ok) break;
+        umma_commit(accf_bar(b));
+      }
+    }
+  } else {
+    // epilogue warps 0-7: TMEM lanes 32 (w % 4) .., columns 64 (w / 4) ..
+    const int q = warp & 3, hf = warp >> 2;
+    const int row = q * 32 + lane;
+    uint32_t tile_it = 0;
+    for (int t = blockIdx.x; t < n_tiles && !*abort_flag; t += gridDim.x, ++tile_it) {
+      int g, mi, nj;
+      tile_of(t, g, mi, nj);
+      const int b = tile_it & 1;
+      if (!mbar_wait(accf_bar(b), (tile_it >> 1) & 1u, abort_flag, &g_yt_error)) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * YT_BN + hf * 64);
+      uint32_t r0[32], r1[32];
+      tmem_ld_32x32(taddr, r0);
+      tmem_ld_32x32(taddr + 32, r1);
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acce_bar(b));   // the accumulator may be overwritten
+      const long long gr = (long long)mi * YT_BM + row;
+      const int gc = nj * YT_BN + hf * 64;
+      if (gr < rows) {
+        float* dst = Yw + (gr * ng + g) * (long long)d + gc;
+#pragma unroll
+        for (int i = 0; i < 32; i += 4) {
+          if (gc + i + 3 < d)
+            *reinterpret_cast<float4*>(dst + i) = make_float4(__uint_as_float(r0[i]), __uint_as_float(r0[i + 1]),
+                                                              __uint_as_float(r0[i + 2]), __uint_as_float(r0[i + 3]));
+          if (gc + 32 + i + 3 < d)
+            *reinterpret_cast<float4*>(dst + 32 + i) = make_float4(__uint_as_float(r1[i]), __uint_as_float(r1[i + 1]),
+                                                                   __uint_as_float(r1[i + 2]), __uint_as_float(r1[i + 3]));
+        }
+      }
+    }
+  }
+
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 8) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(256u) : "memory");
+  }
+}
+
+// Yw (float, [rows][ng][d]) from the codes; WbT ([d][rows] bf16) and Hp ([3][d][d] bf16) are scratch.
+// Requires seg % 64 == 0, d % 8 == 0, rows % 8 == 0.
+tb_status yw_tensor(float* Yw, const unsigned char* codes, const int* zeros, const float* H_in, __nv_bfloat16* WbT,
+                    __nv_bfloat16* Hp, bool split_h, long long rows, int d, int seg, int ng, cudaStream_t st) {
+  const long long dd = (long long)d * d;
+  if (split_h) {
+    k_split3<<<148 * 8, 256, 0, st>>>(H_in, Hp, dd);
+    TB_LAUNCH_CHECK();
+  }
+  k_wbar_transpose<<<dim3(d / 32, (unsigned)((rows + 31) / 32)), dim3(32, 8), 0, st>>>(codes, zeros, WbT, rows, d, seg, ng);
+  TB_LAUNCH_CHECK();
+  CUtensorMap map_a, map_b;
+  TB_TRY(make_map_2d(&map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, WbT, (unsigned long long)rows, (unsigned long long)d,
+                     64, 64, CU_TENSOR_MAP_SWIZZLE_128B));
+  TB_TRY(make_map_2d(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Hp, (unsigned long long)d, (unsigned long long)3 * d,
+                     64, 64, CU_TENSOR_MAP_SWIZZLE_128B));
+  const int m_tiles = (int)((rows + YT_BM - 1) / YT_BM), n_tilesN = (d + YT_BN - 1) / YT_BN;
+  const long long n_tiles = (long long)m_tiles * n_tilesN * ng;
+  if (n_tiles > 0x7fffffffll) return TB_ERR_UNSUPPORTED;
+  int dev = 0, sms = 0;
+  TB_CUDA_CHECK(cudaGetDevice(&dev));
+  TB_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  static bool configured[64] = {false};
+  if (dev < 0 || dev >= 64) return TB_ERR_CUDA;
+  if (!configured[dev]) {
+    TB_CUDA_CHECK(cudaFuncSetAttribute(k_yw_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)YT_SMEM));
+    configured[dev] = true;
+  }
+  const int grid = (int)(n_tiles < sms ? n_tiles : sms);
+  k_yw_tc<<<grid, YT_THREADS, YT_SMEM, st>>>(Yw, map_a, map_b, (int)rows, d, seg, ng, (int)n_tiles);
+  TB_LAUNCH_CHECK();
+  return TB_OK;
+}
+
+int yw_error_read_clear() {
+  int v = 0;
+  if (cudaMemcpyFromSymbol(&v, g_yt_error, sizeof(int)) != cudaSuccess) return -1;
+  if (v) {
+    int z = 0;
+    cudaMemcpyToSymbol(g_yt_error, &z, sizeof(int));
+  }
+  return v;
+}
+
+}  // namespace tb

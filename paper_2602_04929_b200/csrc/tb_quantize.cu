@@ -24,6 +24,12 @@
 namespace cg = cooperative_groups;
 
 namespace tb {
+// tensor-core blockwise product of the scale refinement (tb_gemm_tc.cu)
+tb_status yw_tensor(float* Yw, const unsigned char* codes, const int* zeros, const float* H_in, __nv_bfloat16* WbT,
+                    __nv_bfloat16* Hp, bool split_h, long long rows, int d, int seg, int ng, cudaStream_t st);
+}
+
+namespace tb {
 
 // ---------------------------------------------------------------------------
 // Row bookkeeping.  Active row m of a step maps to head m / g, row i0 + m % g
@@ -636,7 +642,7 @@ __global__ void k_cd_prep(const float* __restrict__ W, const unsigned char* __re
 
 struct CdP {
   double* Dm;           // [rows][d]            (rows of this batch)
-  const double* Yw;     // [rows][ng][d]
+  const void* Yw;       // [rows][ng][d], element type TY of the kernel
   const float* Wb;      // [rows][d]
   const float* Hout;    // [heads][dh][dh] of this batch, or nullptr
   double* sD;           // [rows][ng]
@@ -650,6 +656,7 @@ struct CdP {
 // line = head * lines_per_head + l; its row inside the head is j0 + l.
 // Partial sums are kept per 32-column chunk and added in chunk order, so the
 // result does not depend on warp scheduling.
+template <typename TY>
 __global__ void __launch_bounds__(256) k_cd_row_stats(CdP p) {
   extern __shared__ double cd_sm[];  // part[chunks][ng + 1], then hrow[dh]
   const int tid = threadIdx.x, lane = tid & 31;
@@ -667,7 +674,7 @@ __global__ void __launch_bounds__(256) k_cd_row_stats(CdP p) {
     for (int i = tid; i < dh; i += blockDim.x) hrow[i] = (double)p.Hout[((long long)head * dh + j) * dh + i];
   __syncthreads();
   const double* Dh = p.Dm + (long long)head * dh * d;
-  const double* Yr = p.Yw + row * ng * d;
+  const TY* Yr = static_cast<const TY*>(p.Yw) + row * ng * d;
   const float* wbr = p.Wb + row * d;
   // every warp walks 32 consecutive columns at a time; they lie in one group
   for (int cb = (tid >> 5) * 32; cb < c_count; cb += (blockDim.x >> 5) * 32) {
@@ -685,7 +692,7 @@ __global__ void __launch_bounds__(256) k_cd_row_stats(CdP p) {
     const double v = warp_sum(wb * gj);
     if (lane == 0) part[chunk * (ng + 1) + ng] = v;
     for (int g2 = 0; g2 <= g; ++g2) {
-      const double a = warp_sum(Yr[(long long)g2 * d + col] * wb);
+      const double a = warp_sum((double)Yr[(long long)g2 * d + col] * wb);
       if (lane == 0) part[chunk * (ng + 1) + g2] = a;
     }
   }
@@ -702,6 +709,7 @@ __global__ void __launch_bounds__(256) k_cd_row_stats(CdP p) {
   }
 }
 
+template <typename TY>
 __global__ void __launch_bounds__(256) k_cd_row_update(CdP p) {
   extern __shared__ double cd_sm[];  // num[ng], delta[ng], then A[ng][ng] if it fits
   const int tid = threadIdx.x, lane = tid & 31;
@@ -735,12 +743,12 @@ __global__ void __launch_bounds__(256) k_cd_row_update(CdP p) {
   const int g_first = blockIdx.x * p.groups_per_cta;
   const int g_count = min(p.groups_per_cta, ng - g_first);
   const int c_first = g_first * seg, c_count = g_count * seg;
-  const double* Yr = p.Yw + row * ng * d;
+  const TY* Yr = static_cast<const TY*>(p.Yw) + row * ng * d;
   double* dm = p.Dm + row * d;
   for (int c = tid; c < c_count; c += blockDim.x) {
     const int col = c_first + c;
     double acc = dm[col];
-    for (int g2 = 0; g2 < ng; ++g2) acc = fma(delta[g2], Yr[(long long)g2 * d + col], acc);
+    for (int g2 = 0; g2 < ng; ++g2) acc = fma(delta[g2], (double)Yr[(long long)g2 * d + col], acc);
     dm[col] = acc;
   }
   if (blockIdx.x == 0)
@@ -768,7 +776,7 @@ enum { CDH_THREADS = 512, CDH_BLOCK = 16 };
 struct CdHeadP {
   double* G;           // [heads*dh][d]   H_out Dm, updated in place
   double* Uacc;        // [heads*dh][d]   out: the rank-1 vectors u_i
-  const double* Yw;    // [heads*dh][ng][d]
+  const void* Yw;      // [heads*dh][ng][d], element type TY of the kernel
   const float* Wb;     // [heads*dh][d]
   const float* Hout;   // [heads][dh][dh]
   double* sD;          // [heads*dh][ng]
@@ -777,6 +785,7 @@ struct CdHeadP {
   int uw;              // columns per work unit (a divisor of seg, multiple of 32, at most 128)
 };
 
+template <typename TY>
 __global__ void __launch_bounds__(CDH_THREADS, 1) k_cd_head(CdHeadP p) {
   extern __shared__ double cdh_sm[];
   cg::cluster_group cluster = cg::this_cluster();
@@ -801,7 +810,7 @@ __global__ void __launch_bounds__(CDH_THREADS, 1) k_cd_head(CdHeadP p) {
     const int buf = j & 1;
     const int blk0 = (j / CDH_BLOCK) * CDH_BLOCK;
     const double hjj = (double)Ho[(long long)j * dh + j];
-    const double* Yr = p.Yw + row * ng * d;
+    const TY* Yr = static_cast<const TY*>(p.Yw) + row * ng * d;
     const float* wbr = p.Wb + row * d;
     const double* Gr = p.G + row * d;
     const float* hrow = Ho + (long long)j * dh;
@@ -829,7 +838,7 @@ __global__ void __launch_bounds__(CDH_THREADS, 1) k_cd_head(CdHeadP p) {
       for (int c = 0; c < 4; ++c) v = fma(wb[c], gv[c], v);
       v = warp_sum(v);
       if (lane == 0) part[(size_t)u * (ng + 1) + ng] = v;
-      const double* yb = Yr + cbase + lane;
+      const TY* yb = Yr + cbase + lane;
       int g2 = 0;
       for (; g2 + 4 <= g + 1; g2 += 4) {
         double a4[4] = {0.0, 0.0, 0.0, 0.0};
@@ -837,7 +846,7 @@ __global__ void __launch_bounds__(CDH_THREADS, 1) k_cd_head(CdHeadP p) {
         for (int t = 0; t < 4; ++t)
 #pragma unroll
           for (int c = 0; c < 4; ++c)
-            if (lane + 32 * c < uw) a4[t] = fma(yb[(long long)(g2 + t) * d + 32 * c], wb[c], a4[t]);
+            if (lane + 32 * c < uw) a4[t] = fma((double)yb[(long long)(g2 + t) * d + 32 * c], wb[c], a4[t]);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1)
 #pragma unroll
@@ -848,7 +857,7 @@ __global__ void __launch_bounds__(CDH_THREADS, 1) k_cd_head(CdHeadP p) {
         double a = 0.0;
 #pragma unroll
         for (int c = 0; c < 4; ++c)
-          if (lane + 32 * c < uw) a = fma(yb[(long long)g2 * d + 32 * c], wb[c], a);
+          if (lane + 32 * c < uw) a = fma((double)yb[(long long)g2 * d + 32 * c], wb[c], a);
         a = warp_sum(a);
         if (lane == 0) part[(size_t)u * (ng + 1) + g2] = a;
       }
@@ -887,10 +896,10 @@ __global__ void __launch_bounds__(CDH_THREADS, 1) k_cd_head(CdHeadP p) {
       double acc[4] = {0.0, 0.0, 0.0, 0.0};
       for (int g2 = 0; g2 < ng; ++g2) {
         const double dl = delta[g2];
-        const double* y = Yr + (long long)g2 * d + c_lo + c0;
+        const TY* y = Yr + (long long)g2 * d + c_lo + c0;
 #pragma unroll
         for (int t = 0; t < 4; ++t)
-          if (c0 + t * CDH_THREADS < c_cnt) acc[t] = fma(dl, y[t * CDH_THREADS], acc[t]);
+          if (c0 + t * CDH_THREADS < c_cnt) acc[t] = fma(dl, (double)y[t * CDH_THREADS], acc[t]);
       }
 #pragma unroll
       for (int t = 0; t < 4; ++t)
@@ -1005,6 +1014,8 @@ struct Plan {
   // workspace
   double *Wt, *Wk, *W0c, *E, *sD, *T, *Dq, *Dm, *Yw, *n0, *Amat, *G2;
   float* Wb;
+  __nv_bfloat16 *WbT, *Hp;  // tensor-core path of the blockwise product
+  bool yw_tensor;
   size_t ws_total;
 };
 
@@ -1062,6 +1073,8 @@ static tb_status make_plan(const tb_layer_desc* D, bool has_hout, bool with_r, b
   p.T = (has_hout && p.S > 1) ? b.take<double>((size_t)p.H * p.S * p.dh * p.g) : nullptr;
   p.Dq = p.Dm = p.Yw = p.n0 = p.Amat = p.G2 = nullptr;
   p.Wb = nullptr;
+  p.WbT = p.Hp = nullptr;
+  p.yw_tensor = false;
   p.cd_rows = 0;
   if (p.cd || with_loss) {
     p.Dq = b.take<double>((size_t)p.d_out * dd);
@@ -1080,6 +1093,13 @@ static tb_status make_plan(const tb_layer_desc* D, bool has_hout, bool with_r, b
     if (!(has_hout || p.n_hin > 1) && rows > 128) rows = (rows / 128) * 128;
     p.cd_rows = rows;
     p.Yw = b.take<double>((size_t)rows * p.ng * dd);
+    // blockwise product on the tensor cores (float result): one shared H_in, groups that are whole TMA boxes
+    p.yw_tensor = (p.n_hin == 1) && (p.seg % 64 == 0) && (rows % 8 == 0) && (p.d_out % 8 == 0) &&
+                  (p.dh % 8 == 0 || rows == p.d_out);
+    if (p.yw_tensor) {
+      p.WbT = b.take<__nv_bfloat16>((size_t)rows * dd);
+      p.Hp = b.take<__nv_bfloat16>((size_t)3 * dd * dd);
+    }
     const long long lines = has_hout ? rows / p.dh : rows;
     p.n0 = b.take<double>((size_t)lines * p.ng);
     p.Amat = b.take<double>((size_t)lines * p.ng * p.ng);
@@ -1386,23 +1406,28 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
           h.beta = 1.0;
           TB_TRY((gemm_launch<float, float, double, double, false, true>(h, st)));
         }
-        GemmP y = gemm_params();
-        y.A = p.Wb + rr * d;
-        y.a_m = d;
-        y.a_k = 1;
-        y.a_batch = p.seg;
-        y.B = Hh;
-        y.b_k = d;
-        y.b_n = 1;
-        y.b_batch = (long long)p.seg * d;
-        y.C = p.Yw + q0 * p.ng * d;
-        y.ldc = (long long)p.ng * d;
-        y.c_batch = d;
-        y.M = (int)rows_per_prod;
-        y.N = d;
-        y.K = p.seg;
-        y.n_batch = p.ng;
-        TB_TRY((gemm_launch<float, float, double, double, false, true>(y, st)));
+        if (p.yw_tensor) {
+          TB_TRY(yw_tensor(reinterpret_cast<float*>(p.Yw), codes + rr * d, zeros + rr * p.ng, H_in, p.WbT, p.Hp,
+                           r0 == 0, rows, d, p.seg, p.ng, st));
+        } else {
+          GemmP y = gemm_params();
+          y.A = p.Wb + rr * d;
+          y.a_m = d;
+          y.a_k = 1;
+          y.a_batch = p.seg;
+          y.B = Hh;
+          y.b_k = d;
+          y.b_n = 1;
+          y.b_batch = (long long)p.seg * d;
+          y.C = p.Yw + q0 * p.ng * d;
+          y.ldc = (long long)p.ng * d;
+          y.c_batch = d;
+          y.M = (int)rows_per_prod;
+          y.N = d;
+          y.K = p.seg;
+          y.n_batch = p.ng;
+          TB_TRY((gemm_launch<float, float, double, double, false, true>(y, st)));
+        }
       }
       if (p.has_hout) {
         // rows of a head are coupled through H_out: one CTA per head walks them in order
@@ -1428,8 +1453,12 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
         const size_t sm_head =
             ((size_t)n_units * (p.ng + 1) + 2 * (size_t)p.ng * p.ng + 3 * (size_t)p.ng) * sizeof(double);
         if (sm_head > 200 * 1024) return TB_ERR_UNSUPPORTED;
-        static bool conf_head[64] = {false};
-        TB_TRY(allow_smem(k_cd_head, 200 * 1024, conf_head));
+        static bool conf_head[64] = {false}, conf_head2[64] = {false};
+        auto cd_head_kern = p.yw_tensor ? k_cd_head<float> : k_cd_head<double>;
+        if (p.yw_tensor)
+          TB_TRY(allow_smem(k_cd_head<float>, 200 * 1024, conf_head));
+        else
+          TB_TRY(allow_smem(k_cd_head<double>, 200 * 1024, conf_head2));
         for (int it = 0; it < p.cd_iters; ++it) {
           GemmP g = gemm_params();  // G = H_out Dm, head by head
           g.A = hp.Hout;
@@ -1460,7 +1489,7 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
           attr[0].val.clusterDim.z = 1;
           cfg.attrs = attr;
           cfg.numAttrs = 1;
-          TB_CUDA_CHECK(cudaLaunchKernelEx(&cfg, k_cd_head, hp));
+          TB_CUDA_CHECK(cudaLaunchKernelEx(&cfg, cd_head_kern, hp));
           TB_LAUNCH_CHECK();
           k_axpy<<<ew_blocks(nb_el), 256, 0, st>>>(p.Dm + r0 * d, hp.Uacc, nb_el);
           TB_LAUNCH_CHECK();
@@ -1497,22 +1526,32 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
         cp.a_in_smem = 0;
       }
       static bool conf_stats[64] = {false}, conf_upd[64] = {false};
-      TB_TRY(allow_smem(k_cd_row_stats, 200 * 1024, conf_stats));
-      TB_TRY(allow_smem(k_cd_row_update, 200 * 1024, conf_upd));
+      static bool conf_stats_f[64] = {false}, conf_upd_f[64] = {false};
+      TB_TRY(allow_smem(k_cd_row_stats<double>, 200 * 1024, conf_stats));
+      TB_TRY(allow_smem(k_cd_row_update<double>, 200 * 1024, conf_upd));
+      TB_TRY(allow_smem(k_cd_row_stats<float>, 200 * 1024, conf_stats_f));
+      TB_TRY(allow_smem(k_cd_row_update<float>, 200 * 1024, conf_upd_f));
+      const size_t ysz = p.yw_tensor ? sizeof(float) : sizeof(double);
       if (sm_stats > 200 * 1024) return TB_ERR_UNSUPPORTED;
       for (int it = 0; it < p.cd_iters; ++it) {
         for (int l0 = 0; l0 < lines; l0 += 65535) {
           const int nl = (lines - l0 < 65535) ? (lines - l0) : 65535;
           CdP cq = cp;  // advance every per-line pointer by l0 rows
           cq.Dm = cp.Dm + (long long)l0 * d;
-          cq.Yw = cp.Yw + (long long)l0 * p.ng * d;
+          cq.Yw = static_cast<const char*>(cp.Yw) + (size_t)l0 * p.ng * d * ysz;
           cq.Wb = cp.Wb + (long long)l0 * d;
           cq.sD = cp.sD + (long long)l0 * p.ng;
           cq.n0 = cp.n0 + (long long)l0 * p.ng;
           cq.Amat = cp.Amat + (long long)l0 * p.ng * p.ng;
-          k_cd_row_stats<<<dim3(xctas, nl), 256, sm_stats, st>>>(cq);
-          TB_LAUNCH_CHECK();
-          k_cd_row_update<<<dim3(xctas, nl), 256, sm_upd, st>>>(cq);
+          if (p.yw_tensor) {
+            k_cd_row_stats<float><<<dim3(xctas, nl), 256, sm_stats, st>>>(cq);
+            TB_LAUNCH_CHECK();
+            k_cd_row_update<float><<<dim3(xctas, nl), 256, sm_upd, st>>>(cq);
+          } else {
+            k_cd_row_stats<double><<<dim3(xctas, nl), 256, sm_stats, st>>>(cq);
+            TB_LAUNCH_CHECK();
+            k_cd_row_update<double><<<dim3(xctas, nl), 256, sm_upd, st>>>(cq);
+          }
           TB_LAUNCH_CHECK();
         }
       }

@@ -41,47 +41,6 @@ enum {
 
 __device__ int g_tc_error = 0;
 
-// MN-major, SWIZZLE_128B shared-memory matrix descriptor (see the file header).
-__device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t addr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((addr >> 4) & 0x3FFF);
-  d |= (uint64_t)((8192 >> 4) & 0x3FFF) << 16;  // leading byte offset: next 64-column box
-  d |= (uint64_t)((1024 >> 4) & 0x3FFF) << 32;  // stride byte offset: next 8 tokens
-  d |= (uint64_t)1 << 46;                       // descriptor version of this architecture
-  d |= (uint64_t)2 << 61;                       // SWIZZLE_128B
-  return d;
-}
-
-// kind::f16 instruction descriptor: D = f32, A = B = bf16, both MN-major, M = 128, N = 256.
-__device__ __forceinline__ uint32_t idesc_bf16_mn_128x256() {
-  return (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) | ((256u >> 3) << 17) | ((128u >> 4) << 24);
-}
-
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                          uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
-      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr)
-      : "memory");
-}
-
 __global__ void __launch_bounds__(TC_THREADS, 1)
     k_syrk_tc(float* __restrict__ H, const __grid_constant__ CUtensorMap xmap, int n_tok, int d, int n_tiles) {
   extern __shared__ unsigned char tc_smem_raw[];
@@ -165,7 +124,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
   } else if (warp == 9) {
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
-      const uint32_t idesc = idesc_bf16_mn_128x256();
+      const uint32_t idesc = idesc_bf16_mn(128, 256);
       uint32_t it = 0, chunk_it = 0;
       for (int t = blockIdx.x; t < n_tiles && !*abort_flag; t += gridDim.x) {
         for (int st = 0; st < n_stages; ++st, ++it) {
@@ -279,6 +238,7 @@ tb_status syrk_bf16_tensor(float* H, const __nv_bfloat16* X, long long n_tok, in
 // 0, or 1 once a bounded wait inside a tensor-core kernel has run out (sticky until read).
 namespace tb {
 int sweep_error_read_clear();  // the same word of the column-sweep kernel (tb_quantize.cu)
+int yw_error_read_clear();     // and of the tensor-core product of the scale refinement (tb_gemm_tc.cu)
 }
 
 extern "C" int tb_device_error_flag(void) {
@@ -289,6 +249,7 @@ extern "C" int tb_device_error_flag(void) {
     cudaMemcpyToSymbol(tb::g_tc_error, &z, sizeof(int));
   }
   const int w = tb::sweep_error_read_clear();
-  if (w < 0) return -1;
-  return (v || w) ? 1 : 0;
+  const int y = tb::yw_error_read_clear();
+  if (w < 0 || y < 0) return -1;
+  return (v || w || y) ? 1 : 0;
 }
