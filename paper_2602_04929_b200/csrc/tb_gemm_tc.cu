@@ -254,6 +254,236 @@ tb_status yw_tensor(float* Yw, const unsigned char* codes, const int* zeros, con
   return TB_OK;
 }
 
+// ---------------------------------------------------------------------------
+// C (double, [M][ldc]) = A B for float A [M][K] and float B [K][N], both split
+// exactly into three bf16 pieces; the six piece products that matter to float
+// accuracy (1*1, 1*2, 2*1, 1*3, 3*1, 2*2) run on tcgen05 with float
+// accumulation in TMEM over 128 contraction steps at a time, and the chunks are
+// summed in double by the epilogue warps.  Used for G Hsum of the H_out build
+// (Table 1).  A arrives transposed and split, AT [3][K][M]; B split, [3][K][N].
+// ---------------------------------------------------------------------------
+enum {
+  GS_BM = 128,
+  GS_BN = 128,
+  GS_BK = 32,
+  GS_STAGES = 4,
+  GS_CHUNK = 4,                       // stages per TMEM accumulation (128 contraction steps)
+  GS_BOX = 32 * 64 * 2,
+  GS_A_BYTES = 3 * 2 * GS_BOX,
+  GS_B_BYTES = 3 * 2 * GS_BOX,
+  GS_STAGE_BYTES = GS_A_BYTES + GS_B_BYTES,
+  GS_SMEM = GS_STAGES * GS_STAGE_BYTES + 1024 + 256
+};
+
+// AT[p][k][m] = piece p of A[m][k]
+__global__ void k_split3_transpose(const float* __restrict__ A, __nv_bfloat16* __restrict__ AT, long long M, int K) {
+  __shared__ float tile[32][33];
+  const long long m0 = (long long)blockIdx.y * 32;
+  const int k0 = blockIdx.x * 32;
+  for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+    const long long m = m0 + i;
+    const int k = k0 + threadIdx.x;
+    tile[i][threadIdx.x] = (m < M && k < K) ? A[m * K + k] : 0.0f;
+  }
+  __syncthreads();
+  const long long plane = (long long)K * M;
+  for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+    const int k = k0 + i;
+    const long long m = m0 + threadIdx.x;
+    if (m < M && k < K) {
+      const float x = tile[threadIdx.x][i];
+      const __nv_bfloat16 p1 = __float2bfloat16_rn(x);
+      const float r1 = x - __bfloat162float(p1);
+      const __nv_bfloat16 p2 = __float2bfloat16_rn(r1);
+      const long long o = (long long)k * M + m;
+      AT[o] = p1;
+      AT[plane + o] = p2;
+      AT[2 * plane + o] = __float2bfloat16_rn(r1 - __bfloat162float(p2));
+    }
+  }
+}
+
+__global__ void __launch_bounds__(YT_THREADS, 1)
+    k_gsplit_tc(double* __restrict__ C, long long ldc, const __grid_constant__ CUtensorMap map_a,
+                const __grid_constant__ CUtensorMap map_b, int M, int N, int K, int n_tiles) {
+  extern __shared__ unsigned char gs_raw[];
+  const uint32_t raw = smem_u32(gs_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  unsigned char* gen_base = gs_raw + (base - raw);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(gen_base + GS_STAGES * GS_STAGE_BYTES);
+  // bars[0..3] full, [4..7] empty, [8..9] acc_full, [10..11] acc_empty; then tmem slot, abort flag
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 12);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const uint32_t bar0 = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (4 + s); };
+  auto accf_bar = [&](int b) { return bar0 + 8u * (8 + b); };
+  auto acce_bar = [&](int b) { return bar0 + 8u * (10 + b); };
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < GS_STAGES; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(accf_bar(b), 1);
+      mbar_init(acce_bar(b), 8);
+    }
+    *abort_flag = 0;
+    mbar_fence_init();
+  }
+  if (warp == 8) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(256u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int n_stages = (K + GS_BK - 1) / GS_BK;
+  const int n_tilesN = (N + GS_BN - 1) / GS_BN;
+
+  if (warp == 8) {
+    if (lane == 0) {
+      uint32_t it = 0;
+      for (int t = blockIdx.x; t < n_tiles && !*abort_flag; t += gridDim.x) {
+        const int m0 = (t / n_tilesN) * GS_BM, n0 = (t % n_tilesN) * GS_BN;
+        for (int st = 0; st < n_stages; ++st, ++it) {
+          const int s = it % GS_STAGES;
+          const uint32_t ph = (it / GS_STAGES) & 1u;
+          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, &g_yt_error)) break;
+          mbar_expect_tx(full_bar(s), GS_STAGE_BYTES);
+          const uint32_t sa = base + s * GS_STAGE_BYTES, sb = sa + GS_A_BYTES;
+          const int k0 = st * GS_BK;
+#pragma unroll
+          for (int pc = 0; pc < 3; ++pc)
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+              tma_load_2d(sa + (pc * 2 + j) * GS_BOX, &map_a, m0 + 64 * j, pc * K + k0, full_bar(s));
+              tma_load_2d(sb + (pc * 2 + j) * GS_BOX, &map_b, n0 + 64 * j, pc * K + k0, full_bar(s));
+            }
+        }
+      }
+    }
+  } else if (warp == 9) {
+    if (lane == 0) {
+      const uint32_t idesc = idesc_bf16_mn(GS_BM, GS_BN);
+      uint32_t it = 0, chunk_it = 0;
+      for (int t = blockIdx.x; t < n_tiles && !*abort_flag; t += gridDim.x) {
+        for (int st = 0; st < n_stages; ++st, ++it) {
+          const int in_chunk = st % GS_CHUNK;
+          const int b = chunk_it & 1;
+          if (in_chunk == 0) {
+            if (!mbar_wait(acce_bar(b), ((chunk_it >> 1) & 1u) ^ 1u, abort_flag, &g_yt_error)) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          }
+          const int s = it % GS_STAGES;
+          const uint32_t ph = (it / GS_STAGES) & 1u;
+          if (!mbar_wait(full_bar(s), ph, abort_flag, &g_yt_error)) break;
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t sa = base + s * GS_STAGE_BYTES, sb = sa + GS_A_BYTES;
+          const uint32_t tmem_d = tmem_base + (uint32_t)b * GS_BN;
+          bool first = (in_chunk == 0);
+#pragma unroll
+          for (int kk = 0; kk < GS_BK / 16; ++kk) {
+            // piece pairs (a, b): 1*1, 1*2, 2*1, 1*3, 3*1, 2*2
+            const int pa[6] = {0, 0, 1, 0, 2, 1}, pb[6] = {0, 1, 0, 2, 0, 1};
+#pragma unroll
+            for (int i = 0; i < 6; ++i) {
+              const uint64_t adesc = smem_desc_mn_sw128(sa + pa[i] * 2 * GS_BOX + kk * 2048, GS_BOX);
+              const uint64_t bdesc = smem_desc_mn_sw128(sb + pb[i] * 2 * GS_BOX + kk * 2048, GS_BOX);
+              umma_bf16(tmem_d, adesc, bdesc, idesc, first ? 0u : 1u);
+              first = false;
+            }
+          }
+          umma_commit(empty_bar(s));
+          if (in_chunk == GS_CHUNK - 1 || st == n_stages - 1) {
+            umma_commit(accf_bar(b));
+            ++chunk_it;
+          }
+        }
+      }
+    }
+  } else {
+    const int q = warp & 3, hf = warp >> 2;
+    const int row = q * 32 + lane;
+    uint32_t chunk_it = 0;
+    for (int t = blockIdx.x; t < n_tiles && !*abort_flag; t += gridDim.x) {
+      const int m0 = (t / n_tilesN) * GS_BM, n0 = (t % n_tilesN) * GS_BN;
+      double run[64];
+#pragma unroll
+      for (int i = 0; i < 64; ++i) run[i] = 0.0;
+      bool ok = true;
+      for (int st0 = 0; st0 < n_stages && ok; st0 += GS_CHUNK, ++chunk_it) {
+        const int b = chunk_it & 1;
+        ok = mbar_wait(accf_bar(b), (chunk_it >> 1) & 1u, abort_flag, &g_yt_error);
+        if (!ok) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * GS_BN + hf * 64);
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          uint32_t r[32];
+          tmem_ld_32x32(taddr + c * 32, r);
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+          for (int i = 0; i < 32; ++i) run[c * 32 + i] += (double)__uint_as_float(r[i]);
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(acce_bar(b));
+      }
+      if (ok) {
+        const long long gm = (long long)m0 + row;
+        if (gm < M) {
+          double* dst = C + gm * ldc + n0 + hf * 64;
+#pragma unroll
+          for (int i = 0; i < 64; i += 2)
+            if (n0 + hf * 64 + i + 1 < N) *reinterpret_cast<double2*>(dst + i) = make_double2(run[i], run[i + 1]);
+        }
+      }
+    }
+  }
+
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 8) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(256u) : "memory");
+  }
+}
+
+// C = A B (double result) through split bf16 pieces; AT ([3][K][M]) and Bp ([3][K][N]) are scratch.
+// Requires M % 8 == 0, N % 8 == 0, K % 32 == 0.
+tb_status gemm_split_tensor(double* C, long long ldc, const float* A, const float* B, __nv_bfloat16* AT,
+                            __nv_bfloat16* Bp, long long M, int N, int K, cudaStream_t st) {
+  k_split3<<<148 * 8, 256, 0, st>>>(B, Bp, (long long)K * N);
+  TB_LAUNCH_CHECK();
+  k_split3_transpose<<<dim3((K + 31) / 32, (unsigned)((M + 31) / 32)), dim3(32, 8), 0, st>>>(A, AT, M, K);
+  TB_LAUNCH_CHECK();
+  CUtensorMap map_a, map_b;
+  TB_TRY(make_map_2d(&map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, AT, (unsigned long long)M, (unsigned long long)3 * K,
+                     64, 32, CU_TENSOR_MAP_SWIZZLE_128B));
+  TB_TRY(make_map_2d(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Bp, (unsigned long long)N, (unsigned long long)3 * K,
+                     64, 32, CU_TENSOR_MAP_SWIZZLE_128B));
+  const long long n_tiles = ((M + GS_BM - 1) / GS_BM) * (long long)((N + GS_BN - 1) / GS_BN);
+  if (n_tiles > 0x7fffffffll) return TB_ERR_UNSUPPORTED;
+  int dev = 0, sms = 0;
+  TB_CUDA_CHECK(cudaGetDevice(&dev));
+  TB_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  static bool configured[64] = {false};
+  if (dev < 0 || dev >= 64) return TB_ERR_CUDA;
+  if (!configured[dev]) {
+    TB_CUDA_CHECK(cudaFuncSetAttribute(k_gsplit_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GS_SMEM));
+    configured[dev] = true;
+  }
+  const int grid = (int)(n_tiles < sms ? n_tiles : sms);
+  k_gsplit_tc<<<grid, YT_THREADS, GS_SMEM, st>>>(C, ldc, map_a, map_b, (int)M, N, K, (int)n_tiles);
+  TB_LAUNCH_CHECK();
+  return TB_OK;
+}
+
 int yw_error_read_clear() {
   int v = 0;
   if (cudaMemcpyFromSymbol(&v, g_yt_error, sizeof(int)) != cudaSuccess) return -1;

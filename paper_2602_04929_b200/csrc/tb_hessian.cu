@@ -9,6 +9,11 @@
 namespace tb {
 
 tb_status syrk_bf16_tensor(float* H, const __nv_bfloat16* X, long long n_tok, int d, cudaStream_t st);
+tb_status gemm_split_tensor(double* C, long long ldc, const float* A, const float* B, __nv_bfloat16* AT,
+                            __nv_bfloat16* Bp, long long M, int N, int K, cudaStream_t st);
+
+// G Hsum runs on the tensor cores when the shapes fit the TMA boxes of that kernel
+static bool hout_on_tensor(int rows, int d) { return (rows % 8 == 0) && (d % 32 == 0); }
 
 // Tokens per launch: partial sums of one launch stay in float registers, the
 // running sum in H absorbs one rounding per launch.
@@ -234,6 +239,10 @@ extern "C" size_t tb_build_hout_workspace(int g_heads, int d_head, int d) {
   Bump b(nullptr);
   b.take<double>((size_t)g_heads * d_head * d);       // G Hsum
   b.take<double>((size_t)g_heads * d_head * d_head);  // per-block Grams
+  if (hout_on_tensor(g_heads * d_head, d)) {
+    b.take<__nv_bfloat16>((size_t)3 * g_heads * d_head * d);  // G^T in three bf16 pieces
+    b.take<__nv_bfloat16>((size_t)3 * d * d);                 // Hsum in three bf16 pieces
+  }
   return b.total();
 }
 
@@ -251,7 +260,13 @@ extern "C" tb_status tb_build_hout(float* H_out, const float* G, const float* Hs
   double* blocks = b.take<double>((size_t)g_heads * d_head * d_head);
   const int rows = g_heads * d_head;
   GemmP q = gemm_params();
-  if (Hsum) {
+  if (Hsum && hout_on_tensor(rows, d)) {
+    // T = G Hsum from exact bf16 splits of both operands (float-accurate products, double chunk sums)
+    __nv_bfloat16* GT = b.take<__nv_bfloat16>((size_t)3 * rows * d);
+    __nv_bfloat16* Hp = b.take<__nv_bfloat16>((size_t)3 * d * d);
+    TB_TRY(gemm_split_tensor(T, d, G, Hsum, GT, Hp, rows, d, d, st));
+    q.A = T;
+  } else if (Hsum) {
     GemmP g = gemm_params();  // T = G Hsum
     g.A = G;
     g.a_m = d;

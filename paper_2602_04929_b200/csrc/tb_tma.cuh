@@ -61,13 +61,13 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
 // stack of TMA boxes of 64 contraction rows x 64 columns (128 bytes per row, 128-byte swizzle);
 // 8 rows form one swizzle atom, atoms repeat every 1024 B along K (stride byte offset) and
 // every 8192 B (one box) along M / N (leading byte offset).
-__device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t addr) {
+__device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t addr, uint32_t box_bytes = 8192) {
   uint64_t d = 0;
   d |= (uint64_t)((addr >> 4) & 0x3FFF);
-  d |= (uint64_t)((8192 >> 4) & 0x3FFF) << 16;  // leading byte offset: next 64-column box
-  d |= (uint64_t)((1024 >> 4) & 0x3FFF) << 32;  // stride byte offset: next 8 tokens
-  d |= (uint64_t)1 << 46;                       // descriptor version of this architecture
-  d |= (uint64_t)2 << 61;                       // SWIZZLE_128B
+  d |= (uint64_t)((box_bytes >> 4) & 0x3FFF) << 16;  // leading byte offset: next 64-column box
+  d |= (uint64_t)((1024 >> 4) & 0x3FFF) << 32;       // stride byte offset: next 8 contraction rows
+  d |= (uint64_t)1 << 46;                            // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                            // SWIZZLE_128B
   return d;
 }
 

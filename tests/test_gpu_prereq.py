@@ -81,7 +81,11 @@ def test_build_hout(n_heads, g_heads, with_sum):
     Hout = tb.tb_build_hout(_t(G), _t(Hs32) if with_sum else None, n_heads, dh, 0.01)
     torch.cuda.synchronize()
     ref = oracle.hout_from_projection(G, Hs32 if with_sum else None, n_heads, dh, damp=0.01)
-    assert rel_fro(Hout.cpu().numpy(), ref) <= 1e-6
+    # G Hsum runs on the tensor cores from exact bf16 splits: the six retained piece products drop
+    # terms below 2^-24 and each 128-step chunk is accumulated in float before the double sum
+    err = rel_fro(Hout.cpu().numpy(), ref)
+    print("HOUT rel error", err)
+    assert err <= 2e-6
 
 
 @pytest.mark.parametrize("n_batch,d,cond", [(3, 200, 1e3), (1, 256, 1e5), (2, 64, 1e2), (1, 520, 1e4), (5, 128, 1e3)])
