@@ -275,15 +275,16 @@ enum {
   GS_SMEM = GS_STAGES * GS_STAGE_BYTES + 1024 + 256
 };
 
-// AT[p][k][m] = piece p of A[m][k]
-__global__ void k_split3_transpose(const float* __restrict__ A, __nv_bfloat16* __restrict__ AT, long long M, int K) {
-  __shared__ float tile[32][33];
+// AT[p][k][m] = piece p of A[m][k]; a double input keeps its leading 24 bits
+template <typename TA>
+__global__ void k_split3_transpose(const TA* __restrict__ A, __nv_bfloat16* __restrict__ AT, long long M, int K) {
+  __shared__ TA tile[32][33];
   const long long m0 = (long long)blockIdx.y * 32;
   const int k0 = blockIdx.x * 32;
   for (int i = threadIdx.y; i < 32; i += blockDim.y) {
     const long long m = m0 + i;
     const int k = k0 + threadIdx.x;
-    tile[i][threadIdx.x] = (m < M && k < K) ? A[m * K + k] : 0.0f;
+    tile[i][threadIdx.x] = (m < M && k < K) ? A[m * K + k] : (TA)0;
   }
   __syncthreads();
   const long long plane = (long long)K * M;
@@ -291,21 +292,21 @@ __global__ void k_split3_transpose(const float* __restrict__ A, __nv_bfloat16* _
     const int k = k0 + i;
     const long long m = m0 + threadIdx.x;
     if (m < M && k < K) {
-      const float x = tile[threadIdx.x][i];
-      const __nv_bfloat16 p1 = __float2bfloat16_rn(x);
-      const float r1 = x - __bfloat162float(p1);
-      const __nv_bfloat16 p2 = __float2bfloat16_rn(r1);
+      const TA x = tile[threadIdx.x][i];
+      const __nv_bfloat16 p1 = __float2bfloat16_rn((float)x);
+      const TA r1 = x - (TA)__bfloat162float(p1);  // exact in TA
+      const __nv_bfloat16 p2 = __float2bfloat16_rn((float)r1);
       const long long o = (long long)k * M + m;
       AT[o] = p1;
       AT[plane + o] = p2;
-      AT[2 * plane + o] = __float2bfloat16_rn(r1 - __bfloat162float(p2));
+      AT[2 * plane + o] = __float2bfloat16_rn((float)(r1 - (TA)__bfloat162float(p2)));
     }
   }
 }
 
 __global__ void __launch_bounds__(YT_THREADS, 1)
     k_gsplit_tc(double* __restrict__ C, long long ldc, const __grid_constant__ CUtensorMap map_a,
-                const __grid_constant__ CUtensorMap map_b, int M, int N, int K, int n_tiles) {
+                const __grid_constant__ CUtensorMap map_b, int M, int N, int K, int n_tiles, int accumulate) {
   extern __shared__ unsigned char gs_raw[];
   const uint32_t raw = smem_u32(gs_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -441,7 +442,15 @@ __global__ void __launch_bounds__(YT_THREADS, 1)
           double* dst = C + gm * ldc + n0 + hf * 64;
 #pragma unroll
           for (int i = 0; i < 64; i += 2)
-            if (n0 + hf * 64 + i + 1 < N) *reinterpret_cast<double2*>(dst + i) = make_double2(run[i], run[i + 1]);
+            if (n0 + hf * 64 + i + 1 < N) {
+              double2 v = make_double2(run[i], run[i + 1]);
+              if (accumulate) {
+                const double2 old = *reinterpret_cast<const double2*>(dst + i);
+                v.x += old.x;
+                v.y += old.y;
+              }
+              *reinterpret_cast<double2*>(dst + i) = v;
+            }
         }
       }
     }
@@ -454,14 +463,10 @@ __global__ void __launch_bounds__(YT_THREADS, 1)
   }
 }
 
-// C = A B (double result) through split bf16 pieces; AT ([3][K][M]) and Bp ([3][K][N]) are scratch.
+// C (+)= A B (double result) from operands already split: AT [3][K][M], Bp [3][K][N].
 // Requires M % 8 == 0, N % 8 == 0, K % 32 == 0.
-tb_status gemm_split_tensor(double* C, long long ldc, const float* A, const float* B, __nv_bfloat16* AT,
-                            __nv_bfloat16* Bp, long long M, int N, int K, cudaStream_t st) {
-  k_split3<<<148 * 8, 256, 0, st>>>(B, Bp, (long long)K * N);
-  TB_LAUNCH_CHECK();
-  k_split3_transpose<<<dim3((K + 31) / 32, (unsigned)((M + 31) / 32)), dim3(32, 8), 0, st>>>(A, AT, M, K);
-  TB_LAUNCH_CHECK();
+tb_status gemm_split_presplit(double* C, long long ldc, const __nv_bfloat16* AT, const __nv_bfloat16* Bp, long long M,
+                              int N, int K, bool accumulate, cudaStream_t st) {
   CUtensorMap map_a, map_b;
   TB_TRY(make_map_2d(&map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, AT, (unsigned long long)M, (unsigned long long)3 * K,
                      64, 32, CU_TENSOR_MAP_SWIZZLE_128B));
@@ -479,9 +484,36 @@ tb_status gemm_split_tensor(double* C, long long ldc, const float* A, const floa
     configured[dev] = true;
   }
   const int grid = (int)(n_tiles < sms ? n_tiles : sms);
-  k_gsplit_tc<<<grid, YT_THREADS, GS_SMEM, st>>>(C, ldc, map_a, map_b, (int)M, N, K, (int)n_tiles);
+  k_gsplit_tc<<<grid, YT_THREADS, GS_SMEM, st>>>(C, ldc, map_a, map_b, (int)M, N, K, (int)n_tiles, accumulate ? 1 : 0);
   TB_LAUNCH_CHECK();
   return TB_OK;
+}
+
+// Bp[p][i] = piece p of B[i]
+tb_status split3(const float* B, __nv_bfloat16* Bp, long long n, cudaStream_t st) {
+  k_split3<<<148 * 8, 256, 0, st>>>(B, Bp, n);
+  TB_LAUNCH_CHECK();
+  return TB_OK;
+}
+
+tb_status split3_transpose(const float* A, __nv_bfloat16* AT, long long M, int K, cudaStream_t st) {
+  k_split3_transpose<float><<<dim3((K + 31) / 32, (unsigned)((M + 31) / 32)), dim3(32, 8), 0, st>>>(A, AT, M, K);
+  TB_LAUNCH_CHECK();
+  return TB_OK;
+}
+
+tb_status split3_transpose(const double* A, __nv_bfloat16* AT, long long M, int K, cudaStream_t st) {
+  k_split3_transpose<double><<<dim3((K + 31) / 32, (unsigned)((M + 31) / 32)), dim3(32, 8), 0, st>>>(A, AT, M, K);
+  TB_LAUNCH_CHECK();
+  return TB_OK;
+}
+
+// C = A B (double result) through split bf16 pieces; AT ([3][K][M]) and Bp ([3][K][N]) are scratch.
+tb_status gemm_split_tensor(double* C, long long ldc, const float* A, const float* B, __nv_bfloat16* AT,
+                            __nv_bfloat16* Bp, long long M, int N, int K, cudaStream_t st) {
+  TB_TRY(split3(B, Bp, (long long)K * N, st));
+  TB_TRY(split3_transpose(A, AT, M, K, st));
+  return gemm_split_presplit(C, ldc, AT, Bp, M, N, K, false, st);
 }
 
 int yw_error_read_clear() {

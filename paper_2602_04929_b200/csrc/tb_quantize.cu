@@ -27,6 +27,10 @@ namespace tb {
 // tensor-core blockwise product of the scale refinement (tb_gemm_tc.cu)
 tb_status yw_tensor(float* Yw, const unsigned char* codes, const int* zeros, const float* H_in, __nv_bfloat16* WbT,
                     __nv_bfloat16* Hp, bool split_h, long long rows, int d, int seg, int ng, cudaStream_t st);
+// C (+)= A B in double from operands split into three bf16 pieces each (tb_gemm_tc.cu)
+tb_status gemm_split_presplit(double* C, long long ldc, const __nv_bfloat16* AT, const __nv_bfloat16* Bp, long long M,
+                              int N, int K, bool accumulate, cudaStream_t st);
+tb_status split3_transpose(const double* A, __nv_bfloat16* AT, long long M, int K, cudaStream_t st);
 }
 
 namespace tb {
@@ -1016,6 +1020,7 @@ struct Plan {
   float* Wb;
   __nv_bfloat16 *WbT, *Hp;  // tensor-core path of the blockwise product
   bool yw_tensor;
+  bool dm_tensor;  // (Q - W) H_in through the split-bf16 tensor-core product as well
   size_t ws_total;
 };
 
@@ -1074,7 +1079,7 @@ static tb_status make_plan(const tb_layer_desc* D, bool has_hout, bool with_r, b
   p.Dq = p.Dm = p.Yw = p.n0 = p.Amat = p.G2 = nullptr;
   p.Wb = nullptr;
   p.WbT = p.Hp = nullptr;
-  p.yw_tensor = false;
+  p.yw_tensor = p.dm_tensor = false;
   p.cd_rows = 0;
   if (p.cd || with_loss) {
     p.Dq = b.take<double>((size_t)p.d_out * dd);
@@ -1099,6 +1104,7 @@ static tb_status make_plan(const tb_layer_desc* D, bool has_hout, bool with_r, b
     if (p.yw_tensor) {
       p.WbT = b.take<__nv_bfloat16>((size_t)rows * dd);
       p.Hp = b.take<__nv_bfloat16>((size_t)3 * dd * dd);
+      p.dm_tensor = (p.d % 32 == 0);
     }
     const long long lines = has_hout ? rows / p.dh : rows;
     p.n0 = b.take<double>((size_t)lines * p.ng);
@@ -1386,6 +1392,9 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
       for (long long q0 = 0; q0 < rows; q0 += rows_per_prod) {
         const long long rr = r0 + q0;
         const float* Hh = H_in + ((units > 1) ? (rr / p.dh) * dd : 0);
+        if (p.yw_tensor)  // also splits H_in into its bf16 pieces on the first batch
+          TB_TRY(yw_tensor(reinterpret_cast<float*>(p.Yw), codes + rr * d, zeros + rr * p.ng, H_in, p.WbT, p.Hp,
+                           r0 == 0, rows, d, p.seg, p.ng, st));
         GemmP g = gemm_params();
         g.A = p.Dq + rr * d;
         g.a_m = d;
@@ -1398,7 +1407,15 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
         g.M = (int)rows_per_prod;
         g.N = d;
         g.K = d;
-        TB_TRY((gemm_launch<double, float, double, double, false, true>(g, st)));
+        if (p.dm_tensor) {
+          // the pieces of (Q - W), transposed, live in this batch's rows of the W~ buffer (free by now,
+          // and overwritten by G = H_out Dm only after the product)
+          __nv_bfloat16* DqT = reinterpret_cast<__nv_bfloat16*>(p.Wt + rr * d);
+          TB_TRY(split3_transpose(p.Dq + rr * d, DqT, rows, d, st));
+          TB_TRY(gemm_split_presplit(p.Dm + rr * d, d, DqT, p.Hp, rows, d, d, false, st));
+        } else {
+          TB_TRY((gemm_launch<double, float, double, double, false, true>(g, st)));
+        }
         if (with_r) {
           GemmP h = g;
           h.A = W + rr * d;
@@ -1406,10 +1423,7 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
           h.beta = 1.0;
           TB_TRY((gemm_launch<float, float, double, double, false, true>(h, st)));
         }
-        if (p.yw_tensor) {
-          TB_TRY(yw_tensor(reinterpret_cast<float*>(p.Yw), codes + rr * d, zeros + rr * p.ng, H_in, p.WbT, p.Hp,
-                           r0 == 0, rows, d, p.seg, p.ng, st));
-        } else {
+        if (!p.yw_tensor) {
           GemmP y = gemm_params();
           y.A = p.Wb + rr * d;
           y.a_m = d;
