@@ -13,8 +13,8 @@
 //   1. A = J H J                                        (k_reverse_in)
 //   2. right-looking blocked Cholesky, 64-column panels, two launches per panel:
 //        k_chol_panel  every CTA factors the 64 x 64 diagonal block (one thread
-//                      per row, the row in registers, left-looking) and then
-//                      solves its 128 rows of the panel against it
+//                      per row, the row in registers, right-looking) and then
+//                      solves its 64 rows of the panel against it
 //        GEMM          trailing matrix -= panel panel^T  (tiles on/below the diagonal)
 //   3. inverses of the 64 x 64 diagonal blocks, all at once (k_inv_diag64)
 //   4. L^{-1} by recursive doubling: for block size s = 64, 128, ... every pair of
@@ -55,77 +55,149 @@ __global__ void k_reverse_out(const double* __restrict__ Li, float* __restrict__
 
 // One panel step of the Cholesky factorisation, columns k0 .. k0+63 of the dp x dp matrix.
 // Every CTA factors the diagonal block itself (same arithmetic everywhere, so the same
-// result); CTA x then solves rows k0+64+128x .. +127 of the panel, X L_kk^T = A_panel.
+// result); CTA x then solves rows k0+64+64x .. +63 of the panel, X L_kk^T = A_panel.
 // A non-positive pivot is recorded in info (first one wins) and replaced by 1.
-__global__ void __launch_bounds__(128) k_chol_panel(double* __restrict__ A, int* __restrict__ info,
-                                                    int dp, int k0) {
-  __shared__ double sL[FNB][FNB + 1];
-  __shared__ double rdiag[FNB];
-  const int tid = threadIdx.x, b = blockIdx.y;
+//
+// 256 threads; thread (r, q) keeps columns 16q .. 16q+15 of row r in registers, a warp
+// shares q.  The loops over 16-column blocks are rolled (straight-line code executed once
+// is bound by instruction fetch), the 16 steps inside a block are unrolled.
+//
+// Factorisation, right-looking.  Step j: the owners publish their (final) entries of
+// column j, one barrier, then every thread forms the reciprocal pivot itself and applies
+// a[c] -= a[j] / piv * col_j[c] to its part of the row.  The published raw columns stay in
+// shared memory: the panel solve runs the same elimination on its rows (x_j = a_j / L_jj,
+// then a_c -= x_j / L_jj * col_j[c]), so neither L nor an inverse is stored in between.
+// Entries right of the diagonal go through the same updates and are never used.
+enum { PLD = 66, PQ = 16, PANEL_THREADS = 256 };  // PLD: row pitch of the staged 64 x 64 tiles (doubles)
+static constexpr size_t PANEL_SMEM = (2 * 64 * PLD + 64 + 2 * PQ * 64) * sizeof(double);
+
+__device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gsrc) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((unsigned)__cvta_generic_to_shared(smem_dst)), "l"(gsrc)
+               : "memory");
+}
+
+__global__ void __launch_bounds__(PANEL_THREADS) k_chol_panel(double* __restrict__ A, int* __restrict__ info, int dp,
+                                                              int k0, int d_fact) {
+  extern __shared__ __align__(16) unsigned char panel_raw[];
+  double* sA = reinterpret_cast<double*>(panel_raw);  // this CTA's 64 panel rows
+  double* sC = sA + 64 * PLD;                         // the diagonal block, then its raw columns: sC[j * PLD + r]
+  double* rsv = sC + 64 * PLD;                        // 1 / L_jj
+  double* sY = rsv + 64;                              // multipliers of the panel solve, [2][16][64]
+  const int tid = threadIdx.x, r = tid & 63, q = tid >> 6, b = blockIdx.y;
   double* Ab = A + (long long)b * dp * dp;
-  if (tid < FNB) {
-    // left-looking factorisation, thread r owns row r of the block
-    const int r = tid;
-    double a[FNB];
-    const double* src = Ab + (long long)(k0 + r) * dp + k0;
+  double* diag = Ab + (long long)k0 * dp + k0;
+  const long long row0 = (long long)k0 + FNB + (long long)FNB * blockIdx.x;
+  const bool has_rows = row0 < d_fact;
+  double* pan = Ab + row0 * dp + k0;
+  {
+    const int ch = tid & 31, rr0 = tid >> 5;  // 16-byte piece ch of rows rr0, rr0 + 8, ...
 #pragma unroll
-    for (int c = 0; c < FNB; ++c) a[c] = src[c];
-#pragma unroll
-    for (int j = 0; j < FNB; ++j) {
-      // t = a[r][j] - sum_{k<j} L[r][k] L[j][k]
-      double t0 = a[j], t1 = 0.0;
-#pragma unroll
-      for (int k = 0; k + 1 < j; k += 2) {
-        t0 = fma(-a[k], sL[j][k], t0);
-        t1 = fma(-a[k + 1], sL[j][k + 1], t1);
-      }
-      if (j & 1) t0 = fma(-a[j - 1], sL[j][j - 1], t0);
-      const double t = t0 + t1;
-      if (r == j) {
-        const bool bad = !(t > 0.0);
-        if (bad && blockIdx.x == 0) atomicCAS(&info[b], 0, k0 + j + 1);
-        const double dj = bad ? 1.0 : sqrt(t);
-        sL[j][j] = dj;
-        rdiag[j] = 1.0 / dj;
-        a[j] = dj;
-      }
-      asm volatile("bar.sync 1, 128;" ::: "memory");  // all 128 threads (the other 64 pass the same barriers below)
-      if (r > j) {
-        a[j] = t * rdiag[j];
-        sL[r][j] = a[j];
-      }
-      asm volatile("bar.sync 1, 128;" ::: "memory");
+    for (int i = 0; i < 8; ++i) {
+      const int rr = 8 * i + rr0;
+      cp_async_16(sC + rr * PLD + 2 * ch, diag + (long long)rr * dp + 2 * ch);
     }
-    if (blockIdx.x == 0) {
-      double* dst = Ab + (long long)(k0 + r) * dp + k0;
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    if (has_rows) {
 #pragma unroll
-      for (int c = 0; c < FNB; ++c)
-        if (c <= r) dst[c] = a[c];
+      for (int i = 0; i < 8; ++i) {
+        const int rr = 8 * i + rr0;
+        cp_async_16(sA + rr * PLD + 2 * ch, pan + (long long)rr * dp + 2 * ch);
+      }
     }
-  } else {
-#pragma unroll 1
-    for (int j = 0; j < 2 * FNB; ++j) asm volatile("bar.sync 1, 128;" ::: "memory");
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    asm volatile("cp.async.wait_group 1;" ::: "memory");
   }
-  // rows of the panel below the block
-  const long long row = (long long)k0 + FNB + (long long)blockIdx.x * 128 + tid;
-  if (row < dp) {
-    double x[FNB];
-    double* src = Ab + row * dp + k0;
+  __syncthreads();
+  double a[PQ];
 #pragma unroll
-    for (int c = 0; c < FNB; ++c) x[c] = src[c];
+  for (int i = 0; i < PQ; i += 2) {
+    const double2 v = *reinterpret_cast<const double2*>(sC + r * PLD + q * PQ + i);
+    a[i] = v.x;
+    a[i + 1] = v.y;
+  }
+  __syncthreads();  // the block has been read: its storage now takes the columns
+#pragma unroll 1
+  for (int jb = 0; jb < FNB / PQ; ++jb) {
 #pragma unroll
-    for (int j = 0; j < FNB; ++j) {
-      double t0 = x[j], t1 = 0.0;
-#pragma unroll
-      for (int k = 0; k + 1 < j; k += 2) {
-        t0 = fma(-x[k], sL[j][k], t0);
-        t1 = fma(-x[k + 1], sL[j][k + 1], t1);
+    for (int jl = 0; jl < PQ; ++jl) {
+      const int j = jb * PQ + jl;
+      if (q == jb) sC[j * PLD + r] = a[jl];
+      __syncthreads();
+      if (q < jb || (r | 31) < j) continue;  // warps wholly left of or above the pivot only keep the barriers
+      const double* col = sC + j * PLD;
+      double piv = col[j];
+      if (!(piv > 0.0)) {
+        if (tid == j + 64 * jb && blockIdx.x == 0) atomicCAS(&info[b], 0, k0 + j + 1);
+        piv = 1.0;
       }
-      if (j & 1) t0 = fma(-x[j - 1], sL[j][j - 1], t0);
-      x[j] = (t0 + t1) * rdiag[j];
-    }
+      const double mult = col[r] * __drcp_rn(piv);
+      if (q == jb) {
 #pragma unroll
-    for (int c = 0; c < FNB; ++c) src[c] = x[c];
+        for (int i = jl + 1; i < PQ; ++i) a[i] = fma(-mult, col[jb * PQ + i], a[i]);
+        const double rs = rsqrt(piv);
+        a[jl] = (r == j) ? piv * rs : a[jl] * rs;
+        if (r == j) rsv[j] = rs;
+      } else {
+#pragma unroll
+        for (int i = 0; i < PQ; ++i) a[i] = fma(-mult, col[q * PQ + i], a[i]);
+      }
+    }
+  }
+  if (blockIdx.x == 0) {
+    double* dst = diag + (long long)r * dp + q * PQ;
+#pragma unroll
+    for (int i = 0; i < PQ; ++i)
+      if (q * PQ + i <= r) dst[i] = a[i];
+  }
+  if (!has_rows) return;
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+  __syncthreads();  // panel rows staged by every thread; rsv complete
+  double x[PQ];
+#pragma unroll
+  for (int i = 0; i < PQ; i += 2) {
+    const double2 v = *reinterpret_cast<const double2*>(sA + r * PLD + q * PQ + i);
+    x[i] = v.x;
+    x[i + 1] = v.y;
+  }
+#pragma unroll 1
+  for (int jb = 0; jb < FNB / PQ; ++jb) {
+    double* yb = sY + (jb & 1) * PQ * 64;
+    if (q == jb) {
+#pragma unroll
+      for (int jl = 0; jl < PQ; ++jl) {
+        const int j = jb * PQ + jl;
+        const double rs = rsv[j];
+        const double xj = x[jl] * rs;
+        x[jl] = xj;
+        const double y = xj * rs;
+        yb[jl * 64 + r] = y;
+#pragma unroll
+        for (int i = jl + 1; i < PQ; ++i) x[i] = fma(-y, sC[j * PLD + jb * PQ + i], x[i]);
+      }
+    }
+    __syncthreads();
+    if (q > jb) {
+#pragma unroll
+      for (int jl = 0; jl < PQ; ++jl) {
+        const double y = yb[jl * 64 + r];
+        const double* col = sC + (jb * PQ + jl) * PLD + q * PQ;
+#pragma unroll
+        for (int i = 0; i < PQ; ++i) x[i] = fma(-y, col[i], x[i]);
+      }
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < PQ; i += 2)
+    *reinterpret_cast<double2*>(sA + r * PLD + q * PQ + i) = make_double2(x[i], x[i + 1]);
+  __syncthreads();
+  {
+    const int ch = tid & 31, rr0 = tid >> 5;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int rr = 8 * i + rr0;
+      *reinterpret_cast<double2*>(pan + (long long)rr * dp + 2 * ch) =
+          *reinterpret_cast<const double2*>(sA + rr * PLD + 2 * ch);
+    }
   }
 }
 
@@ -210,12 +282,14 @@ extern "C" tb_status tb_factor(const float* H, int n_batch, int d, float* U, flo
   k_reverse_in<<<dim3(eb, n_batch), 256, 0, st>>>(H, f.A, d, dp);
   TB_LAUNCH_CHECK();
 
+  static bool panel_configured[64] = {false};
+  TB_TRY(allow_smem(k_chol_panel, PANEL_SMEM, panel_configured));
   // the padding is an identity block decoupled from the rest: factor the leading part only
   const int d_fact = ((d + FNB - 1) / FNB) * FNB;
   for (int k0 = 0; k0 < d_fact; k0 += FNB) {
     const int r0 = k0 + FNB, m = d_fact - r0;
-    const int xt = (m > 0) ? (m + 127) / 128 : 1;
-    k_chol_panel<<<dim3(xt, n_batch), 128, 0, st>>>(f.A, info, dp, k0);
+    const int xt = (m > 0) ? m / FNB : 1;
+    k_chol_panel<<<dim3(xt, n_batch), PANEL_THREADS, PANEL_SMEM, st>>>(f.A, info, dp, k0, d_fact);
     TB_LAUNCH_CHECK();
     if (m <= 0) break;
     GemmP s = gemm_params();  // trailing -= panel panel^T, tiles on or below the diagonal

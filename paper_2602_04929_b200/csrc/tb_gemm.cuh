@@ -278,19 +278,41 @@ __device__ __forceinline__ void gemm_tile(const GemmP& p, int m0, int n0, int ba
   gemm_mainloop<TAcc, A_MCONTIG, B_NCONTIG>(acc, la, ca, lb, cb, k_begin, k_end, smem);
 
   const TAcc alpha = static_cast<TAcc>(p.alpha), beta = static_cast<TAcc>(p.beta);
-  const bool use_c = (p.beta != 0.0);
+  if (p.beta == 0.0) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int m = m0 + GemmAcc<TAcc>::row(i);
+      if (m >= M) continue;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int n = n0 + GemmAcc<TAcc>::col(j);
+        if (n < N) C[(long long)m * p.ldc + n] = static_cast<TC>(alpha * acc.at(i, j));
+      }
+    }
+    return;
+  }
+  // C is read and written: the old values of row i + 1 are fetched before row i is stored,
+  // so that the loads of a row go out together and their latency overlaps the stores
+  // (a load placed after a store through the same pointer type cannot be moved above it).
+  TAcc cold[2][8];
+  auto fetch_row = [&](int i, TAcc* dst) {
+    const int m = m0 + GemmAcc<TAcc>::row(i);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int n = n0 + GemmAcc<TAcc>::col(j);
+      dst[j] = (m < M && n < N) ? static_cast<TAcc>(C[(long long)m * p.ldc + n]) : TAcc(0);
+    }
+  };
+  fetch_row(0, cold[0]);
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
+    if (i + 1 < 8) fetch_row(i + 1, cold[(i + 1) & 1]);
     const int m = m0 + GemmAcc<TAcc>::row(i);
     if (m >= M) continue;
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
       const int n = n0 + GemmAcc<TAcc>::col(j);
-      if (n >= N) continue;
-      TC* c = C + (long long)m * p.ldc + n;
-      TAcc v = alpha * acc.at(i, j);
-      if (use_c) v = fma(beta, static_cast<TAcc>(*c), v);
-      *c = static_cast<TC>(v);
+      if (n < N) C[(long long)m * p.ldc + n] = static_cast<TC>(fma(beta, cold[i & 1][j], alpha * acc.at(i, j)));
     }
   }
 }
