@@ -933,6 +933,207 @@ __global__ void __launch_bounds__(CDH_THREADS, 1) k_cd_head(CdHeadP p) {
   cluster.sync();  // no CTA may exit while another can still store into its shared memory
 }
 
+// ---------------------------------------------------------------------------
+// Column-parallel form of the same pass, for up to 32 groups and at most 1024
+// columns per CTA.  The quadratic forms A[g2][g] = Wbar_g2^T H_in[g2, g] Wbar_g
+// of a row depend on the integers only, so k_cd_amat forms them for every row
+// up front, in parallel.  In the walk, thread t owns columns 2t, 2t+1 of its
+// CTA for the whole pass: the u_i of the current block of 16 rows stay in its
+// registers, the lazily corrected row of G is formed there, and one row costs
+// two block barriers, one cluster barrier and a 32-step chain run in registers
+// by warp 0 of every CTA.  What the next row needs (its row of G, Wbar, A and
+// H_out) is fetched while the current row is processed, and the next row's
+// slice of Yw is pulled into L2.
+// ---------------------------------------------------------------------------
+template <typename TY>
+__global__ void __launch_bounds__(256) k_cd_amat(const void* __restrict__ Yw_, const float* __restrict__ Wb,
+                                                 double* __restrict__ Amat, int d, int seg, int ng) {
+  extern __shared__ float amat_wb[];
+  const long long row = blockIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  for (int c = tid; c < d; c += 256) amat_wb[c] = Wb[row * d + c];
+  __syncthreads();
+  const TY* Yr = static_cast<const TY*>(Yw_) + row * ng * d;
+  double* A = Amat + row * ng * ng;
+  for (int g2 = 0; g2 < ng; ++g2)
+    for (int g = g2 + warp; g < ng; g += 8) {
+      const TY* y = Yr + (long long)g2 * d + g * seg;
+      const float* w = amat_wb + g * seg;
+      double v = 0.0;
+      for (int c = lane; c < seg; c += 32) v = fma((double)y[c], (double)w[c], v);
+      v = warp_sum(v);
+      if (lane == 0) A[g2 * ng + g] = v;
+    }
+}
+
+enum { CDC_THREADS = 512, CDC_MAXG = 32 };
+__device__ __forceinline__ double2 load_pair(const float* q) {
+  const float2 v = *reinterpret_cast<const float2*>(q);
+  return make_double2((double)v.x, (double)v.y);
+}
+__device__ __forceinline__ double2 load_pair(const double* q) { return *reinterpret_cast<const double2*>(q); }
+struct CdColP {
+  double* G;           // [heads*dh][d]   H_out Dm, rows still to come updated in place at block ends
+  double* Uacc;        // [heads*dh][d]   out: the rank-1 vectors u_i
+  const void* Yw;      // [heads*dh][ng][d], element type TY of the kernel
+  const float* Wb;     // [heads*dh][d]
+  const float* Hout;   // [heads][dh][dh]
+  const double* Amat;  // [heads*dh][ng][ng], entries g2 <= g
+  double* sD;          // [heads*dh][ng]
+  int d, seg, ng, dh;
+  int csize;           // CTAs per cluster (divides ng)
+};
+
+template <typename TY>
+__global__ void __launch_bounds__(CDC_THREADS, 1) k_cd_head_cols(CdColP p) {
+  __shared__ double part[CDC_THREADS];
+  __shared__ double Am[2][CDC_MAXG * CDC_MAXG];
+  __shared__ double num[2][CDC_MAXG];
+  __shared__ double delta[CDC_MAXG];
+  __shared__ float hs[2][CDH_BLOCK];
+  __shared__ float hd[2];
+  cg::cluster_group cluster = cg::this_cluster();
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int rank = (int)cluster.block_rank();
+  const int head = blockIdx.x / p.csize;
+  const int d = p.d, seg = p.seg, ng = p.ng, dh = p.dh;
+  const int gpc = ng / p.csize, g_lo = rank * gpc;
+  const int c_lo = g_lo * seg, c_cnt = gpc * seg;
+  const int c0 = 2 * tid;
+  const bool on = c0 < c_cnt;
+  const int col = c_lo + c0;
+  const long long row0 = (long long)head * dh;
+  const float* Ho = p.Hout + (long long)head * dh * dh;
+  const TY* Yw = static_cast<const TY*>(p.Yw);
+  const int a_cnt = ng * ng;
+  const int half = seg / 2;  // partial sums per group
+  const size_t slab_lines = ((size_t)c_cnt * sizeof(TY) + 127) / 128;
+
+  // what row 0 needs
+  double2 gn = make_double2(0.0, 0.0);
+  float2 wn = make_float2(0.0f, 0.0f);
+  double an0 = 0.0, an1 = 0.0;
+  if (on) {
+    gn = *reinterpret_cast<const double2*>(p.G + row0 * d + col);
+    wn = *reinterpret_cast<const float2*>(p.Wb + row0 * d + col);
+  }
+  if (tid < a_cnt) an0 = p.Amat[row0 * a_cnt + tid];
+  if (tid + CDC_THREADS < a_cnt) an1 = p.Amat[row0 * a_cnt + tid + CDC_THREADS];
+  // hs[.][k] multiplies ureg[k]; the vectors move down one slot per row, so slot k of row j
+  // holds u of row j - 16 + k (zero while that row lies before the block)
+  if (tid < CDH_BLOCK) hs[0][tid] = 0.0f;
+  if (tid == CDH_BLOCK) hd[0] = Ho[0];
+  __syncthreads();
+
+  double2 ureg[CDH_BLOCK];
+#pragma unroll
+  for (int i = 0; i < CDH_BLOCK; ++i) ureg[i] = make_double2(0.0, 0.0);
+#pragma unroll 1
+  for (int j = 0; j < dh; ++j) {
+    const long long row = row0 + j;
+    const int buf = j & 1;
+    double2 gv = gn;
+    const float2 w = wn;
+    if (tid < a_cnt) Am[buf][tid] = an0;
+    if (tid + CDC_THREADS < a_cnt) Am[buf][tid + CDC_THREADS] = an1;
+    // ---- fetch for row j + 1 ----
+    if (j + 1 < dh) {
+      const long long rn = row + 1;
+      if (on) {
+        gn = *reinterpret_cast<const double2*>(p.G + rn * d + col);
+        wn = *reinterpret_cast<const float2*>(p.Wb + rn * d + col);
+      }
+      if (tid < a_cnt) an0 = p.Amat[rn * a_cnt + tid];
+      if (tid + CDC_THREADS < a_cnt) an1 = p.Amat[rn * a_cnt + tid + CDC_THREADS];
+      const int blkn = ((j + 1) / CDH_BLOCK) * CDH_BLOCK;
+      if (tid < CDH_BLOCK) {
+        const int ci = j + 1 - CDH_BLOCK + tid;
+        hs[buf ^ 1][tid] = (ci >= blkn && ci <= j) ? Ho[(long long)(j + 1) * dh + ci] : 0.0f;
+      }
+      if (tid == CDH_BLOCK) hd[buf ^ 1] = Ho[(long long)(j + 1) * dh + j + 1];
+      for (size_t idx = tid; idx < slab_lines * ng; idx += CDC_THREADS) {
+        const size_t g2 = idx / slab_lines, l = idx % slab_lines;
+        const char* ptr = reinterpret_cast<const char*>(Yw + (rn * ng + (long long)g2) * d + c_lo) + l * 128;
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
+      }
+    }
+    // ---- numerators of this CTA's groups: Wbar . (G + pending rank-1 terms of the block) ----
+#pragma unroll
+    for (int i = 0; i < CDH_BLOCK; ++i) {
+      const double h = (double)hs[buf][i];
+      gv.x = fma(h, ureg[i].x, gv.x);
+      gv.y = fma(h, ureg[i].y, gv.y);
+    }
+    part[tid] = on ? fma((double)w.y, gv.y, (double)w.x * gv.x) : 0.0;
+    const double hjj = (double)hd[buf];
+    __syncthreads();
+    for (int gl = warp; gl < gpc; gl += CDC_THREADS / 32) {
+      double v = 0.0;
+      for (int k = lane; k < half; k += 32) v += part[gl * half + k];
+      v = warp_sum(v);
+      if (lane == 0)
+        for (int r = 0; r < p.csize; ++r) cluster.map_shared_rank(&num[0][0], r)[buf * CDC_MAXG + g_lo + gl] = v;
+    }
+    cluster.sync();
+    // ---- the scalar chain over the row's groups, lane g holding num[g] (every CTA runs it) ----
+    if (warp == 0) {
+      const bool in = lane < ng;
+      double nm = in ? num[buf][lane] : 0.0;
+      const double den = in ? Am[buf][lane * ng + lane] * hjj : 0.0;
+      const double rinv = (den == 0.0) ? 0.0 : 1.0 / den;
+      double mine = 0.0;
+      for (int g2 = 0; g2 < ng; ++g2) {
+        const double dl = -__shfl_sync(0xffffffffu, nm, g2) * __shfl_sync(0xffffffffu, rinv, g2);
+        if (lane == g2) mine = dl;
+        if (in && lane > g2) nm = fma(hjj * dl, Am[buf][g2 * ng + lane], nm);
+      }
+      if (in) {
+        delta[lane] = mine;
+        if (rank == 0) p.sD[row * ng + lane] += mine;
+      }
+    }
+    __syncthreads();
+    // ---- u_j on this thread's columns ----
+    double2 u = make_double2(0.0, 0.0);
+    if (on) {
+      const TY* y = Yw + row * ng * d + col;
+#pragma unroll 8
+      for (int g2 = 0; g2 < ng; ++g2) {
+        const double dl = delta[g2];
+        const double2 yv = load_pair(y + (long long)g2 * d);
+        u.x = fma(dl, yv.x, u.x);
+        u.y = fma(dl, yv.y, u.y);
+      }
+      *reinterpret_cast<double2*>(p.Uacc + row * d + col) = u;
+    }
+#pragma unroll
+    for (int i = 0; i + 1 < CDH_BLOCK; ++i) ureg[i] = ureg[i + 1];
+    ureg[CDH_BLOCK - 1] = u;
+    // ---- end of a block: fold its vectors into the rows of G still to come ----
+    if ((j + 1) % CDH_BLOCK == 0 && j + 1 < dh) {
+      const int blk0 = j + 1 - CDH_BLOCK;
+      if (on) {
+#pragma unroll 2
+        for (int jj = j + 1; jj < dh; ++jj) {
+          const float* hr = Ho + (long long)jj * dh + blk0;
+          double2 g = *reinterpret_cast<const double2*>(p.G + (row0 + jj) * d + col);
+#pragma unroll
+          for (int i = 0; i < CDH_BLOCK; ++i) {
+            const double h = (double)__ldg(hr + i);
+            g.x = fma(h, ureg[i].x, g.x);
+            g.y = fma(h, ureg[i].y, g.y);
+          }
+          *reinterpret_cast<double2*>(p.G + (row0 + jj) * d + col) = g;
+          if (jj == j + 1) gn = g;
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < CDH_BLOCK; ++i) ureg[i] = make_double2(0.0, 0.0);
+    }
+  }
+  cluster.sync();  // no CTA may exit while another can still store into its shared memory
+}
+
 // Dm += Uacc (the effect of one pass on (Q - W) H_in + W R)
 __global__ void k_axpy(double* __restrict__ y, const double* __restrict__ x, long long n) {
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n;
@@ -1106,7 +1307,7 @@ static tb_status make_plan(const tb_layer_desc* D, bool has_hout, bool with_r, b
       p.Hp = b.take<__nv_bfloat16>((size_t)3 * dd * dd);
       p.dm_tensor = (p.d % 32 == 0);
     }
-    const long long lines = has_hout ? rows / p.dh : rows;
+    const long long lines = rows;  // one set of statistics per row (the column-parallel pass keeps them all)
     p.n0 = b.take<double>((size_t)lines * p.ng);
     p.Amat = b.take<double>((size_t)lines * p.ng * p.ng);
   }
@@ -1473,6 +1674,30 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
           TB_TRY(allow_smem(k_cd_head<float>, 200 * 1024, conf_head));
         else
           TB_TRY(allow_smem(k_cd_head<double>, 200 * 1024, conf_head2));
+        // column-parallel pass where a CTA's columns fit two per thread and the chain fits a warp
+        const int c_cnt = (p.ng / csize) * p.seg;
+        const bool by_cols = (p.ng <= CDC_MAXG) && (c_cnt <= 2 * CDC_THREADS) && (p.seg % 2 == 0) && (d % 2 == 0) &&
+                             ((size_t)d * sizeof(float) <= 48 * 1024);
+        CdColP cp2;
+        cp2.G = hp.G;
+        cp2.Uacc = hp.Uacc;
+        cp2.Yw = hp.Yw;
+        cp2.Wb = hp.Wb;
+        cp2.Hout = hp.Hout;
+        cp2.Amat = p.Amat;
+        cp2.sD = hp.sD;
+        cp2.d = d;
+        cp2.seg = p.seg;
+        cp2.ng = p.ng;
+        cp2.dh = p.dh;
+        cp2.csize = csize;
+        if (by_cols) {
+          if (p.yw_tensor)
+            k_cd_amat<float><<<(unsigned)rows, 256, (size_t)d * sizeof(float), st>>>(p.Yw, hp.Wb, p.Amat, d, p.seg, p.ng);
+          else
+            k_cd_amat<double><<<(unsigned)rows, 256, (size_t)d * sizeof(float), st>>>(p.Yw, hp.Wb, p.Amat, d, p.seg, p.ng);
+          TB_LAUNCH_CHECK();
+        }
         for (int it = 0; it < p.cd_iters; ++it) {
           GemmP g = gemm_params();  // G = H_out Dm, head by head
           g.A = hp.Hout;
@@ -1493,8 +1718,8 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
           TB_TRY((gemm_launch<float, double, double, double, false, true>(g, st)));
           cudaLaunchConfig_t cfg = {};
           cfg.gridDim = dim3((unsigned)(heads_b * csize));
-          cfg.blockDim = dim3(CDH_THREADS);
-          cfg.dynamicSmemBytes = sm_head;
+          cfg.blockDim = dim3(by_cols ? CDC_THREADS : CDH_THREADS);
+          cfg.dynamicSmemBytes = by_cols ? 0 : sm_head;
           cfg.stream = st;
           cudaLaunchAttribute attr[1];
           attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -1503,7 +1728,14 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
           attr[0].val.clusterDim.z = 1;
           cfg.attrs = attr;
           cfg.numAttrs = 1;
-          TB_CUDA_CHECK(cudaLaunchKernelEx(&cfg, cd_head_kern, hp));
+          if (by_cols) {
+            if (p.yw_tensor)
+              TB_CUDA_CHECK(cudaLaunchKernelEx(&cfg, k_cd_head_cols<float>, cp2));
+            else
+              TB_CUDA_CHECK(cudaLaunchKernelEx(&cfg, k_cd_head_cols<double>, cp2));
+          } else {
+            TB_CUDA_CHECK(cudaLaunchKernelEx(&cfg, cd_head_kern, hp));
+          }
           TB_LAUNCH_CHECK();
           k_axpy<<<ew_blocks(nb_el), 256, 0, st>>>(p.Dm + r0 * d, hp.Uacc, nb_el);
           TB_LAUNCH_CHECK();
