@@ -24,14 +24,14 @@ namespace tb {
 enum {
   YT_BM = 128,
   YT_BN = 128,
-  YT_BK = 64,
-  YT_STAGES = 3,
+  YT_BK = 128,                        // a whole quantization group per product
+  YT_STAGES = 2,
   YT_BOX = 64 * 64 * 2,
-  YT_A_BYTES = 2 * YT_BOX,            // Wbar^T: 64 k x 128 rows
-  YT_B_BYTES = 3 * 2 * YT_BOX,        // three pieces of H_in: 64 k x 128 columns each
-  YT_STAGE_BYTES = YT_A_BYTES + YT_B_BYTES,
+  YT_A_BYTES = 4 * YT_BOX,            // Wbar^T: 128 k x 128 rows
+  YT_B_BYTES = 3 * 4 * YT_BOX,        // three pieces of H_in: 128 k x 128 columns each
+  YT_STAGE_OUT = 8 * 32 * 33 * 4,     // epilogue staging, one 32 x 33 float tile per warp
   YT_THREADS = 320,
-  YT_SMEM = YT_STAGES * YT_STAGE_BYTES + 1024 + 256
+  YT_SMEM = YT_B_BYTES + YT_STAGES * YT_A_BYTES + YT_STAGE_OUT + 1024 + 256
 };
 
 __device__ int g_yt_error = 0;
@@ -72,12 +72,194 @@ __global__ void k_wbar_transpose(const unsigned char* __restrict__ codes, const 
 
 __global__ void __launch_bounds__(YT_THREADS, 1)
     k_yw_tc(float* __restrict__ Yw, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-            int rows, int d, int seg, int ng, int n_tiles) {
+            int rows, int d, int seg, int ng, int n_units) {
   extern __shared__ unsigned char yt_raw[];
   const uint32_t raw = smem_u32(yt_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   unsigned char* gen_base = yt_raw + (base - raw);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(gen_base + YT_STAGES * YT_STAGE_BYTES);
+  const uint32_t sb = base;                      // H_in pieces of the unit: [3][2 k-halves][2 n-halves] boxes
+  const uint32_t sa0 = base + YT_B_BYTES;        // Wbar^T ring: [stage][2 k-halves][2 row-halves] boxes
+  float* stage = reinterpret_cast<float*>(gen_base + YT_B_BYTES + YT_STAGES * YT_A_BYTES);  // [8 warps][32][33]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(gen_base + YT_B_BYTES + YT_STAGES * YT_A_BYTES + YT_STAGE_OUT);
+  // bars[0..1] a_full, [2..3] a_empty, [4] b_full, [5] b_empty, [6..7] acc_full, [8..9] acc_empty
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 10);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const uint32_t bar0 = smem_u32(bars);
+  auto afull_bar = [&](int s) { return bar0 + 8u * s; };
+  auto aempty_bar = [&](int s) { return bar0 + 8u * (2 + s); };
+  const uint32_t bfull_bar = bar0 + 8u * 4, bempty_bar = bar0 + 8u * 5;
+  auto accf_bar = [&](int b) { return bar0 + 8u * (6 + b); };
+  auto acce_bar = [&](int b) { return bar0 + 8u * (8 + b); };
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < YT_STAGES; ++s) {
+      mbar_init(afull_bar(s), 1);
+      mbar_init(aempty_bar(s), 1);
+    }
+    mbar_init(bfull_bar, 1);
+    mbar_init(bempty_bar, 1);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(accf_bar(b), 1);
+      mbar_init(acce_bar(b), 8);
+    }
+    *abort_flag = 0;
+    mbar_fence_init();
+  }
+  if (warp == 8) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(256u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int m_tiles = (rows + YT_BM - 1) / YT_BM, n_tilesN = (d + YT_BN - 1) / YT_BN;
+  const int khalves = seg / 64;  // 1 or 2 boxes of 64 contraction steps per group
+  // unit u -> (group g, column tile nj): the unit's slice of H_in stays in shared memory while
+  // the row tiles stream through
+  if (warp == 8) {
+    if (lane == 0) {
+      uint32_t it = 0, unit_it = 0;
+      for (int u = blockIdx.x; u < n_units && !*abort_flag; u += gridDim.x, ++unit_it) {
+        const int g = u / n_tilesN, nj = u % n_tilesN;
+        const int n0 = nj * YT_BN, k00 = g * seg;
+        if (!mbar_wait(bempty_bar, (unit_it & 1u) ^ 1u, abort_flag, &g_yt_error)) break;
+        mbar_expect_tx(bfull_bar, 3u * khalves * 2u * YT_BOX);
+#pragma unroll
+        for (int pc = 0; pc < 3; ++pc)
+          for (int kh = 0; kh < khalves; ++kh)
+#pragma unroll
+            for (int j = 0; j < 2; ++j)
+              tma_load_2d(sb + ((pc * 2 + kh) * 2 + j) * YT_BOX, &map_b, n0 + 64 * j, pc * d + k00 + 64 * kh, bfull_bar);
+        bool ok = true;
+        for (int mi = 0; mi < m_tiles; ++mi, ++it) {
+          const int s = it % YT_STAGES;
+          const uint32_t ph = (it / YT_STAGES) & 1u;
+          if (!mbar_wait(aempty_bar(s), ph ^ 1u, abort_flag, &g_yt_error)) {
+            ok = false;
+            break;
+          }
+          mbar_expect_tx(afull_bar(s), khalves * 2u * YT_BOX);
+          const uint32_t sa = sa0 + s * YT_A_BYTES;
+          for (int kh = 0; kh < khalves; ++kh)
+#pragma unroll
+            for (int j = 0; j < 2; ++j)
+              tma_load_2d(sa + (kh * 2 + j) * YT_BOX, &map_a, mi * YT_BM + 64 * j, k00 + 64 * kh, afull_bar(s));
+        }
+        if (!ok) break;
+      }
+    }
+  } else if (warp == 9) {
+    if (lane == 0) {
+      const uint32_t idesc = idesc_bf16_mn(YT_BM, YT_BN);
+      uint32_t it = 0, unit_it = 0;
+      for (int u = blockIdx.x; u < n_units && !*abort_flag; u += gridDim.x, ++unit_it) {
+        if (!mbar_wait(bfull_bar, unit_it & 1u, abort_flag, &g_yt_error)) break;
+        bool ok = true;
+        for (int mi = 0; mi < m_tiles; ++mi, ++it) {
+          const int b = it & 1;
+          if (!mbar_wait(acce_bar(b), ((it >> 1) & 1u) ^ 1u, abort_flag, &g_yt_error)) {
+            ok = false;
+            break;
+          }
+          const int s = it % YT_STAGES;
+          const uint32_t ph = (it / YT_STAGES) & 1u;
+          if (!mbar_wait(afull_bar(s), ph, abort_flag, &g_yt_error)) {
+            ok = false;
+            break;
+          }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t tmem_d = tmem_base + (uint32_t)b * YT_BN;
+          const uint32_t sa = sa0 + s * YT_A_BYTES;
+          for (int kk = 0; kk < 4 * khalves; ++kk) {
+            const uint32_t koff = (uint32_t)(kk >> 2) * 2 * YT_BOX + (uint32_t)(kk & 3) * 2048;
+            const uint64_t adesc = smem_desc_mn_sw128(sa + koff);
+#pragma unroll
+            for (int pc = 0; pc < 3; ++pc) {
+              const uint64_t bdesc = smem_desc_mn_sw128(sb + pc * 4 * YT_BOX + koff);
+              umma_bf16(tmem_d, adesc, bdesc, idesc, (kk > 0 || pc > 0) ? 1u : 0u);
+            }
+          }
+          umma_commit(aempty_bar(s));
+          umma_commit(accf_bar(b));
+        }
+        if (!ok) break;
+        umma_commit(bempty_bar);  // every product of the unit has read its H_in slice
+      }
+    }
+  } else {
+    // epilogue warps 0-7: TMEM lanes 32 (w % 4) .., columns 64 (w / 4) ..; a warp turns its
+    // 32 x 32 pieces through shared memory so that every store covers one 128-byte row piece
+    const int q = warp & 3, hf = warp >> 2;
+    float* st = stage + warp * (32 * 33);
+    uint32_t it = 0;
+    for (int u = blockIdx.x; u < n_units && !*abort_flag; u += gridDim.x) {
+      const int g = u / n_tilesN, nj = u % n_tilesN;
+      bool ok = true;
+      for (int mi = 0; mi < m_tiles; ++mi, ++it) {
+        const int b = it & 1;
+        if (!mbar_wait(accf_bar(b), (it >> 1) & 1u, abort_flag, &g_yt_error)) {
+          ok = false;
+          break;
+        }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * YT_BN + hf * 64);
+        uint32_t r0[32], r1[32];
+        tmem_ld_32x32(taddr, r0);
+        tmem_ld_32x32(taddr + 32, r1);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(acce_bar(b));   // the accumulator may be overwritten
+        const long long gr0 = (long long)mi * YT_BM + q * 32;
+        const int gc0 = nj * YT_BN + hf * 64;
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) st[lane * 33 + i] = __uint_as_float(c == 0 ? r0[i] : r1[i]);
+          __syncwarp();
+          const int gc = gc0 + 32 * c + lane;
+          if (gc < d) {
+#pragma unroll 8
+            for (int r = 0; r < 32; ++r)
+              if (gr0 + r < rows) Yw[((gr0 + r) * ng + g) * (long long)d + gc] = st[r * 33 + lane];
+          }
+          __syncwarp();
+        }
+      }
+      if (!ok) break;
+    }
+  }
+
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 8) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(256u) : "memory");
+  }
+}
+
+// The same product for groups wider than 128 columns: the H_in pieces stream through the
+// ring together with Wbar^T, 64 contraction steps per stage (no slice stays resident).
+enum {
+  YS_BK = 64,
+  YS_STAGES = 3,
+  YS_A_BYTES = 2 * YT_BOX,            // Wbar^T: 64 k x 128 rows
+  YS_B_BYTES = 3 * 2 * YT_BOX,        // three pieces of H_in: 64 k x 128 columns each
+  YS_STAGE_BYTES = YS_A_BYTES + YS_B_BYTES,
+  YS_SMEM = YS_STAGES * YS_STAGE_BYTES + 1024 + 256
+};
+
+__global__ void __launch_bounds__(YT_THREADS, 1)
+    k_yw_tc_stream(float* __restrict__ Yw, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+            int rows, int d, int seg, int ng, int n_tiles) {
+  extern __shared__ unsigned char ys_raw[];
+  const uint32_t raw = smem_u32(ys_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  unsigned char* gen_base = ys_raw + (base - raw);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(gen_base + YS_STAGES * YS_STAGE_BYTES);
   // bars[0..2] full, [3..5] empty, [6..7] acc_full, [8..9] acc_empty; then tmem slot, abort flag
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 10);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -89,7 +271,7 @@ __global__ void __launch_bounds__(YT_THREADS, 1)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
-    for (int s = 0; s < YT_STAGES; ++s) {
+    for (int s = 0; s < YS_STAGES; ++s) {
       mbar_init(full_bar(s), 1);
       mbar_init(empty_bar(s), 1);
     }
@@ -110,7 +292,7 @@ __global__ void __launch_bounds__(YT_THREADS, 1)
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
 
-  const int n_stages = seg / YT_BK;                       // stages per tile
+  const int n_stages = seg / YS_BK;                       // stages per tile
   const int m_tiles = (rows + YT_BM - 1) / YT_BM, n_tilesN = (d + YT_BN - 1) / YT_BN;
   // tile t -> (group g, row tile mi, column tile nj), column tiles innermost
   auto tile_of = [&](int t, int& g, int& mi, int& nj) {
@@ -127,12 +309,12 @@ __global__ void __launch_bounds__(YT_THREADS, 1)
         tile_of(t, g, mi, nj);
         const int m0 = mi * YT_BM, n0 = nj * YT_BN, k00 = g * seg;
         for (int st = 0; st < n_stages; ++st, ++it) {
-          const int s = it % YT_STAGES;
-          const uint32_t ph = (it / YT_STAGES) & 1u;
+          const int s = it % YS_STAGES;
+          const uint32_t ph = (it / YS_STAGES) & 1u;
           if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, &g_yt_error)) break;
-          mbar_expect_tx(full_bar(s), YT_STAGE_BYTES);
-          const uint32_t sa = base + s * YT_STAGE_BYTES, sb = sa + YT_A_BYTES;
-          const int k0 = k00 + st * YT_BK;
+          mbar_expect_tx(full_bar(s), YS_STAGE_BYTES);
+          const uint32_t sa = base + s * YS_STAGE_BYTES, sb = sa + YS_A_BYTES;
+          const int k0 = k00 + st * YS_BK;
 #pragma unroll
           for (int j = 0; j < 2; ++j) tma_load_2d(sa + j * YT_BOX, &map_a, m0 + 64 * j, k0, full_bar(s));
 #pragma unroll
@@ -154,16 +336,16 @@ __global__ void __launch_bounds__(YT_THREADS, 1)
         const uint32_t tmem_d = tmem_base + (uint32_t)b * YT_BN;
         bool ok = true;
         for (int st = 0; st < n_stages; ++st, ++it) {
-          const int s = it % YT_STAGES;
-          const uint32_t ph = (it / YT_STAGES) & 1u;
+          const int s = it % YS_STAGES;
+          const uint32_t ph = (it / YS_STAGES) & 1u;
           if (!mbar_wait(full_bar(s), ph, abort_flag, &g_yt_error)) {
             ok = false;
             break;
           }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const uint32_t sa = base + s * YT_STAGE_BYTES, sb = sa + YT_A_BYTES;
+          const uint32_t sa = base + s * YS_STAGE_BYTES, sb = sa + YS_A_BYTES;
 #pragma unroll
-          for (int kk = 0; kk < YT_BK / 16; ++kk) {
+          for (int kk = 0; kk < YS_BK / 16; ++kk) {
             const uint64_t adesc = smem_desc_mn_sw128(sa + kk * 2048);
 #pragma unroll
             for (int pc = 0; pc < 3; ++pc) {
@@ -237,7 +419,9 @@ tb_status yw_tensor(float* Yw, const unsigned char* codes, const int* zeros, con
   TB_TRY(make_map_2d(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Hp, (unsigned long long)d, (unsigned long long)3 * d,
                      64, 64, CU_TENSOR_MAP_SWIZZLE_128B));
   const int m_tiles = (int)((rows + YT_BM - 1) / YT_BM), n_tilesN = (d + YT_BN - 1) / YT_BN;
-  const long long n_tiles = (long long)m_tiles * n_tilesN * ng;
+  const bool resident = (seg <= 128);  // the group's slice of H_in fits next to the Wbar^T ring
+  const long long n_tiles = resident ? (long long)n_tilesN * ng   // units: one (group, column tile) pair each
+                                     : (long long)m_tiles * n_tilesN * ng;
   if (n_tiles > 0x7fffffffll) return TB_ERR_UNSUPPORTED;
   int dev = 0, sms = 0;
   TB_CUDA_CHECK(cudaGetDevice(&dev));
@@ -246,10 +430,14 @@ tb_status yw_tensor(float* Yw, const unsigned char* codes, const int* zeros, con
   if (dev < 0 || dev >= 64) return TB_ERR_CUDA;
   if (!configured[dev]) {
     TB_CUDA_CHECK(cudaFuncSetAttribute(k_yw_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)YT_SMEM));
+    TB_CUDA_CHECK(cudaFuncSetAttribute(k_yw_tc_stream, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)YS_SMEM));
     configured[dev] = true;
   }
   const int grid = (int)(n_tiles < sms ? n_tiles : sms);
-  k_yw_tc<<<grid, YT_THREADS, YT_SMEM, st>>>(Yw, map_a, map_b, (int)rows, d, seg, ng, (int)n_tiles);
+  if (resident)
+    k_yw_tc<<<grid, YT_THREADS, YT_SMEM, st>>>(Yw, map_a, map_b, (int)rows, d, seg, ng, (int)n_tiles);
+  else
+    k_yw_tc_stream<<<grid, YT_THREADS, YS_SMEM, st>>>(Yw, map_a, map_b, (int)rows, d, seg, ng, (int)n_tiles);
   TB_LAUNCH_CHECK();
   return TB_OK;
 }

@@ -1156,31 +1156,9 @@ __global__ void k_dequant(const unsigned char* __restrict__ codes, const double*
   }
 }
 
-// loss[h] = sum_{j,i} H_out[j][i] G2[i][j],  G2 = Z dW^T  (tr(dW H_in dW^T H_out) + cross term)
-__global__ void __launch_bounds__(256) k_loss_hout(const float* __restrict__ Hout,
-                                                   const double* __restrict__ G2,
-                                                   double* __restrict__ loss, int dh) {
-  __shared__ double part[8];
-  const int h = blockIdx.x;
-  const float* Ho = Hout + (long long)h * dh * dh;
-  const double* G = G2 + (long long)h * dh * dh;
-  double acc = 0.0;
-  for (int idx = threadIdx.x; idx < dh * dh; idx += blockDim.x) {
-    const int j = idx / dh, i = idx % dh;
-    acc = fma((double)Ho[idx], G[(long long)i * dh + j], acc);
-  }
-  acc = warp_sum(acc);
-  if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = acc;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    double t = 0.0;
-    for (int i = 0; i < 8; ++i) t += part[i];
-    loss[h] = t;
-  }
-}
-
-// H_out = I: loss[h] = sum over the head's rows of <Z[r,:], dW[r,:]>, in two steps with a
-// fixed order: one partial sum per block of 32 rows, then the partial sums of a head.
+// loss[h] = sum over the head's rows of <Z[r,:], dW[r,:]> (Z already multiplied by H_out when there
+// is one: tr(H_out Z dW^T) = sum of (H_out Z) .* dW), in two steps with a fixed order: one partial
+// sum per block of 32 rows, then the partial sums of a head.
 __global__ void __launch_bounds__(256) k_loss_identity_partial(const double* __restrict__ Z,
                                                                const double* __restrict__ Dq,
                                                                double* __restrict__ partial,
@@ -1845,31 +1823,34 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
       h.beta = 1.0;
       TB_TRY((gemm_launch<float, float, double, double, false, true>(h, st)));
     }
+    // loss_h = tr(H_out,h Z_h dW_h^T) = sum over the head's entries of (H_out,h Z_h) .* dW_h: a product
+    // with d_in columns (many tiles) and an elementwise reduction, instead of a d_head x d_head product
+    // whose contraction runs over d_in on a handful of tiles.
+    const double* lhs = p.Dm;
     if (p.has_hout) {
       GemmP q = gemm_params();
-      q.A = p.Dm;  // Z
-      q.a_m = d;
+      q.A = H_out;
+      q.a_m = p.dh;
       q.a_k = 1;
-      q.a_batch = (long long)p.dh * d;
-      q.B = p.Dq;  // B(k, n) = dW[n][k]
-      q.b_k = 1;
-      q.b_n = d;
+      q.a_batch = (long long)p.dh * p.dh;
+      q.B = p.Dm;  // Z
+      q.b_k = d;
+      q.b_n = 1;
       q.b_batch = (long long)p.dh * d;
-      q.C = p.G2;
-      q.ldc = p.dh;
-      q.c_batch = (long long)p.dh * p.dh;
+      q.C = p.Wt;  // W~ is no longer needed
+      q.ldc = d;
+      q.c_batch = (long long)p.dh * d;
       q.M = p.dh;
-      q.N = p.dh;
-      q.K = d;
+      q.N = d;
+      q.K = p.dh;
       q.n_batch = p.H;
-      TB_TRY((gemm_launch<double, double, double, double, false, false>(q, st)));
-      k_loss_hout<<<p.H, 256, 0, st>>>(H_out, p.G2, loss, p.dh);
-    } else {
-      const int chunks = (p.dh + 31) / 32;
-      k_loss_identity_partial<<<dim3(chunks, p.H), 256, 0, st>>>(p.Dm, p.Dq, p.G2, p.dh, d, chunks);
-      TB_LAUNCH_CHECK();
-      k_loss_identity_final<<<p.H, 32, 0, st>>>(p.G2, loss, chunks);
+      TB_TRY((gemm_launch<float, double, double, double, false, true>(q, st)));
+      lhs = p.Wt;
     }
+    const int chunks = (p.dh + 31) / 32;
+    k_loss_identity_partial<<<dim3(chunks, p.H), 256, 0, st>>>(lhs, p.Dq, p.G2, p.dh, d, chunks);
+    TB_LAUNCH_CHECK();
+    k_loss_identity_final<<<p.H, 32, 0, st>>>(p.G2, loss, chunks);
     TB_LAUNCH_CHECK();
   }
   return TB_OK;
