@@ -120,7 +120,7 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def count_launches(cfg, proj, n_tok: int, with_loss=True) -> int:
+def count_launches(cfg, proj, n_tok: int, with_loss=True, cd_iters=1) -> int:
     """Kernel launches of one step of this library (torch's own fill / reduce kernels not counted),
     from the launch loops of the library for a shared H_in without the propagated-error term."""
     d, dh, H = proj.d_in, proj.d_head, proj.n_heads
@@ -134,18 +134,41 @@ def count_launches(cfg, proj, n_tok: int, with_loss=True) -> int:
         levels = dp_blocks.bit_length() - 1
         return 1 + blocks + (blocks - 1) + 1 + 2 * levels + 1   # reverse, panels, trailing, block inverses, doubling, reverse
 
+    d_out = proj.d_out
+    seg = cfg.quant_group or d
+    ng = d // seg
     n = 1 + 1 + 2                                       # tensor-core accumulate, mirror, finalize (2)
     if has_hout:
-        n += 3                                          # G Hsum, per-head Gram, combine
+        hout_tensor = d_out % 8 == 0 and d % 32 == 0    # G Hsum as a split-bf16 tensor-core product
+        n += (3 if hout_tensor else 1) + 2              # (two splits +) product, per-head Gram, combine
     n += factor(d) + (factor(dh) if has_hout else 0)
     n += 1 + (1 if has_hout and S > 1 else 0)           # widen, compensation matrices
     n += (S if cfg.adaptive else 1) + S                 # grid search, one sweep launch per step
     n += 2 * (S - 1) if has_hout else 0                 # residual + compensation GEMM
     if cfg.cd:
-        n += 3 + (3 if has_hout else 2)                 # prep, Dm, Yw; then G, cluster pass, refresh (or two row kernels)
+        # rows per batch: whole heads (or blocks of 128 rows) whose blockwise products fit 4 GiB
+        unit_rows = dh if has_hout else 1
+        rows = max(1, (4 << 30) // (ng * d * 8 * unit_rows)) * unit_rows
+        rows = min(rows, d_out)
+        if not has_hout and rows > 128:
+            rows = rows // 128 * 128
+        batches = -(-d_out // rows)
+        yw_tensor = seg % 64 == 0 and rows % 8 == 0 and d_out % 8 == 0 and (dh % 8 == 0 or rows == d_out)
+        dm_tensor = yw_tensor and d % 32 == 0
+        per_batch = (3 if yw_tensor else 1) - (1 if yw_tensor else 0)   # transpose + product (the split of H_in is once)
+        per_batch += 2 if dm_tensor else 1                               # (split of Q - W +) product with H_in
+        if has_hout:
+            csize = 8
+            while csize > 1 and (ng % csize or (rows // dh) * csize > 148):
+                csize //= 2
+            by_cols = ng <= 32 and (ng // csize) * seg <= 1024 and seg % 2 == 0 and d % 2 == 0 and d * 4 <= 48 * 1024
+            per_batch += (1 if by_cols else 0) + 3 * cd_iters            # row statistics; then G, cluster pass, refresh
+        else:
+            per_batch += 2 * cd_iters                                    # the two row kernels
+        n += 1 + (1 if yw_tensor else 0) + batches * per_batch           # prep, split of H_in
     n += 1                                              # dequant
     if with_loss:
-        n += 1 + (0 if cfg.cd else 1) + 2               # prep, (Z product), Z dW^T / partial sums, reduction
+        n += 1 + (0 if cfg.cd else 1) + (1 if has_hout else 0) + 2      # prep, (Z product), (H_out Z), partial sums, reduction
     return n
 
 
@@ -495,37 +518,37 @@ def main():
     syrk_tiles = sum(mi // 2 + 1 for mi in range(m_blocks))
     fl = {
         "hessian": 2.0 * 128 * 256 * n_tok * syrk_tiles,
-        "gemm": 2.0 * d_out * d * d + 2.0 * d_out * dh * d,     # G Hsum, then the per-head Grams
         "sweep": 1.0 * d_out * d * d,                             # d_in^2 flop per out-channel
         "grid": 2.0 * 16 * d_out * d * seg,
-        "cd": (4.0 * d_out * d * d + 2.0 * d_out * dh * d + 3.0 * d_out * d * (d // seg)) if cfg.cd else 0.0,
+        # Cholesky of the reversed matrix (d^3 / 3) and the triangular inverse (d^3 / 3), for H_in and per head for H_out
+        "factor": (2.0 / 3.0) * d ** 3 + ((2.0 / 3.0) * dh ** 3 * H if has_hout else 0.0),
     }
     fp64_kind = "FP64 FMA / FP64 tensor pipe, 148 SM x 64 lanes x 2 x 1.965 GHz"
     roof_all = {}
+    times = {}
     if phases.get("hessian"):
-        t = phases["hessian"] * 1e-3
+        times["hessian"] = phases["hessian"]
         roof_all["hessian"] = {"kernel": "k_syrk_tc (+ zero, mirror, finalize)", "bound": "tensor",
-                               "achieved": fl["hessian"] / t / 1e12, "peak": bf16_peak, "unit": "TFLOP/s",
-                               "peak_kind": bf16_kind}
-    if has_hout and phases.get("hout"):
-        t = phases["hout"] * 1e-3
-        roof_all["gemm"] = {"kernel": "gemm_kernel<float,float,double,double> (timed through tb_build_hout)",
-                            "bound": "alu", "achieved": fl["gemm"] / t / 1e12, "peak": FP64_ALU_PEAK_TFLOPS,
-                            "unit": "TFLOP/s", "peak_kind": fp64_kind}
-    names = {"sweep": "k_sweep_rows", "grid": "k_grid", "cd": "scale refinement (3 GEMMs + k_cd_head)"}
-    for nm in ("sweep", "grid", "cd"):
-        if q_ms.get(nm) and fl[nm]:
-            t = q_ms[nm] * 1e-3
-            roof_all[nm] = {"kernel": names[nm], "bound": "alu", "achieved": fl[nm] / t / 1e12,
+                               "achieved": fl["hessian"] / (phases["hessian"] * 1e-3) / 1e12, "peak": bf16_peak,
+                               "unit": "TFLOP/s", "peak_kind": bf16_kind}
+    names = {"sweep": "k_sweep_rows", "grid": "k_grid"}
+    for nm in ("sweep", "grid"):
+        if q_ms.get(nm):
+            times[nm] = q_ms[nm]
+            roof_all[nm] = {"kernel": names[nm], "bound": "alu", "achieved": fl[nm] / (q_ms[nm] * 1e-3) / 1e12,
                             "peak": FP64_ALU_PEAK_TFLOPS, "unit": "TFLOP/s", "peak_kind": fp64_kind}
+    if phases.get("factor"):
+        roof_all["factor"] = {"kernel": "k_chol_panel + FP64 GEMM engine (trailing updates, recursive-doubling inverse)",
+                              "bound": "alu", "achieved": fl["factor"] / (phases["factor"] * 1e-3) / 1e12,
+                              "peak": FP64_ALU_PEAK_TFLOPS, "unit": "TFLOP/s", "peak_kind": fp64_kind}
     # DRAM traffic per launch from the committed ncu captures (profiles/), bytes; None where no capture applies
     traffic = {"sweep": NCU_TRAFFIC.get((cfg.name, "k_sweep_rows")), "grid": NCU_TRAFFIC.get((cfg.name, "k_grid")),
-               "gemm": NCU_TRAFFIC.get((cfg.name, "gemm_hout")), "hessian": NCU_TRAFFIC.get((cfg.name, "k_syrk_tc"))}
+               "hessian": NCU_TRAFFIC.get((cfg.name, "k_syrk_tc"))}
     for k, v in roof_all.items():
         v["frac"] = v["achieved"] / v["peak"]
         v["traffic"] = traffic.get(k) if not args.heads and not args.tokens else None
-    # the kernel with the largest share of the step: the FP64 GEMM engine (H_out build, Dm, Yw, factor updates)
-    dominant = "gemm" if "gemm" in roof_all else "sweep"
+    # the single kernel with the largest share of the step (the Hessian product, the column sweep or the grid search)
+    dominant = max(times, key=times.get) if times else None
     roofline = dict(roof_all.get(dominant, {}))
     loop_ms = q_ms.get("grid", 0.0) + q_ms.get("sweep", 0.0) + q_ms.get("compensation", 0.0)
     loop_fl = fl["sweep"] + fl["grid"] + (1.0 * d_out * d * (dh - cfg.out_block) if has_hout else 0.0)
