@@ -25,9 +25,32 @@ struct HostPlan {
   int *info, *zeros;
   unsigned char* codes;
   double* loss;
-  void* sub;
-  size_t sub_bytes, total;
+  void* sub;    // workspace of the calls on the caller's stream
+  void* sub2;   // workspace of the H_out build and factor, which run beside the factor of H_in
+  size_t sub_bytes, sub2_bytes, total;
 };
+
+// One helper stream per device for the part of the path that runs beside the factor of H_in,
+// created on first use and kept for the life of the process.
+struct SideStream {
+  cudaStream_t stream;
+  cudaEvent_t fork, join;
+  bool ready;
+};
+
+SideStream* side_stream() {
+  static SideStream per_device[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  SideStream* s = &per_device[dev];
+  if (!s->ready) {
+    if (cudaStreamCreateWithFlags(&s->stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&s->fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&s->join, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    s->ready = true;
+  }
+  return s;
+}
 
 size_t max_sz(size_t a, size_t b) { return a > b ? a : b; }
 
@@ -51,13 +74,16 @@ HostPlan host_plan(const tb_layer_desc* D, long long n_tok, int g_heads, void* w
   h.What = b.take<float>(dout * d);
   h.loss = b.take<double>((size_t)D->n_heads);
   size_t sub = tb_factor_workspace(1, D->d_in);
-  if (g_heads > 0) {
-    sub = max_sz(sub, tb_factor_workspace(D->n_heads, D->d_head));
-    sub = max_sz(sub, tb_build_hout_workspace(g_heads, D->d_head, D->d_in));
-  }
   sub = max_sz(sub, tb_quantize_layer_workspace(D, 0, 1));
   h.sub = b.take<unsigned char>(sub);
   h.sub_bytes = sub;
+  h.sub2 = nullptr;
+  h.sub2_bytes = 0;
+  if (g_heads > 0) {
+    h.sub2_bytes = max_sz(tb_factor_workspace(D->n_heads, D->d_head),
+                          tb_build_hout_workspace(g_heads, D->d_head, D->d_in));
+    h.sub2 = b.take<unsigned char>(h.sub2_bytes);
+  }
   h.total = b.total();
   return h;
 }
@@ -107,14 +133,22 @@ extern "C" tb_status tb_quantize_from_host(const tb_layer_desc* desc, const floa
   TB_CUDA_CHECK(cudaMemsetAsync(h.Hin, 0, d * d * sizeof(float), st));
   TB_TRY(tb_accumulate_hessian(h.Hin, h.X, TB_BF16, n_tok, (int)d, stream));
   TB_TRY(tb_finalize_hessian(h.Hin, nullptr, h.Hsum, (int)d, n_tok, damp_in, stream));
-  TB_TRY(tb_factor(h.Hin, 1, (int)d, h.Uin, nullptr, h.info, h.sub, h.sub_bytes, stream));
+  SideStream* ss = nullptr;
   if (g_heads > 0) {
-    TB_TRY(tb_build_hout(h.Hout, h.G, h.Hsum, H, g_heads, dh, (int)d, damp_out, h.sub, h.sub_bytes,
-                         stream));
-    TB_TRY(tb_factor(h.Hout, H, dh, h.Uout, nullptr, h.info + 1, h.sub, h.sub_bytes, stream));
+    // H_out and its factor need the Hessian only: they run on a second stream beside the factor of
+    // H_in (a chain of small launches that leaves SMs idle), with their own part of the workspace
+    ss = side_stream();
+    if (!ss) return TB_ERR_CUDA;
+    TB_CUDA_CHECK(cudaEventRecord(ss->fork, st));
+    TB_CUDA_CHECK(cudaStreamWaitEvent(ss->stream, ss->fork, 0));
+    TB_TRY(tb_build_hout(h.Hout, h.G, h.Hsum, H, g_heads, dh, (int)d, damp_out, h.sub2, h.sub2_bytes, ss->stream));
+    TB_TRY(tb_factor(h.Hout, H, dh, h.Uout, nullptr, h.info + 1, h.sub2, h.sub2_bytes, ss->stream));
+    TB_CUDA_CHECK(cudaEventRecord(ss->join, ss->stream));
   } else {
     TB_CUDA_CHECK(cudaMemsetAsync(h.info + 1, 0, sizeof(int) * (size_t)H, st));
   }
+  TB_TRY(tb_factor(h.Hin, 1, (int)d, h.Uin, nullptr, h.info, h.sub, h.sub_bytes, stream));
+  if (ss) TB_CUDA_CHECK(cudaStreamWaitEvent(st, ss->join, 0));
   TB_TRY(tb_quantize_layer(desc, h.W, h.Hin, h.Uin, h.Hout, h.Uout, nullptr, nullptr, nullptr,
                            h.codes, h.scales, h.zeros, nullptr, W_hat_host ? h.What : nullptr,
                            loss_host ? h.loss : nullptr, nullptr, h.sub, h.sub_bytes, stream));

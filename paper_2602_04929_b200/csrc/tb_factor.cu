@@ -56,6 +56,7 @@ __global__ void k_reverse_out(const double* __restrict__ Li, float* __restrict__
 // One panel step of the Cholesky factorisation, columns k0 .. k0+63 of the dp x dp matrix.
 // Every CTA factors the diagonal block itself (same arithmetic everywhere, so the same
 // result); CTA x then solves rows k0+64+64x .. +63 of the panel, X L_kk^T = A_panel.
+// L_kk itself is stored in Ldiag[k0 / 64] (64 x 64, row-major), not in A.
 // A non-positive pivot is recorded in info (first one wins) and replaced by 1.
 //
 // 256 threads; thread (r, q) keeps columns 16q .. 16q+15 of row r in registers, a warp
@@ -76,7 +77,8 @@ __device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gsrc) {
                : "memory");
 }
 
-__global__ void __launch_bounds__(PANEL_THREADS) k_chol_panel(double* __restrict__ A, int* __restrict__ info, int dp,
+__global__ void __launch_bounds__(PANEL_THREADS) k_chol_panel(double* __restrict__ A, double* __restrict__ Ldiag,
+                                                              long long ldiag_batch, int* __restrict__ info, int dp,
                                                               int k0, int d_fact) {
   extern __shared__ __align__(16) unsigned char panel_raw[];
   double* sA = reinterpret_cast<double*>(panel_raw);  // this CTA's 64 panel rows
@@ -144,10 +146,11 @@ __global__ void __launch_bounds__(PANEL_THREADS) k_chol_panel(double* __restrict
     }
   }
   if (blockIdx.x == 0) {
-    double* dst = diag + (long long)r * dp + q * PQ;
+    // The factored block goes to its own array, never over the input: the CTAs of this launch need
+    // not run at the same time, and one that starts late must still find the unfactored block.
+    double* dst = Ldiag + (long long)b * ldiag_batch + (long long)(k0 / FNB) * FNB * FNB + r * FNB + q * PQ;
 #pragma unroll
-    for (int i = 0; i < PQ; ++i)
-      if (q * PQ + i <= r) dst[i] = a[i];
+    for (int i = 0; i < PQ; ++i) dst[i] = (q * PQ + i <= r) ? a[i] : 0.0;
   }
   if (!has_rows) return;
   asm volatile("cp.async.wait_group 0;" ::: "memory");
@@ -203,12 +206,15 @@ __global__ void __launch_bounds__(PANEL_THREADS) k_chol_panel(double* __restrict
 
 // Inverse of every 64 x 64 diagonal block of L into the same block of Li (lower triangular):
 // forward substitution, one thread per column, the column in registers.
-__global__ void __launch_bounds__(64) k_inv_diag64(const double* __restrict__ A, double* __restrict__ Li, int dp) {
+__global__ void __launch_bounds__(64) k_inv_diag64(const double* __restrict__ Ldiag, long long ldiag_batch,
+                                                   int n_factored, double* __restrict__ Li, int dp) {
   __shared__ double Ls[FNB][FNB + 1];
   __shared__ double rdiag[FNB];
   const int blk = blockIdx.x, b = blockIdx.y, c = threadIdx.x;
   const long long off = (long long)b * dp * dp + (long long)blk * FNB * (dp + 1);
-  for (int r = 0; r < FNB; ++r) Ls[r][c] = A[off + (long long)r * dp + c];
+  // blocks of the identity padding were never factored: their factor is the identity
+  const double* src = Ldiag + (long long)b * ldiag_batch + (long long)blk * FNB * FNB;
+  for (int r = 0; r < FNB; ++r) Ls[r][c] = (blk < n_factored) ? src[r * FNB + c] : (r == c ? 1.0 : 0.0);
   __syncthreads();
   rdiag[c] = 1.0 / Ls[c][c];
   __syncthreads();
@@ -237,6 +243,7 @@ __global__ void k_mask_strict_upper(const double* __restrict__ src, double* __re
 struct FactorWs {
   double *A, *Li, *tmp;
   int dp;
+  size_t tmp_per;  // doubles of tmp per matrix
   size_t total;
 };
 
@@ -253,7 +260,10 @@ static FactorWs factor_ws(int n_batch, int d, void* ws) {
   const size_t n = (size_t)f.dp * f.dp;
   f.A = b.take<double>((size_t)n_batch * n);
   f.Li = b.take<double>((size_t)n_batch * n);
-  f.tmp = b.take<double>((size_t)n_batch * n / 4 + 64);
+  // tmp: the factored diagonal blocks during the Cholesky sweep (dp x 64 per matrix), then the
+  // intermediate products of the doubling steps (dp^2 / 4 per matrix)
+  f.tmp_per = (n / 4 > (size_t)f.dp * FNB) ? n / 4 : (size_t)f.dp * FNB;
+  f.tmp = b.take<double>((size_t)n_batch * f.tmp_per + 64);
   f.total = b.total();
   return f;
 }
@@ -289,7 +299,8 @@ extern "C" tb_status tb_factor(const float* H, int n_batch, int d, float* U, flo
   for (int k0 = 0; k0 < d_fact; k0 += FNB) {
     const int r0 = k0 + FNB, m = d_fact - r0;
     const int xt = (m > 0) ? m / FNB : 1;
-    k_chol_panel<<<dim3(xt, n_batch), PANEL_THREADS, PANEL_SMEM, st>>>(f.A, info, dp, k0, d_fact);
+    k_chol_panel<<<dim3(xt, n_batch), PANEL_THREADS, PANEL_SMEM, st>>>(f.A, f.tmp, (long long)f.tmp_per, info, dp, k0,
+                                                                       d_fact);
     TB_LAUNCH_CHECK();
     if (m <= 0) break;
     GemmP s = gemm_params();  // trailing -= panel panel^T, tiles on or below the diagonal
@@ -315,7 +326,7 @@ extern "C" tb_status tb_factor(const float* H, int n_batch, int d, float* U, flo
   }
 
   // L^{-1}: diagonal blocks, then recursive doubling
-  k_inv_diag64<<<dim3(dp / FNB, n_batch), 64, 0, st>>>(f.A, f.Li, dp);
+  k_inv_diag64<<<dim3(dp / FNB, n_batch), 64, 0, st>>>(f.tmp, (long long)f.tmp_per, d_fact / FNB, f.Li, dp);
   TB_LAUNCH_CHECK();
   for (int sblk = FNB; sblk < dp; sblk <<= 1) {
     const int pairs = dp / (2 * sblk);
@@ -325,8 +336,8 @@ extern "C" tb_status tb_factor(const float* H, int n_batch, int d, float* U, flo
       const long long moff = (long long)mb * pp;
       const long long pair_stride = (pairs == 1) ? pp : (long long)2 * sblk * (dp + 1);
       const int batch = (pairs == 1) ? n_batch : pairs;
-      double* tmp = f.tmp + (long long)mb * (pp / 4);
-      const long long tmp_stride = (pairs == 1) ? (pp / 4) : (long long)sblk * sblk;
+      double* tmp = f.tmp + (long long)mb * (long long)f.tmp_per;
+      const long long tmp_stride = (pairs == 1) ? (long long)f.tmp_per : (long long)sblk * sblk;
       GemmP g = gemm_params();  // T = C A^{-1}: C = L[s:2s, 0:s], A^{-1} = Li[0:s, 0:s] (lower triangular)
       g.A = f.A + moff + (long long)sblk * dp;
       g.a_m = dp;
@@ -344,6 +355,7 @@ extern "C" tb_status tb_factor(const float* H, int n_batch, int d, float* U, flo
       g.K = sblk;
       g.n_batch = batch;
       g.btrim = 2;
+      g.flags = GEMM_HEAVY_N_FIRST;
       TB_TRY((gemm_launch<double, double, double, double, false, true>(g, st)));
       GemmP h = gemm_params();  // Li[s:2s, 0:s] = -B^{-1} T, B^{-1} = Li[s:2s, s:2s] (lower triangular)
       h.A = f.Li + moff + (long long)sblk * (dp + 1);
@@ -363,6 +375,7 @@ extern "C" tb_status tb_factor(const float* H, int n_batch, int d, float* U, flo
       h.n_batch = batch;
       h.alpha = -1.0;
       h.atrim = 1;
+      h.flags = GEMM_HEAVY_M_LAST;
       TB_TRY((gemm_launch<double, double, double, double, false, true>(h, st)));
     }
   }

@@ -20,7 +20,13 @@
 namespace tb {
 
 enum { GEMM_BM = 128, GEMM_BN = 128, GEMM_BK = 16, GEMM_THREADS = 256 };
-enum { GEMM_LOWER_TILES = 1 };  // skip tiles that lie strictly above the diagonal
+enum {
+  GEMM_LOWER_TILES = 1,  // skip tiles that lie strictly above the diagonal
+  // Launch order of the tiles when the K range depends on the tile (btrim / atrim): blocks start in
+  // linear order as SMs free up, so the tiles with the longest K range are given the lowest indices.
+  GEMM_HEAVY_N_FIRST = 2,  // K range grows as n0 falls (btrim 2): column tiles ascending, slowest index
+  GEMM_HEAVY_M_LAST = 4    // K range grows with m0 (atrim 1): row tiles descending, slowest index
+};
 
 struct GemmP {
   const void* A;
@@ -320,7 +326,18 @@ __device__ __forceinline__ void gemm_tile(const GemmP& p, int m0, int n0, int ba
 template <typename TA, typename TB, typename TC, typename TAcc, bool A_MCONTIG, bool B_NCONTIG>
 __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(GemmP p) {
   extern __shared__ __align__(16) unsigned char gemm_smem[];
-  const int m0 = blockIdx.y * GEMM_BM, n0 = blockIdx.x * GEMM_BN;
+  int tm = blockIdx.y, tn = blockIdx.x;
+  if (p.flags & (GEMM_HEAVY_N_FIRST | GEMM_HEAVY_M_LAST)) {
+    const int lin = blockIdx.y * gridDim.x + blockIdx.x, tiles_m = gridDim.y, tiles_n = gridDim.x;
+    if (p.flags & GEMM_HEAVY_N_FIRST) {
+      tn = lin / tiles_m;
+      tm = lin % tiles_m;
+    } else {
+      tm = tiles_m - 1 - lin / tiles_n;
+      tn = lin % tiles_n;
+    }
+  }
+  const int m0 = tm * GEMM_BM, n0 = tn * GEMM_BN;
   if ((p.flags & GEMM_LOWER_TILES) && n0 >= m0 + GEMM_BM) return;
   gemm_tile<TA, TB, TC, TAcc, A_MCONTIG, B_NCONTIG>(p, m0, n0, blockIdx.z, gemm_smem);
 }

@@ -120,6 +120,36 @@ def test_factor_reports_a_non_positive_pivot():
     assert info[0] == 0 and info[1] == 1 and info[2] == 1
 
 
+def test_factor_is_independent_of_other_work_on_the_gpu():
+    """The factor must not depend on how many of a launch's blocks run at the same time.
+    A second stream keeps every SM busy with unrelated work while the factor is queued
+    several times without a host synchronisation in between; every result must equal,
+    bit for bit, the one computed on an idle GPU."""
+    import torch
+    import paper_2602_04929_b200 as tb
+    d = 2048
+    g = torch.Generator(device="cuda:0").manual_seed(5)
+    X = torch.randn(2 * d, d, device="cuda:0", generator=g)
+    H = (X.T @ X / (2 * d) + 0.01 * torch.eye(d, device="cuda:0")).contiguous()
+    U0, info0 = tb.tb_factor(H)
+    torch.cuda.synchronize()
+    assert int(info0.max()) == 0
+    side = torch.cuda.Stream(device="cuda:0")
+    filler = torch.empty(32 << 20, device="cuda:0")
+    results = []
+    for _ in range(4):
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for _ in range(12):
+                filler.normal_()
+        results.append(tb.tb_factor(H))
+        torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    for U, info in results:
+        assert int(info.max()) == 0
+        assert torch.equal(U, U0)
+
+
 @pytest.mark.parametrize("n_batch,d", [(1, 256), (2, 200)])
 def test_prepare_correction(n_batch, d):
     """P = ((R U^T) masked strictly upper) U (Algorithm 2, line 2); C = R U^T U (Proposition 3.2)."""
