@@ -524,7 +524,8 @@ def main():
     fl = {
         "hessian": 2.0 * 128 * 256 * n_tok * syrk_tiles,
         "sweep": 1.0 * d_out * d * d,                             # d_in^2 flop per out-channel
-        "grid": 2.0 * 16 * d_out * d * seg,
+        # e H e^T of a symmetric H: seg (seg + 1) / 2 products and as many additions per candidate and group
+        "grid": 16.0 * d_out * d * (seg + 1),
         # Cholesky of the reversed matrix (d^3 / 3) and the triangular inverse (d^3 / 3), for H_in and per head for H_out
         "factor": (2.0 / 3.0) * d ** 3 + ((2.0 / 3.0) * dh ** 3 * H if has_hout else 0.0),
     }

@@ -249,6 +249,197 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) k_grid(GridP p) {
 }
 
 // ---------------------------------------------------------------------------
+// The same search for groups of at most 128 columns, where the whole problem of a
+// CTA (128 candidate rows x one group) fits shared memory.  H_in[G,G] is symmetric,
+// so e H e^T = 2 e T e^T with T the upper triangle of H (diagonal halved): only the
+// part k <= n of the product is formed, about half of the tensor-pipe work.  The
+// scores are compared, never output, so the factor 2 is dropped.  The candidate
+// errors are staged once (and read again for the row dots), T as float; after one
+// barrier the product runs without further synchronisation.  Column fragments
+// (8 columns) are dealt to the warps so that every warp has the same share of the
+// triangle: warp column c owns fragments c, 7-c, 8+c, 15-c.  Reads the upper
+// triangle of H_in only.
+// ---------------------------------------------------------------------------
+enum { GT_LDE = 132, GT_LDB = 136 };
+static constexpr size_t GRID_TRI_SMEM = (size_t)128 * GT_LDE * sizeof(double) + (size_t)128 * GT_LDB * sizeof(float);
+
+__global__ void __launch_bounds__(GEMM_THREADS, 1) k_grid_tri(GridP p) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  double* Es = reinterpret_cast<double*>(smem_raw);                                    // [k][candidate row]
+  float* Bs = reinterpret_cast<float*>(smem_raw + (size_t)128 * GT_LDE * sizeof(double));  // [k][n]
+  __shared__ double c_s[128], c_rs[128], c_z[128], c_J[128];
+  __shared__ long long c_row[128];  // global row of a candidate row, or -1
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int grp = blockIdx.x;
+  const int unit = blockIdx.y / p.tiles_per_unit;
+  const int tile = blockIdx.y % p.tiles_per_unit;
+  const int seg0 = grp * p.seg;
+  const int d = p.d, seg = p.seg;
+  const double maxq = (double)p.maxq;
+  const float* H = p.Hin + (long long)unit * p.d * p.d * (p.units > 1 ? 1 : 0);
+
+  // T = upper triangle of H_in[G,G], diagonal halved; issued first, it lands while phase 1 runs
+  {
+    const int n = tid & 127;
+    float hv[64];
+#pragma unroll
+    for (int i = 0; i < 64; ++i) {
+      const int k = (tid >> 7) + 2 * i;
+      hv[i] = (k <= n && n < seg) ? H[(long long)(seg0 + k) * d + seg0 + n] : 0.0f;
+    }
+#pragma unroll
+    for (int i = 0; i < 64; ++i) {
+      const int k = (tid >> 7) + 2 * i;
+      Bs[k * GT_LDB + n] = (k == n) ? 0.5f * hv[i] : hv[i];
+    }
+  }
+
+  // Phase 1: min / max of every row segment, then the candidates' (s, z).
+  for (int r = warp; r < p.rt; r += GEMM_THREADS / 32) {
+    const int rloc = tile * p.rt + r;
+    const bool valid = rloc < p.rows_per_unit;
+    long long grow = -1;
+    double mn = 0.0, mx = 0.0;
+    if (valid) {
+      grow = p.rm.row(unit * p.rows_per_unit + rloc);
+      const double* w = p.Wt + grow * p.d + seg0;
+      for (int a = lane; a < p.seg; a += 32) {
+        const double v = w[a];
+        mn = fmin(mn, v);
+        mx = fmax(mx, v);
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        mn = fmin(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+        mx = fmax(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      }
+    }
+    if (lane < p.ncp) {
+      const int k = lane, cr = r * p.ncp + k;
+      double s = 1.0, z = 0.0;
+      if (valid && k < p.n_cand) {
+        const double pk = 1.0 - (double)k / 32.0;
+        const double lo = pk * mn, hi = pk * mx;
+        if (hi != lo) {
+          s = (hi - lo) / maxq;
+          z = fmin(fmax(rne(-lo / s), 0.0), maxq);
+        }
+      }
+      c_s[cr] = s;
+      c_rs[cr] = 1.0 / s;
+      c_z[cr] = z;
+      c_row[cr] = (valid && k < p.n_cand) ? grow : -1;
+    }
+  }
+  __syncthreads();
+
+  // Phase 2: the candidates' round-to-nearest errors, Es[k][cr] (0 outside the problem)
+  {
+    const int cr = tid & 127;
+    const long long grow = c_row[cr];
+    const double s = c_s[cr], rs = c_rs[cr], z = c_z[cr];
+    const double* w = p.Wt + (grow < 0 ? 0 : grow) * d + seg0;
+#pragma unroll 8
+    for (int i = 0; i < 64; ++i) {
+      const int k = (tid >> 7) + 2 * i;
+      double e = 0.0;
+      if (grow >= 0 && k < seg) {
+        const double v = w[k];
+        const double q = fmin(fmax(rne(fma(v, rs, z)), 0.0), maxq);
+        e = v - s * (q - z);
+      }
+      Es[k * GT_LDE + cr] = e;
+    }
+  }
+  __syncthreads();
+
+  // Phase 3: acc = E T on the FP64 tensor pipe, fragments with k <= n only
+  const int wc = warp & 3, kq = lane & 3, rq = lane >> 2;
+  int fr[4];
+  fr[0] = wc;
+  fr[1] = 7 - wc;
+  fr[2] = 8 + wc;
+  fr[3] = 15 - wc;
+  double acc[8][4][2];
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j][0] = acc[i][j][1] = 0.0;
+  const double* ap = Es + kq * GT_LDE + (warp >> 2) * 64 + rq;
+  const float* bp = Bs + kq * GT_LDB + rq;
+  const int k4_end = (seg + 3) / 4;
+#pragma unroll 1
+  for (int k4 = 0; k4 < k4_end; ++k4) {
+    double a[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) a[i] = ap[k4 * 4 * GT_LDE + i * 8];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (8 * fr[j] + 7 < 4 * k4 || 8 * fr[j] >= seg) continue;  // wholly below the diagonal, or outside the group
+      const double b = (double)bp[k4 * 4 * GT_LDB + 8 * fr[j]];
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+                     : "+d"(acc[i][j][0]), "+d"(acc[i][j][1])
+                     : "d"(a[i]), "d"(b));
+    }
+  }
+
+  // Phase 4: row dots of (E T) with E.  A candidate row's score is spread over the 4 lanes of a
+  // quad and the 4 warps that share its rows; quads reduce by shuffle, warps through shared
+  // memory in a fixed order.
+  double jpart[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int cr = (warp >> 2) * 64 + i * 8 + rq;
+    double v = 0.0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int n = 8 * fr[j] + 2 * kq;
+      v = fma(acc[i][j][0], Es[n * GT_LDE + cr], v);
+      v = fma(acc[i][j][1], Es[(n + 1) * GT_LDE + cr], v);
+    }
+    jpart[i] = v;
+  }
+  __syncthreads();  // every warp is done with Bs: its storage takes the partial scores
+  double* c_Jw = reinterpret_cast<double*>(Bs);  // [4][128]
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    double v = jpart[i];
+    v += __shfl_xor_sync(0xffffffffu, v, 1);
+    v += __shfl_xor_sync(0xffffffffu, v, 2);
+    if (kq == 0) c_Jw[wc * 128 + (warp >> 2) * 64 + i * 8 + rq] = v;
+  }
+  __syncthreads();
+  if (tid < 128) c_J[tid] = ((c_Jw[tid] + c_Jw[128 + tid]) + c_Jw[256 + tid]) + c_Jw[384 + tid];
+  __syncthreads();
+
+  // Phase 5: argmin per row, strict '<' so that the lowest k wins ties.
+  if (tid < p.rt) {
+    const int r = tid;
+    const long long grow = c_row[r * p.ncp];
+    if (grow >= 0) {
+      int best = 0;
+      double bj = c_J[r * p.ncp];
+      for (int k = 1; k < p.n_cand; ++k) {
+        const double j = c_J[r * p.ncp + k];
+        if (j < bj) {
+          bj = j;
+          best = k;
+        }
+      }
+      const int cr = r * p.ncp + best;
+      const long long o = grow * p.ng + grp;
+      p.sD[o] = c_s[cr];
+      p.s_out[o] = (float)c_s[cr];
+      p.z_out[o] = (int)c_z[cr];
+      if (p.cand_out) p.cand_out[o] = (unsigned char)best;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------
 // Column sweep (Algorithm 2; Eq. 2), one launch per step.  Rows never interact
 // inside the sweep, so a CTA keeps 8 active rows for the whole sweep and no CTA
 // ever waits for another.
@@ -1355,12 +1546,16 @@ static tb_status run_grid(const Plan& p, const float* H_in, float* scales, int* 
   gp.units = (p.n_hin == 1) ? 1 : p.H;
   gp.rows_per_unit = M / gp.units;
   gp.tiles_per_unit = (gp.rows_per_unit + p.rt - 1) / p.rt;
-  static bool configured[64] = {false};
+  static bool configured[64] = {false}, configured_tri[64] = {false};
   TB_TRY(allow_smem(k_grid, GemmSmem<double>::bytes, configured));
+  TB_TRY(allow_smem(k_grid_tri, GRID_TRI_SMEM, configured_tri));
   const long long ytiles = (long long)gp.units * gp.tiles_per_unit;
   if (ytiles > 65535) return TB_ERR_UNSUPPORTED;
   dim3 grid(p.ng, (unsigned)ytiles);
-  k_grid<<<grid, GEMM_THREADS, GemmSmem<double>::bytes, st>>>(gp);
+  if (p.seg <= 128)
+    k_grid_tri<<<grid, GEMM_THREADS, GRID_TRI_SMEM, st>>>(gp);
+  else
+    k_grid<<<grid, GEMM_THREADS, GemmSmem<double>::bytes, st>>>(gp);
   TB_LAUNCH_CHECK();
   return TB_OK;
 }
