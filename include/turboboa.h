@@ -190,7 +190,9 @@ tb_status tb_prepare_correction(const float* R, const float* U_in, int n_batch, 
  *
  * Inputs
  *   W      [d_out][d_in] float
- *   H_in   [n_hin][d_in][d_in] float, symmetric
+ *   H_in   [n_hin][d_in][d_in] float, symmetric (for groups of at most 128
+ *          columns the grid search reads the upper triangle of its diagonal
+ *          blocks only)
  *   U_in   [n_hin][d_in][d_in] float, upper factor of H_in^{-1}
  *   H_out  [n_heads][d_head][d_head] float, or NULL for the identity (the GPTQ /
  *          GPTAQ row of Table 1: every row of a head is quantized at once and
