@@ -102,9 +102,16 @@ int tb_device_error_flag(void);
 
 /* R += alpha * (X - Xfp)^T X, the deviation correlation alpha (X - X~) X^T of
  * Algorithm 1 line 5 in the same un-normalised form: R[a][b] accumulates
- * alpha * sum_t (x_t[a] - xfp_t[a]) * x_t[b].  R: [d][d] float, not symmetric. */
+ * alpha * sum_t (x_t[a] - xfp_t[a]) * x_t[b].  R: [d][d] float, not symmetric.
+ * bf16 activations run on the tensor cores (same bounded waits and error word
+ * as tb_accumulate_hessian): the deviation is split into two bf16 pieces held
+ * in ws, a DEVICE workspace of tb_accumulate_cross_workspace bytes (256-byte
+ * aligned; 0 bytes and ws = NULL for float activations, which run on the FP32
+ * pipe).  X, Xfp and R must be 16-byte aligned for bf16. */
+size_t tb_accumulate_cross_workspace(tb_dtype x_type, long long n_tok, int d);
 tb_status tb_accumulate_cross(float* R, const void* X, const void* Xfp, tb_dtype x_type,
-                              long long n_tok, int d, float alpha, void* stream);
+                              long long n_tok, int d, float alpha, void* ws, size_t ws_bytes,
+                              void* stream);
 
 /* H <- H / n_total + damp * mean(diag(H / n_total)) * I ; R <- R / n_total when
  * R is not NULL.  The paper does not mention damping; damp = 0 reproduces

@@ -58,7 +58,8 @@ _SIGNATURES = {
     "tb_status_string": (ctypes.c_char_p, [_int]),
     "tb_accumulate_hessian": (_int, [_vp, _vp, _int, _ll, _int, _vp]),
     "tb_device_error_flag": (_int, []),
-    "tb_accumulate_cross": (_int, [_vp, _vp, _vp, _int, _ll, _int, _f, _vp]),
+    "tb_accumulate_cross_workspace": (_sz, [_int, _ll, _int]),
+    "tb_accumulate_cross": (_int, [_vp, _vp, _vp, _int, _ll, _int, _f, _vp, _sz, _vp]),
     "tb_finalize_hessian": (_int, [_vp, _vp, _vp, _int, _ll, _f, _vp]),
     "tb_build_hout_workspace": (_sz, [_int, _int, _int]),
     "tb_build_hout": (_int, [_vp, _vp, _vp, _int, _int, _int, _int, _f, _vp, _sz, _vp]),
@@ -157,8 +158,12 @@ def tb_accumulate_cross(R, X, Xfp, alpha: float) -> None:
     n_tok, d = X.shape
     if Xfp.dtype != X.dtype or Xfp.shape != X.shape:
         raise ValueError("X and Xfp must agree in shape and dtype")
-    _check(load().tb_accumulate_cross(_ptr(R, torch.float32), _ptr(X), _ptr(Xfp), _xtype(X), n_tok, d,
-                                      float(alpha), _stream()), "tb_accumulate_cross")
+    lib = load()
+    nbytes = lib.tb_accumulate_cross_workspace(_xtype(X), n_tok, d)
+    ws = _workspace(nbytes, X.device) if nbytes else None
+    _check(lib.tb_accumulate_cross(_ptr(R, torch.float32), _ptr(X), _ptr(Xfp), _xtype(X), n_tok, d, float(alpha),
+                                   _ptr(ws, None, True), nbytes if ws is not None else 0, _stream()),
+           "tb_accumulate_cross")
 
 
 def tb_finalize_hessian(H, R, n_total: int, damp: float, Hsum_out=None) -> None:

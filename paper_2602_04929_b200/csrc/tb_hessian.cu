@@ -9,6 +9,9 @@
 namespace tb {
 
 tb_status syrk_bf16_tensor(float* H, const __nv_bfloat16* X, long long n_tok, int d, cudaStream_t st);
+size_t cross_bf16_workspace(long long n_tok, int d);
+tb_status cross_bf16_tensor(float* R, const __nv_bfloat16* X, const __nv_bfloat16* Xfp, long long n_tok, int d,
+                            float alpha, void* ws, cudaStream_t st);
 tb_status gemm_split_tensor(double* C, long long ldc, const float* A, const float* B, __nv_bfloat16* AT,
                             __nv_bfloat16* Bp, long long M, int N, int K, cudaStream_t st);
 
@@ -208,16 +211,26 @@ extern "C" tb_status tb_accumulate_hessian(float* H, const void* X, tb_dtype x_t
   return accumulate_typed<float>(H, static_cast<const float*>(X), n_tok, d, st);
 }
 
+extern "C" size_t tb_accumulate_cross_workspace(tb_dtype x_type, long long n_tok, int d) {
+  if (x_type != TB_BF16 || n_tok <= 0 || d <= 0) return 0;
+  return cross_bf16_workspace(n_tok, d);
+}
+
 extern "C" tb_status tb_accumulate_cross(float* R, const void* X, const void* Xfp, tb_dtype x_type,
-                                         long long n_tok, int d, float alpha, void* stream) {
+                                         long long n_tok, int d, float alpha, void* ws, size_t ws_bytes,
+                                         void* stream) {
   if (!R || n_tok < 0 || d <= 0 || (d % 8)) return TB_ERR_INVALID_ARG;
   if (x_type != TB_F32 && x_type != TB_BF16) return TB_ERR_INVALID_ARG;
   if (n_tok == 0) return TB_OK;
   if (!X || !Xfp) return TB_ERR_INVALID_ARG;
   cudaStream_t st = as_stream(stream);
-  if (x_type == TB_BF16)
-    return cross_typed<__nv_bfloat16>(R, static_cast<const __nv_bfloat16*>(X),
-                                      static_cast<const __nv_bfloat16*>(Xfp), n_tok, d, alpha, st);
+  if (x_type == TB_BF16) {
+    // bf16 activations: tensor cores, the deviation in two exact bf16 pieces
+    if (!aligned(X, 16) || !aligned(Xfp, 16) || !aligned(R, 16)) return TB_ERR_INVALID_ARG;
+    if (!ws || !aligned(ws, 256) || ws_bytes < cross_bf16_workspace(n_tok, d)) return TB_ERR_WORKSPACE;
+    return cross_bf16_tensor(R, static_cast<const __nv_bfloat16*>(X), static_cast<const __nv_bfloat16*>(Xfp),
+                             n_tok, d, alpha, ws, st);
+  }
   return cross_typed<float>(R, static_cast<const float*>(X), static_cast<const float*>(Xfp), n_tok, d,
                             alpha, st);
 }

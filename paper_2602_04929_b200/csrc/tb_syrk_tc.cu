@@ -239,6 +239,7 @@ tb_status syrk_bf16_tensor(float* H, const __nv_bfloat16* X, long long n_tok, in
 namespace tb {
 int sweep_error_read_clear();  // the same word of the column-sweep kernel (tb_quantize.cu)
 int yw_error_read_clear();     // and of the tensor-core product of the scale refinement (tb_gemm_tc.cu)
+int cross_error_read_clear();  // and of the deviation correlation (tb_cross_tc.cu)
 }
 
 extern "C" int tb_device_error_flag(void) {
@@ -250,6 +251,7 @@ extern "C" int tb_device_error_flag(void) {
   }
   const int w = tb::sweep_error_read_clear();
   const int y = tb::yw_error_read_clear();
-  if (w < 0 || y < 0) return -1;
-  return (v || w || y) ? 1 : 0;
+  const int x = tb::cross_error_read_clear();
+  if (w < 0 || y < 0 || x < 0) return -1;
+  return (v || w || y || x) ? 1 : 0;
 }
