@@ -31,6 +31,8 @@ tb_status yw_tensor(float* Yw, const unsigned char* codes, const int* zeros, con
 tb_status gemm_split_presplit(double* C, long long ldc, const __nv_bfloat16* AT, const __nv_bfloat16* Bp, long long M,
                               int N, int K, bool accumulate, cudaStream_t st);
 tb_status split3_transpose(const double* A, __nv_bfloat16* AT, long long M, int K, cudaStream_t st);
+tb_status split3_transpose(const float* A, __nv_bfloat16* AT, long long M, int K, cudaStream_t st);
+tb_status split3(const float* B, __nv_bfloat16* Bp, long long n, cudaStream_t st);
 }
 
 namespace tb {
@@ -1768,7 +1770,7 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
         const float* Hh = H_in + ((units > 1) ? (rr / p.dh) * dd : 0);
         if (p.yw_tensor)  // also splits H_in into its bf16 pieces on the first batch
           TB_TRY(yw_tensor(reinterpret_cast<float*>(p.Yw), codes + rr * d, zeros + rr * p.ng, H_in, p.WbT, p.Hp,
-                           r0 == 0, rows, d, p.seg, p.ng, st));
+                           r0 == 0 || with_r, rows, d, p.seg, p.ng, st));  // with R the pieces of R replace H_in's below
         GemmP g = gemm_params();
         g.A = p.Dq + rr * d;
         g.a_m = d;
@@ -1790,7 +1792,13 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
         } else {
           TB_TRY((gemm_launch<double, float, double, double, false, true>(g, st)));
         }
-        if (with_r) {
+        if (with_r && p.dm_tensor) {
+          // Dm += W R through the same split-bf16 product; the pieces of R take the place of H_in's
+          __nv_bfloat16* WT = reinterpret_cast<__nv_bfloat16*>(p.Wt + rr * d);
+          TB_TRY(split3_transpose(W + rr * d, WT, rows, d, st));
+          TB_TRY(split3(R, p.Hp, dd, st));
+          TB_TRY(gemm_split_presplit(p.Dm + rr * d, d, WT, p.Hp, rows, d, d, true, st));
+        } else if (with_r) {
           GemmP h = g;
           h.A = W + rr * d;
           h.B = R + ((units > 1) ? (rr / p.dh) * dd : 0);
@@ -2008,13 +2016,19 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
     g.b_batch = (units > 1) ? dd : 0;
     // Z = dW H_in (+ 2 W R).  After the scale refinement without R the buffer Dm already holds
     // dW H_in for the final scales (it was kept current through the pass), so the product is skipped.
-    const bool dm_is_current = p.cd && !with_r;
+    // With R the pass keeps Dm = dW H_in + W R, so only one more W R is missing.
+    const bool dm_is_current = p.cd;
     if (!dm_is_current) TB_TRY((gemm_launch<double, float, double, double, false, true>(g, st)));
-    if (with_r) {
+    if (with_r && dm_is_current && p.dm_tensor && units == 1) {
+      __nv_bfloat16* WT = reinterpret_cast<__nv_bfloat16*>(p.Wt);  // W~ is no longer needed
+      TB_TRY(split3_transpose(W, WT, p.d_out, d, st));
+      TB_TRY(split3(R, p.Hp, dd, st));
+      TB_TRY(gemm_split_presplit(p.Dm, d, WT, p.Hp, p.d_out, d, d, true, st));
+    } else if (with_r) {
       GemmP h = g;
       h.A = W;
       h.B = R;
-      h.alpha = 2.0;
+      h.alpha = dm_is_current ? 1.0 : 2.0;
       h.beta = 1.0;
       TB_TRY((gemm_launch<float, float, double, double, false, true>(h, st)));
     }
