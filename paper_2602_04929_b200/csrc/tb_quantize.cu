@@ -1393,6 +1393,7 @@ struct Plan {
   __nv_bfloat16 *WbT, *Hp;  // tensor-core path of the blockwise product
   bool yw_tensor;
   bool dm_tensor;  // (Q - W) H_in through the split-bf16 tensor-core product as well
+  bool loss_tensor;  // the loss's own dW H_in (no scale refinement) through it too
   size_t ws_total;
 };
 
@@ -1482,6 +1483,9 @@ static tb_status make_plan(const tb_layer_desc* D, bool has_hout, bool with_r, b
     p.n0 = b.take<double>((size_t)lines * p.ng);
     p.Amat = b.take<double>((size_t)lines * p.ng * p.ng);
   }
+  // without the scale refinement the loss forms dW H_in itself: the same split-bf16 product
+  p.loss_tensor = with_loss && !p.cd && (p.n_hin == 1) && (p.d % 32 == 0) && (p.d_out % 8 == 0);
+  if (p.loss_tensor) p.Hp = b.take<__nv_bfloat16>((size_t)3 * dd * dd);
   if (with_loss) p.G2 = b.take<double>((size_t)p.H * p.dh * (has_hout ? p.dh : 1));  // Z dW^T, or partial sums
   p.ws_total = b.total();
   return TB_OK;
@@ -2018,12 +2022,20 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
     // dW H_in for the final scales (it was kept current through the pass), so the product is skipped.
     // With R the pass keeps Dm = dW H_in + W R, so only one more W R is missing.
     const bool dm_is_current = p.cd;
-    if (!dm_is_current) TB_TRY((gemm_launch<double, float, double, double, false, true>(g, st)));
-    if (with_r && dm_is_current && p.dm_tensor && units == 1) {
+    if (!dm_is_current && p.loss_tensor) {
+      __nv_bfloat16* DqT = reinterpret_cast<__nv_bfloat16*>(p.Wt);  // W~ is no longer needed
+      TB_TRY(split3_transpose(p.Dq, DqT, p.d_out, d, st));
+      TB_TRY(split3(H_in, p.Hp, dd, st));
+      TB_TRY(gemm_split_presplit(p.Dm, d, DqT, p.Hp, p.d_out, d, d, false, st));
+    } else if (!dm_is_current) {
+      TB_TRY((gemm_launch<double, float, double, double, false, true>(g, st)));
+    }
+    if (with_r && (p.loss_tensor || (dm_is_current && p.dm_tensor)) && units == 1) {
       __nv_bfloat16* WT = reinterpret_cast<__nv_bfloat16*>(p.Wt);  // W~ is no longer needed
       TB_TRY(split3_transpose(W, WT, p.d_out, d, st));
       TB_TRY(split3(R, p.Hp, dd, st));
       TB_TRY(gemm_split_presplit(p.Dm, d, WT, p.Hp, p.d_out, d, d, true, st));
+      if (!dm_is_current) TB_TRY(gemm_split_presplit(p.Dm, d, WT, p.Hp, p.d_out, d, d, true, st));  // 2 W R
     } else if (with_r) {
       GemmP h = g;
       h.A = W;
