@@ -311,8 +311,10 @@ def report_configs(args):
                 loop_ms = q["grid"] + q["sweep"] + q["compensation"]
                 seg = cfg.quant_group or proj.d_in
                 S = proj.d_head // g if Hout is not None else 1
-                fl = (1 + (R is not None)) * proj.d_out * proj.d_in ** 2 + 2.0 * 16 * proj.d_out * proj.d_in * seg * \
-                    (1 if cfg.adaptive else 1) + (2.0 * (1 + (R is not None)) * proj.d_out * proj.d_in ** 2 if (R is not None and S > 1) else 0)
+                # algorithmic FP64 work of the loop: sweep d_in^2 per row (twice with the P term), the symmetric
+                # quadratic forms of the grid search, and with R the W0 C product of every step but the last
+                fl = (1 + (R is not None)) * proj.d_out * proj.d_in ** 2 + 16.0 * proj.d_out * proj.d_in * (seg + 1) + \
+                    (2.0 * proj.d_out * proj.d_in ** 2 * (S - 1) / S if (R is not None and S > 1) else 0.0)
                 print(json.dumps({"config": name, "projection": proj.name, "shape": [proj.d_out, proj.d_in],
                                   "heads": proj.n_heads, "out_block": g, "bits": cfg.bits, "with_r": R is not None,
                                   "adaptive": cfg.adaptive, "cd": cfg.cd, "ms_per_layer": ms,
