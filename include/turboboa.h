@@ -242,10 +242,11 @@ int tb_profile_read(double* ms_by_phase, int n);
  * Every *_host pointer is host memory (pinned memory makes the copies
  * asynchronous); dev_ws is a DEVICE workspace of
  * tb_quantize_from_host_workspace bytes.  The call synchronises the stream
- * before it returns.  With G_host the H_out build and its factor run on a
- * helper stream of the library (one per device, created at the first such call
- * and kept until exit), forked from and joined back into `stream` by events, so
- * that they overlap the factor of H_in.  X_host is bf16 [n_tok][d_in]; G_host is the partner
+ * before it returns.  A helper stream of the library (one per device, created
+ * at the first call and kept until exit), forked from and joined back into
+ * `stream` by events, carries X to the device in pieces while the Hessian of
+ * the pieces that have arrived accumulates, and later runs the H_out build and
+ * its factor beside the factor of H_in.  X_host is bf16 [n_tok][d_in]; G_host is the partner
  * projection [g_heads*d_head][d_in] float or NULL (then H_out = identity).
  * Returns TB_ERR_NOT_SPD if a factorisation met a non-positive pivot. */
 size_t tb_quantize_from_host_workspace(const tb_layer_desc* desc, long long n_tok, int g_heads);

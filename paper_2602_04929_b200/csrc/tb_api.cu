@@ -32,9 +32,11 @@ struct HostPlan {
 
 // One helper stream per device for the part of the path that runs beside the factor of H_in,
 // created on first use and kept for the life of the process.
+enum { COPY_CHUNKS_MAX = 16 };
 struct SideStream {
   cudaStream_t stream;
   cudaEvent_t fork, join;
+  cudaEvent_t chunk[COPY_CHUNKS_MAX];  // one per piece of X in flight
   bool ready;
 };
 
@@ -47,6 +49,8 @@ SideStream* side_stream() {
     if (cudaStreamCreateWithFlags(&s->stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
     if (cudaEventCreateWithFlags(&s->fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
     if (cudaEventCreateWithFlags(&s->join, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    for (int i = 0; i < COPY_CHUNKS_MAX; ++i)
+      if (cudaEventCreateWithFlags(&s->chunk[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
     s->ready = true;
   }
   return s;
@@ -124,21 +128,35 @@ extern "C" tb_status tb_quantize_from_host(const tb_layer_desc* desc, const floa
   const size_t ng = desc->quant_group > 0 ? d / (size_t)desc->quant_group : 1;
   const int H = desc->n_heads, dh = desc->d_head;
 
-  TB_CUDA_CHECK(cudaMemcpyAsync(h.W, W_host, dout * d * sizeof(float), cudaMemcpyHostToDevice, st));
-  TB_CUDA_CHECK(cudaMemcpyAsync(h.X, X_host, (size_t)n_tok * d * sizeof(__nv_bfloat16),
-                                cudaMemcpyHostToDevice, st));
-  if (g_heads > 0)
-    TB_CUDA_CHECK(cudaMemcpyAsync(h.G, G_host, (size_t)g_heads * dh * d * sizeof(float),
-                                  cudaMemcpyHostToDevice, st));
+  // X is by far the largest transfer: it goes over in pieces on the helper stream while the Hessian
+  // of the pieces that have arrived accumulates on the caller's stream.  Pieces are multiples of 2048
+  // tokens, so the sums are those of a single accumulation over all tokens.
+  SideStream* ss = side_stream();
+  if (!ss) return TB_ERR_CUDA;
+  long long piece = ((n_tok + COPY_CHUNKS_MAX / 2 - 1) / (COPY_CHUNKS_MAX / 2) + 2047) / 2048 * 2048;  // about 8 pieces
+  TB_CUDA_CHECK(cudaEventRecord(ss->fork, st));  // earlier work on the caller's stream may still use the buffers
+  TB_CUDA_CHECK(cudaStreamWaitEvent(ss->stream, ss->fork, 0));
   TB_CUDA_CHECK(cudaMemsetAsync(h.Hin, 0, d * d * sizeof(float), st));
-  TB_TRY(tb_accumulate_hessian(h.Hin, h.X, TB_BF16, n_tok, (int)d, stream));
+  int n_pieces = 0;
+  for (long long t0 = 0; t0 < n_tok; t0 += piece, ++n_pieces) {
+    const long long nt = (n_tok - t0 < piece) ? (n_tok - t0) : piece;
+    const __nv_bfloat16* src = static_cast<const __nv_bfloat16*>(X_host) + (size_t)t0 * d;
+    TB_CUDA_CHECK(cudaMemcpyAsync(h.X + (size_t)t0 * d, src, (size_t)nt * d * sizeof(__nv_bfloat16),
+                                  cudaMemcpyHostToDevice, ss->stream));
+    TB_CUDA_CHECK(cudaEventRecord(ss->chunk[n_pieces], ss->stream));
+    if (n_pieces == 0) {  // the small inputs ride on the caller's stream beside the first piece
+      TB_CUDA_CHECK(cudaMemcpyAsync(h.W, W_host, dout * d * sizeof(float), cudaMemcpyHostToDevice, st));
+      if (g_heads > 0)
+        TB_CUDA_CHECK(cudaMemcpyAsync(h.G, G_host, (size_t)g_heads * dh * d * sizeof(float),
+                                      cudaMemcpyHostToDevice, st));
+    }
+    TB_CUDA_CHECK(cudaStreamWaitEvent(st, ss->chunk[n_pieces], 0));
+    TB_TRY(tb_accumulate_hessian(h.Hin, h.X + (size_t)t0 * d, TB_BF16, nt, (int)d, stream));
+  }
   TB_TRY(tb_finalize_hessian(h.Hin, nullptr, h.Hsum, (int)d, n_tok, damp_in, stream));
-  SideStream* ss = nullptr;
   if (g_heads > 0) {
-    // H_out and its factor need the Hessian only: they run on a second stream beside the factor of
+    // H_out and its factor need the Hessian only: they run on the helper stream beside the factor of
     // H_in (a chain of small launches that leaves SMs idle), with their own part of the workspace
-    ss = side_stream();
-    if (!ss) return TB_ERR_CUDA;
     TB_CUDA_CHECK(cudaEventRecord(ss->fork, st));
     TB_CUDA_CHECK(cudaStreamWaitEvent(ss->stream, ss->fork, 0));
     TB_TRY(tb_build_hout(h.Hout, h.G, h.Hsum, H, g_heads, dh, (int)d, damp_out, h.sub2, h.sub2_bytes, ss->stream));
@@ -148,7 +166,7 @@ extern "C" tb_status tb_quantize_from_host(const tb_layer_desc* desc, const floa
     TB_CUDA_CHECK(cudaMemsetAsync(h.info + 1, 0, sizeof(int) * (size_t)H, st));
   }
   TB_TRY(tb_factor(h.Hin, 1, (int)d, h.Uin, nullptr, h.info, h.sub, h.sub_bytes, stream));
-  if (ss) TB_CUDA_CHECK(cudaStreamWaitEvent(st, ss->join, 0));
+  if (g_heads > 0) TB_CUDA_CHECK(cudaStreamWaitEvent(st, ss->join, 0));
   TB_TRY(tb_quantize_layer(desc, h.W, h.Hin, h.Uin, h.Hout, h.Uout, nullptr, nullptr, nullptr,
                            h.codes, h.scales, h.zeros, nullptr, W_hat_host ? h.What : nullptr,
                            loss_host ? h.loss : nullptr, nullptr, h.sub, h.sub_bytes, stream));

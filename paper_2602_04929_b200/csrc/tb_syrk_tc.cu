@@ -164,9 +164,17 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
       int mi, nj;
       tile_of(t, mi, nj);
       const int m0 = mi * TC_BM, n0 = nj * TC_BN;
+      // The running sums start from the values already in H and are stored back at the end, so that
+      // accumulating the tokens over several calls (split at multiples of 2048 tokens) performs
+      // exactly the additions of one call over all of them.
       float run[128];
+      const int gm = m0 + row;
+      float* hrow = H + (long long)gm * d;
 #pragma unroll
-      for (int i = 0; i < 128; ++i) run[i] = 0.0f;
+      for (int i = 0; i < 128; ++i) {
+        const int gn = n0 + hf * 128 + i;
+        run[i] = (gm < d && gn < d && gn < m0 + TC_BM) ? hrow[gn] : 0.0f;
+      }
       bool ok = true;
       for (int st0 = 0; st0 < n_stages && ok; st0 += TC_CHUNK, ++chunk_it) {
         const int b = chunk_it & 1;
@@ -186,16 +194,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
         __syncwarp();
         if (lane == 0) mbar_arrive(acce_bar(b));
       }
-      if (ok) {
-        const int gm = m0 + row;
-        if (gm < d) {
-          float* hrow = H + (long long)gm * d;
+      if (ok && gm < d) {
 #pragma unroll
-          for (int i = 0; i < 128; ++i) {
-            const int gn = n0 + hf * 128 + i;
-            // column blocks strictly above the diagonal block are filled by the mirror pass
-            if (gn < d && gn < m0 + TC_BM) hrow[gn] += run[i];
-          }
+        for (int i = 0; i < 128; ++i) {
+          const int gn = n0 + hf * 128 + i;
+          // column blocks strictly above the diagonal block are filled by the mirror pass
+          if (gn < d && gn < m0 + TC_BM) hrow[gn] = run[i];
         }
       }
     }
