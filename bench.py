@@ -44,9 +44,9 @@ FP32_ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under
 # profiles/ (full-size workload, one launch each); filled in when a capture of the current kernel exists
 NCU_TRAFFIC = {
-    ("l2_7b_q", "k_sweep_rows"): 78.0e6,   # 69.4 MB read + 8.6 MB written per launch (4 launches per layer)
-    ("l2_7b_q", "k_grid"): 35.7e6,         # per launch (4 launches per layer)
-    ("l2_7b_q", "k_syrk_tc"): 6.667e9,     # one launch per layer; X itself is 2.15 GB
+    ("l2_7b_q", "k_sweep_rows"): 80.0e6,   # 69.4 MB read + 8.8-11.5 MB written per launch (4 launches per layer)
+    ("l2_7b_q", "k_grid_tri"): 35.0e6,     # read per launch (4 launches per layer); nothing written to DRAM
+    ("l2_7b_q", "k_syrk_tc"): 6.367e9,     # 6.271 GB read + 0.096 GB written, one launch per layer; X itself is 2.15 GB
 }
 
 
@@ -539,7 +539,7 @@ def main():
         roof_all["hessian"] = {"kernel": "k_syrk_tc (+ zero, mirror, finalize)", "bound": "tensor",
                                "achieved": fl["hessian"] / (phases["hessian"] * 1e-3) / 1e12, "peak": bf16_peak,
                                "unit": "TFLOP/s", "peak_kind": bf16_kind}
-    names = {"sweep": "k_sweep_rows", "grid": "k_grid"}
+    names = {"sweep": "k_sweep_rows", "grid": "k_grid_tri"}
     for nm in ("sweep", "grid"):
         if q_ms.get(nm):
             times[nm] = q_ms[nm]
@@ -551,7 +551,7 @@ def main():
                               "bound": "alu", "achieved": fl["factor"] / (phases["factor"] * 1e-3) / 1e12,
                               "peak": FP64_ALU_PEAK_TFLOPS, "unit": "TFLOP/s", "peak_kind": fp64_kind}
     # DRAM traffic per launch from the committed ncu captures (profiles/), bytes; None where no capture applies
-    traffic = {"sweep": NCU_TRAFFIC.get((cfg.name, "k_sweep_rows")), "grid": NCU_TRAFFIC.get((cfg.name, "k_grid")),
+    traffic = {"sweep": NCU_TRAFFIC.get((cfg.name, "k_sweep_rows")), "grid": NCU_TRAFFIC.get((cfg.name, "k_grid_tri")),
                "hessian": NCU_TRAFFIC.get((cfg.name, "k_syrk_tc"))}
     for k, v in roof_all.items():
         v["frac"] = v["achieved"] / v["peak"]
