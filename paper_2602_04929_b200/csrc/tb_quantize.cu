@@ -341,14 +341,20 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) k_grid_tri(GridP p) {
     const int cr = tid & 127;
     const long long grow = c_row[cr];
     const double s = c_s[cr], rs = c_rs[cr], z = c_z[cr];
+    const double magic = 6755399441055744.0;  // 1.5 * 2^52
+    const double zm = z + magic;
     const double* w = p.Wt + (grow < 0 ? 0 : grow) * d + seg0;
 #pragma unroll 8
     for (int i = 0; i < 64; ++i) {
       const int k = (tid >> 7) + 2 * i;
       double e = 0.0;
       if (grow >= 0 && k < seg) {
+        // the fused multiply-add into z + 1.5 * 2^52 rounds to nearest-even and leaves the integer in the
+        // low word (|v / s + z| < 2^31), where the clamp is two integer instructions
         const double v = w[k];
-        const double q = fmin(fmax(rne(fma(v, rs, z)), 0.0), maxq);
+        int n = __double2loint(fma(v, rs, zm));
+        n = min(max(n, 0), p.maxq);
+        const double q = __hiloint2double(0x43380000, n) - magic;
         e = v - s * (q - z);
       }
       Es[k * GT_LDE + cr] = e;
