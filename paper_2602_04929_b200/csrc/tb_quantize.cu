@@ -701,7 +701,11 @@ __global__ void __launch_bounds__(RS_THREADS, 1)
   // fragment 1 the odd ones, so that one 8-byte load feeds both.
   const int n_lo = uw * 16;
   volatile int* abort_flag = &sm.abort_flag;
-  const bool producer = (uw == 0 && lane == 0);
+  // Loading a chunk costs its issuer a few hundred cycles, and a ring slot is only free once all eight
+  // warps have released it, so a fixed issuer would hold everybody back: the duty rotates, chunk c of a
+  // block is loaded by lane 0 of update warp c mod 8.  Every warp keeps the ring position of the
+  // producer side itself (it is a function of the chunk count alone).
+  const bool lane0 = (lane == 0);
   const int u_row0 = unit * d * (p.units > 1 ? 1 : 0);
   // ring positions: `c_*` of the consumers (all update warps), `p_*` of the producer thread
   int c_slot = 0, p_slot = 0;
@@ -727,8 +731,9 @@ __global__ void __launch_bounds__(RS_THREADS, 1)
         w0[t][e] = fr_valid ? p.Wt[fr_grow * d + cn + n_lo + 2 * (2 * fk + e) + t] : 0.0;
 
     // step c: 64-row chunk c / NOP of the contraction, operand pair c % NOP
-    auto produce = [&](int c) {   // producer thread only
+    auto produce = [&](int c) {   // every lane 0 keeps count; the warp whose turn it is loads
       if (c < n_all) {
+        if ((c & 7) == uw) {
         RowSweepStage& st = sm.ring[p_slot];
         const uint32_t fb = smem_u32(&sm.full_bar[p_slot]);
         if (mbar_wait(smem_u32(&sm.empty_bar[p_slot]), p_phase ^ 1u, abort_flag, &g_sweep_error)) {
@@ -739,13 +744,14 @@ __global__ void __launch_bounds__(RS_THREADS, 1)
           tma_load_2d(smem_u32(&st.Ub[0][0]), second ? &map_p : &map_u, cn, u_row0 + kc * RS_CHUNK, fb);
           if (hist) tma_load_2d(smem_u32(&st.Eb[0][0]), second ? &map_a : &map_e, kc * RS_CHUNK, m_base, fb);
         }
+        }
         if (++p_slot == STAGES) {
           p_slot = 0;
           p_phase ^= 1u;
         }
       }
     };
-    if (producer)
+    if (lane0)
       for (int c = 0; c < STAGES - 1; ++c) produce(c);
     for (int c = 0; c < n_all; ++c) {
       if (c == n_hist) bar_all();  // the panel warps have finished block b: Es (and As) are complete
@@ -775,7 +781,7 @@ __global__ void __launch_bounds__(RS_THREADS, 1)
         c_slot = 0;
         c_phase ^= 1u;
       }
-      if (producer) produce(c + STAGES - 1);
+      if (lane0) produce(c + STAGES - 1);
     }
 #pragma unroll
     for (int t = 0; t < 2; ++t)
