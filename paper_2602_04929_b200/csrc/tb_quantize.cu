@@ -719,9 +719,11 @@ __global__ void __launch_bounds__(RS_THREADS, 1)
     const int cn = (b + 1) * 128;            // first column of the target block
     const int n_hist = 2 * b * NOP;          // steps whose left operand comes from a history (blocks < b)
     const int n_all = n_hist + 2 * NOP;      // plus the two chunks of block b itself
-    double acc[2][2][2];
+    // four accumulators per fragment, used in turn: with two there are not enough independent
+    // tensor instructions in flight to cover their latency
+    double acc[2][4][2];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) (&acc[0][0][0])[i] = 0.0;
+    for (int i = 0; i < 16; ++i) (&acc[0][0][0])[i] = 0.0;
     // the block's own weights, needed at the end: tile-column ci = 2 fk + e is column n_lo + 2 ci + t
     double w0[2][2];
 #pragma unroll
@@ -771,8 +773,8 @@ __global__ void __launch_bounds__(RS_THREADS, 1)
         for (int q = 0; q < 16; ++q) {
           const double a = ap[4 * q];
           const float2 bb = *reinterpret_cast<const float2*>(bp + 4 * q * RS_LDB);
-          mma_f64(acc[0][q & 1], a, (double)bb.x);
-          mma_f64(acc[1][q & 1], a, (double)bb.y);
+          mma_f64(acc[0][q & 3], a, (double)bb.x);
+          mma_f64(acc[1][q & 3], a, (double)bb.y);
         }
       }
       __syncwarp();
@@ -787,7 +789,8 @@ __global__ void __launch_bounds__(RS_THREADS, 1)
     for (int t = 0; t < 2; ++t)
 #pragma unroll
       for (int e = 0; e < 2; ++e)
-        sm.wblk[fr][n_lo + 2 * (2 * fk + e) + t] = w0[t][e] - (acc[t][0][e] + acc[t][1][e]);
+        sm.wblk[fr][n_lo + 2 * (2 * fk + e) + t] =
+            w0[t][e] - ((acc[t][0][e] + acc[t][1][e]) + (acc[t][2][e] + acc[t][3][e]));
     bar_all();  // block b+1 handed over
   }
 }
