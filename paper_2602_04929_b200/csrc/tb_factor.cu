@@ -268,6 +268,31 @@ static FactorWs factor_ws(int n_batch, int d, void* ws) {
   return f;
 }
 
+// Helper stream of the look-ahead (one per device, created on first use, kept until exit).
+struct FactorSide {
+  cudaStream_t stream;
+  cudaEvent_t fork, panel, trail;
+  bool ready;
+};
+
+static FactorSide* factor_side() {
+  static FactorSide per_device[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  FactorSide* s = &per_device[dev];
+  if (!s->ready) {
+    if (cudaStreamCreateWithFlags(&s->stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&s->fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&s->panel, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&s->trail, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    s->ready = true;
+  }
+  return s;
+}
+
+tb_status factor_run(const float* H, int n_batch, int d, float* U, float* Hinv, int* info, void* ws, size_t ws_bytes,
+                     void* stream, bool lookahead);
+
 }  // namespace tb
 
 using namespace tb;
@@ -279,6 +304,16 @@ extern "C" size_t tb_factor_workspace(int n_batch, int d) {
 
 extern "C" tb_status tb_factor(const float* H, int n_batch, int d, float* U, float* Hinv, int* info,
                                void* ws, size_t ws_bytes, void* stream) {
+  return factor_run(H, n_batch, d, U, Hinv, info, ws, ws_bytes, stream, true);
+}
+
+// lookahead: the trailing update of a panel is split in two.  The part that the next panel needs (its
+// 64 columns) stays on the caller's stream, followed at once by the next panel; the rest runs on a
+// helper stream beside them.  Every entry still receives its updates in the same order, so the result
+// is the same bit for bit.  Without it (callers that must not create a stream) everything runs on the
+// caller's stream.
+tb_status tb::factor_run(const float* H, int n_batch, int d, float* U, float* Hinv, int* info, void* ws,
+                         size_t ws_bytes, void* stream, bool lookahead) {
   if (!H || !U || !info || n_batch <= 0 || n_batch > 65535 || d <= 0) return TB_ERR_INVALID_ARG;
   if (!ws || !aligned(ws, 256) || ws_bytes < tb_factor_workspace(n_batch, d)) return TB_ERR_WORKSPACE;
   cudaStream_t st = as_stream(stream);
@@ -296,6 +331,14 @@ extern "C" tb_status tb_factor(const float* H, int n_batch, int d, float* U, flo
   TB_TRY(allow_smem(k_chol_panel, PANEL_SMEM, panel_configured));
   // the padding is an identity block decoupled from the rest: factor the leading part only
   const int d_fact = ((d + FNB - 1) / FNB) * FNB;
+  FactorSide* side = nullptr;
+  if (lookahead && d_fact >= 16 * FNB) {
+    side = factor_side();
+    if (!side) return TB_ERR_CUDA;
+    TB_CUDA_CHECK(cudaEventRecord(side->fork, st));
+    TB_CUDA_CHECK(cudaStreamWaitEvent(side->stream, side->fork, 0));
+  }
+  bool trail_pending = false;
   for (int k0 = 0; k0 < d_fact; k0 += FNB) {
     const int r0 = k0 + FNB, m = d_fact - r0;
     const int xt = (m > 0) ? m / FNB : 1;
@@ -322,8 +365,36 @@ extern "C" tb_status tb_factor(const float* H, int n_batch, int d, float* U, flo
     s.alpha = -1.0;
     s.beta = 1.0;
     s.flags = GEMM_LOWER_TILES;
+    if (!side) {
+      TB_TRY((gemm_launch<double, double, double, double, false, false>(s, st)));
+      continue;
+    }
+    // the rest of the trailing matrix (columns from r0 + 64 on, hence rows from r0 + 64 on): helper stream
+    if (m > FNB) {
+      TB_CUDA_CHECK(cudaEventRecord(side->panel, st));
+      TB_CUDA_CHECK(cudaStreamWaitEvent(side->stream, side->panel, 0));
+      GemmP t = s;
+      t.A = f.A + (long long)(r0 + FNB) * dp + k0;
+      t.B = t.A;
+      t.C = f.A + (long long)(r0 + FNB) * dp + (r0 + FNB);
+      t.M = m - FNB;
+      t.N = m - FNB;
+      TB_TRY((gemm_launch<double, double, double, double, false, false>(t, side->stream)));
+    }
+    // the next panel's 64 columns: caller's stream, after the helper's update of the previous panel,
+    // which touched the same entries
+    if (trail_pending) TB_CUDA_CHECK(cudaStreamWaitEvent(st, side->trail, 0));
+    if (m > FNB) {
+      TB_CUDA_CHECK(cudaEventRecord(side->trail, side->stream));
+      trail_pending = true;
+    } else {
+      trail_pending = false;
+    }
+    s.N = FNB;
+    s.flags = 0;
     TB_TRY((gemm_launch<double, double, double, double, false, false>(s, st)));
   }
+  if (side && trail_pending) TB_CUDA_CHECK(cudaStreamWaitEvent(st, side->trail, 0));
 
   // L^{-1}: diagonal blocks, then recursive doubling
   k_inv_diag64<<<dim3(dp / FNB, n_batch), 64, 0, st>>>(f.tmp, (long long)f.tmp_per, d_fact / FNB, f.Li, dp);

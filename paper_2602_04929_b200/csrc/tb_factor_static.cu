@@ -5,6 +5,10 @@
 
 namespace tb {
 
+// the factorisation itself (tb_factor.cu); lookahead = false keeps it on the caller's stream
+tb_status factor_run(const float* H, int n_batch, int d, float* U, float* Hinv, int* info, void* ws, size_t ws_bytes,
+                     void* stream, bool lookahead);
+
 // 32 MiB: enough for 64 matrices of 128 x 128 (the per-head H_out of a
 // 64-head attention layer) or one matrix of 1024 x 1024.  Each GPU on which
 // the library is loaded keeps this array until the process exits.
@@ -44,5 +48,6 @@ extern "C" tb_status tb_factor_static(const float* H, int n_batch, int d, float*
   // tb_factor clears the parts of its workspace that must start at zero (the
   // inverse factor and the info words) on the stream before it uses them, so
   // what an earlier call left in the array cannot leak into this one.
-  return tb_factor(H, n_batch, d, U, nullptr, info, scratch, tb::kStaticScratchBytes, stream);
+  // single stream: this entry point creates nothing, not even the helper stream of tb_factor's look-ahead
+  return tb::factor_run(H, n_batch, d, U, nullptr, info, scratch, tb::kStaticScratchBytes, stream, false);
 }
