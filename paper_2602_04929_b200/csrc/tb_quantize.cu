@@ -458,7 +458,9 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) k_grid_tri(GridP p) {
 // columns already quantized (the second product only with the propagated-error
 // term, WITH_P).  16 warps: warps 0-7 are the panel warps (one row each, one
 // lane per column, the 128 columns of a block strictly in order); warps 8-15
-// are the update warps (two 8-column fragments each, on the FP64 tensor pipe).
+// are the update warps (two 8-column fragments each, on the FP64 tensor pipe,
+// four accumulators per fragment in turn so that enough independent tensor
+// instructions are in flight).
 // While the panel warps walk block b, the update warps form the part of block
 // b+1's sum that needs only blocks < b: 64-row chunks of U (and P) and of the
 // histories arrive by TMA (one box each, 8 spare columns per row so that
