@@ -145,7 +145,10 @@ tb_status tb_build_hout(float* H_out, const float* G, const float* Hsum, int n_h
  * Hinv (optional, may be NULL): [n_batch][d][d] float, U^T U.
  * info (device, [n_batch] int): 0, or the 1-based index (counted in the
  * elimination order, which runs from the last row to the first) of the first
- * pivot that was not positive; U of that matrix is then meaningless. */
+ * pivot that was not positive; U of that matrix is then meaningless.
+ * For matrices of 1024 columns or more part of the work runs on a helper
+ * stream of the library (one per device, created at the first such call and
+ * kept until exit), forked from and joined back into `stream` by events. */
 size_t tb_factor_workspace(int n_batch, int d);
 tb_status tb_factor(const float* H, int n_batch, int d, float* U, float* Hinv, int* info,
                     void* ws, size_t ws_bytes, void* stream);
@@ -178,7 +181,10 @@ tb_status tb_factor_static(const float* H, int n_batch, int d, float* U, int* in
 /* Operands of the propagated-error terms from R and U_in:
  *   P = ((R U^T) masked to its strictly upper triangle) U   (Algorithm 2, line 2)
  *   C = R U^T U = R H_in^{-1}                               (Proposition 3.2)
- * All [n_batch][d][d] float.  U must have a zero strictly-lower triangle. */
+ * All [n_batch][d][d] float.  U must have a zero strictly-lower triangle.
+ * For d a multiple of 32 the three products run on the tensor cores through
+ * exact bf16 splits with double sums of 128-step runs (relative error of P and
+ * C about 1e-6, they are float outputs); otherwise in double. */
 size_t tb_prepare_correction_workspace(int n_batch, int d);
 tb_status tb_prepare_correction(const float* R, const float* U_in, int n_batch, int d, float* P,
                                 float* C, void* ws, size_t ws_bytes, void* stream);
