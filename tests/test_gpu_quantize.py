@@ -133,3 +133,52 @@ def test_llama70b_q_proj_shape_sampled_head(g):
     prob = make_problem(3, 8192, 64, 128, 8192)
     gpu = run_gpu(prob, 2, 128, g, 0)
     compare(prob, gpu, 2, 128, g, 0, heads=[37], label=f"70b-q g={g}, sampled head")
+
+
+@pytest.mark.parametrize("with_partner,n_tok", [(True, 5000), (False, 2048)])
+def test_host_entry_point_matches_the_device_path(with_partner, n_tok):
+    """tb_quantize_from_host chains the same calls (X crosses in pieces, H_out and its factor on
+    the helper stream): its outputs must equal, bit for bit, those of the separate calls on
+    device-resident inputs."""
+    import torch
+    import paper_2602_04929_b200 as tb
+    d, H, dh = 256, 4, 64
+    W_h = tb_inputs.weight(11, H * dh, d)
+    G_h = tb_inputs.weight(11, H * dh, d, tid=tb_inputs.T_WPARTNER) if with_partner else None
+    X_h = tb_inputs.HeavyTailRecipe(d, seed=11).chunk(0, n_tok)
+    Xb = torch.from_numpy(X_h).to(torch.bfloat16)
+    desc = tb.layer_desc(H * dh, d, H, dh, 3, 64, 16 if with_partner else dh, flags=3)
+    dev = torch.device("cuda:0")
+    # separate calls
+    X = Xb.to(dev)
+    W = torch.from_numpy(W_h).to(dev)
+    Hin = torch.zeros((d, d), dtype=torch.float32, device=dev)
+    Hsum = torch.empty_like(Hin)
+    tb.tb_accumulate_hessian(Hin, X)
+    tb.tb_finalize_hessian(Hin, None, n_tok, 0.01, Hsum_out=Hsum)
+    Uin, info = tb.tb_factor(Hin)
+    Hout = Uout = None
+    if with_partner:
+        Hout = tb.tb_build_hout(torch.from_numpy(G_h).to(dev), Hsum, H, dh, 0.01)
+        Uout, info_out = tb.tb_factor(Hout)
+    res = tb.tb_quantize_layer(desc, W, Hin, Uin, Hout, Uout, want_loss=True)
+    torch.cuda.synchronize()
+    # one call from pinned host buffers
+    ng = desc.n_groups
+    outs = {"codes": torch.empty((H * dh, d), dtype=torch.uint8).pin_memory(),
+            "scales": torch.empty((H * dh, ng), dtype=torch.float32).pin_memory(),
+            "zeros": torch.empty((H * dh, ng), dtype=torch.int32).pin_memory(),
+            "w_hat": torch.empty((H * dh, d), dtype=torch.float32).pin_memory(),
+            "loss": torch.empty(H, dtype=torch.float64).pin_memory()}
+    ws = torch.empty(tb.tb_quantize_from_host_workspace(desc, n_tok, H if with_partner else 0), dtype=torch.uint8,
+                     device=dev)
+    Gp = torch.from_numpy(G_h).pin_memory() if with_partner else None
+    for _ in range(2):  # the second call reuses the helper stream and the workspace
+        tb.tb_quantize_from_host(desc, torch.from_numpy(W_h).pin_memory(), Xb.view(torch.int16).pin_memory(), Gp, 0.01,
+                                 0.01, outs, ws)
+        assert tb.tb_device_error_flag() == 0
+        assert torch.equal(outs["codes"], res.codes.cpu())
+        assert torch.equal(outs["zeros"], res.zeros.cpu())
+        assert torch.equal(outs["scales"], res.scales.cpu())
+        assert torch.equal(outs["w_hat"], res.w_hat.cpu())
+        assert torch.equal(outs["loss"], res.loss.cpu())
