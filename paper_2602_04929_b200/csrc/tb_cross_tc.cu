@@ -16,7 +16,7 @@
 // Operand layout, pipeline, warp roles and the bounded waits are those of
 // tb_syrk_tc.cu (TMA boxes of 64 tokens x 64 columns with the 128-byte swizzle =
 // MN-major SWIZZLE_128B operands; warps 0-7 epilogue, warp 8 TMA producer, warp 9
-// MMA issuer).  No cluster launch, no multicast.
+// MMA issuer).  No cluster launch; every CTA issues its own loads.
 #include "tb_common.cuh"
 #include "tb_tma.cuh"
 

@@ -1,5 +1,5 @@
 // mbarrier / TMA helpers shared by the kernels that stage operands with
-// cp.async.bulk.tensor (no cluster multicast anywhere: every CTA issues its own loads).
+// cp.async.bulk.tensor (every CTA issues its own loads; no load is shared across CTAs of a cluster).
 #pragma once
 
 #include <cuda.h>
