@@ -1229,6 +1229,7 @@ __global__ void __launch_bounds__(CDC_THREADS, 1) k_cd_head_cols(CdColP p) {
   }
   if (tid < a_cnt) an0 = p.Amat[row0 * a_cnt + tid];
   if (tid + CDC_THREADS < a_cnt) an1 = p.Amat[row0 * a_cnt + tid + CDC_THREADS];
+  double sdn = (rank == 0 && tid < ng) ? p.sD[row0 * ng + tid] : 0.0;  // the row's scales, fetched one row ahead
   // hs[.][k] multiplies ureg[k]; the vectors move down one slot per row, so slot k of row j
   // holds u of row j - 16 + k (zero while that row lies before the block)
   if (tid < CDH_BLOCK) hs[0][tid] = 0.0f;
@@ -1244,6 +1245,7 @@ __global__ void __launch_bounds__(CDC_THREADS, 1) k_cd_head_cols(CdColP p) {
     const int buf = j & 1;
     double2 gv = gn;
     const float2 w = wn;
+    const double sd_cur = sdn;
     if (tid < a_cnt) Am[buf][tid] = an0;
     if (tid + CDC_THREADS < a_cnt) Am[buf][tid + CDC_THREADS] = an1;
     // ---- fetch for row j + 1 ----
@@ -1255,6 +1257,7 @@ __global__ void __launch_bounds__(CDC_THREADS, 1) k_cd_head_cols(CdColP p) {
       }
       if (tid < a_cnt) an0 = p.Amat[rn * a_cnt + tid];
       if (tid + CDC_THREADS < a_cnt) an1 = p.Amat[rn * a_cnt + tid + CDC_THREADS];
+      if (rank == 0 && tid < ng) sdn = p.sD[rn * ng + tid];
       const int blkn = ((j + 1) / CDH_BLOCK) * CDH_BLOCK;
       if (tid < CDH_BLOCK) {
         const int ci = j + 1 - CDH_BLOCK + tid;
@@ -1287,19 +1290,25 @@ __global__ void __launch_bounds__(CDC_THREADS, 1) k_cd_head_cols(CdColP p) {
     cluster.sync();
     // ---- the scalar chain over the row's groups, lane g holding num[g] (every CTA runs it) ----
     if (warp == 0) {
+      // delta_g2 = -num[g2] / (A[g2][g2] hjj); num[g] += hjj delta_g2 A[g2][g] for g > g2.  Only num is
+      // carried from step to step: the factor -A[g2][g] / A[g2][g2] of lane g is formed beside the
+      // chain, which is then one shuffle and one multiply-add per step.
       const bool in = lane < ng;
       double nm = in ? num[buf][lane] : 0.0;
       const double den = in ? Am[buf][lane * ng + lane] * hjj : 0.0;
-      const double rinv = (den == 0.0) ? 0.0 : 1.0 / den;
+      const double rinv = (den == 0.0) ? 0.0 : 1.0 / den;   // 1 / (A[g][g] hjj)
+      const double ratio = -hjj * rinv;                     // -1 / A[g][g], or 0 for a skipped coordinate
       double mine = 0.0;
+#pragma unroll 4
       for (int g2 = 0; g2 < ng; ++g2) {
-        const double dl = -__shfl_sync(0xffffffffu, nm, g2) * __shfl_sync(0xffffffffu, rinv, g2);
-        if (lane == g2) mine = dl;
-        if (in && lane > g2) nm = fma(hjj * dl, Am[buf][g2 * ng + lane], nm);
+        const double k = __shfl_sync(0xffffffffu, ratio, g2) * ((in && lane > g2) ? Am[buf][g2 * ng + lane] : 0.0);
+        const double n2 = __shfl_sync(0xffffffffu, nm, g2);
+        if (lane == g2) mine = -n2 * rinv;
+        nm = fma(n2, k, nm);
       }
       if (in) {
         delta[lane] = mine;
-        if (rank == 0) p.sD[row * ng + lane] += mine;
+        if (rank == 0) p.sD[row * ng + lane] = sd_cur + mine;
       }
     }
     __syncthreads();
