@@ -273,8 +273,31 @@ def report_configs(args):
             cache[tag] = (H, Hsum, U, R, P, C)
             return cache[tag]
 
+        def hessian_per_head(n_heads):
+            """Value projection (Table 1): one H_in per head from X-bar_h = A_h X with the synthetic causal
+            decay of tb_inputs; no propagated-error term on this projection (there is no X-bar of the
+            full-precision path in the recipe)."""
+            if "v" in cache:
+                return cache["v"]
+            rec = tb_inputs.HeavyTailRecipe(d, seed=0)
+            Xh = rec.chunk(0, n_tok)
+            Hs = torch.empty((n_heads, d, d), dtype=torch.float32, device=dev)
+            for h in range(n_heads):
+                Xb = torch.from_numpy(tb_inputs.causal_decay_mix(Xh, tb_inputs.decay_rate(h), 2048)).to(dev).to(torch.bfloat16)
+                Hs[h].zero_()
+                tb.tb_accumulate_hessian(Hs[h], Xb)
+                tb.tb_finalize_hessian(Hs[h], None, n_tok, cfg.damp)
+            Us, info = tb.tb_factor(Hs)
+            assert int(info.max().item()) == 0
+            cache["v"] = (Hs, None, Us, None, None, None)
+            return cache["v"]
+
         for proj in cfg.projections:
-            H, Hsum, U, R, P, C = hessian("o" if proj.name == "o" else "attn", cfg.with_r)
+            per_head = proj.name == "v" and name != "tiny"
+            if per_head:
+                H, Hsum, U, R, P, C = hessian_per_head(proj.n_heads)
+            else:
+                H, Hsum, U, R, P, C = hessian("o" if proj.name == "o" else "attn", cfg.with_r)
             W = torch.from_numpy(tb_inputs.weight(0, proj.d_out, proj.d_in, tid=tb_inputs.T_W + (hash(proj.name) % 3))).to(dev)
             Hout = Uout = None
             if name == "tiny":
@@ -293,7 +316,8 @@ def report_configs(args):
             for g in blocks:
                 flags = (FLAGS_ADAPT if cfg.adaptive else 0) | (FLAGS_CD if cfg.cd else 0)
                 desc = tb.layer_desc(proj.d_out, proj.d_in, proj.n_heads, proj.d_head, cfg.bits, cfg.quant_group,
-                                     g if Hout is not None else proj.d_head, flags=flags)
+                                     g if Hout is not None else proj.d_head, n_hin=proj.n_heads if per_head else 1,
+                                     flags=flags)
                 ws = torch.empty(tb.tb_quantize_layer_workspace(desc, R is not None, True), dtype=torch.uint8, device=dev)
                 res = None
                 for rep in range(3):
@@ -316,7 +340,8 @@ def report_configs(args):
                 fl = (1 + (R is not None)) * proj.d_out * proj.d_in ** 2 + 16.0 * proj.d_out * proj.d_in * (seg + 1) + \
                     (2.0 * proj.d_out * proj.d_in ** 2 * (S - 1) / S if (R is not None and S > 1) else 0.0)
                 print(json.dumps({"config": name, "projection": proj.name, "shape": [proj.d_out, proj.d_in],
-                                  "heads": proj.n_heads, "out_block": g, "bits": cfg.bits, "with_r": R is not None,
+                                  "heads": proj.n_heads, "n_hin": proj.n_heads if per_head else 1, "out_block": g, "bits": cfg.bits,
+                                  "with_r": R is not None,
                                   "adaptive": cfg.adaptive, "cd": cfg.cd, "ms_per_layer": ms,
                                   "out_channels_per_s": proj.d_out / (ms * 1e-3), "phases_ms": q, "loop_ms": loop_ms,
                                   "loop_out_channels_per_s": proj.d_out / (loop_ms * 1e-3),

@@ -111,6 +111,28 @@ class DeviationRecipe:
         return x, xfp
 
 
+def decay_rate(head: int) -> float:
+    """Decay of the synthetic causal attention of a head: rho_h = 1 - 2^-(1 + h mod 6)."""
+    return 1.0 - 2.0 ** -(1 + head % 6)
+
+
+def causal_decay_mix(X: np.ndarray, rho: float, seq_len: int, bf16: bool = True) -> np.ndarray:
+    """Stand-in for the attention-weighted inputs A_h X of a value projection: inside every
+    sequence of seq_len tokens, row t of A_h holds rho^(t-s) for s <= t, normalised to sum 1.
+    Evaluated as the recurrence num_t = rho num_(t-1) + x_t, den_t = rho den_(t-1) + 1,
+    xbar_t = num_t / den_t, in float64; the result is rounded to bf16-representable float32."""
+    n, d = X.shape
+    out = np.empty((n, d), np.float32)
+    for s0 in range(0, n, seq_len):
+        num = np.zeros(d, np.float64)
+        den = 0.0
+        for t in range(s0, min(s0 + seq_len, n)):
+            num = rho * num + X[t]
+            den = rho * den + 1.0
+            out[t] = (num / den).astype(np.float32)
+    return bf16_bits_to_f32(to_bf16_bits(out)) if bf16 else out
+
+
 def spd_matrix(seed: int, n: int, cond: float = 1e3, tid: int = T_HOUT) -> np.ndarray:
     """V diag(lambda) V^T with V the Q-factor of a Gaussian matrix and lambda
     log-spaced from 1 down to 1/cond.  float32 (the layout the library takes)."""

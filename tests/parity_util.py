@@ -28,13 +28,17 @@ def f32(a):
 
 
 def make_problem(seed, d_in, n_heads, d_head, n_tok, *, with_r=False, hout="proj", n_hin=1,
-                 g_heads=None, damp=0.01, alpha=0.25, gaussian_x=False):
+                 g_heads=None, damp=0.01, alpha=0.25, gaussian_x=False, vmix_seq=None):
     """float32 inputs of one projection, every derived tensor computed by the oracle."""
     d_out = n_heads * d_head
     W = tb_inputs.weight(seed, d_out, d_in)
     Hin, Uin, Hsum, R, P, C = [], [], [], [], [], []
     for u in range(n_hin):
-        if gaussian_x:
+        if vmix_seq:
+            # value projection: head u sees the attention-weighted inputs A_u X of the same tokens
+            base = tb_inputs.HeavyTailRecipe(d_in, seed=seed).chunk(0, n_tok)
+            X, Xfp = tb_inputs.causal_decay_mix(base, tb_inputs.decay_rate(u), vmix_seq), None
+        elif gaussian_x:
             X = tb_inputs.activations_gaussian(seed + 101 * u, n_tok, d_in)
             Xfp = None
         else:

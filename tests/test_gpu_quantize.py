@@ -126,6 +126,15 @@ def test_o_proj_identity_hout_sampled_rows():
     compare(prob, gpu, 2, 128, 32, ADAPT | CD, heads=[3], label="o_proj GPTQ mode, sampled rows")
 
 
+def test_v_proj_per_head_hessians_full_width():
+    """v_proj row of Table 1 at full width: every head has its own H_in = X-bar_h^T X-bar_h with
+    X-bar_h = A_h X (synthetic causal decay per head), its own factor, and H_out from the output
+    projection side (here an explicit SPD block).  Two heads of 128 rows, 4096 wide, INT2, g = 32."""
+    prob = make_problem(4, 4096, 2, 128, 4096, n_hin=2, hout="spd", vmix_seq=2048)
+    gpu = run_gpu(prob, 2, 128, 32, ADAPT | CD)
+    compare(prob, gpu, 2, 128, 32, ADAPT | CD, heads=[1], label="v_proj per-head H_in, sampled head")
+
+
 @pytest.mark.parametrize("g", [32, 1])
 def test_llama70b_q_proj_shape_sampled_head(g):
     """Config 5's q_proj: 8192 x 8192, 64 heads x 128, INT2, group 128, fixed grid, no CD (the paper's
