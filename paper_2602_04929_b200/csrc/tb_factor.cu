@@ -28,7 +28,7 @@ namespace tb {
 
 // split-bf16 tensor-core product (tb_gemm_tc.cu): C (+)= A B in double from operands in three bf16 pieces
 tb_status gemm_split_presplit(double* C, long long ldc, const __nv_bfloat16* AT, const __nv_bfloat16* Bp, long long M,
-                              int N, int K, bool accumulate, cudaStream_t st);
+                              int N, int K, bool accumulate, cudaStream_t st, int hunits = 1);
 tb_status split3_transpose(const double* A, __nv_bfloat16* AT, long long M, int K, cudaStream_t st);
 tb_status split3_transpose(const float* A, __nv_bfloat16* AT, long long M, int K, cudaStream_t st);
 tb_status split3(const float* B, __nv_bfloat16* Bp, long long n, cudaStream_t st);

@@ -72,7 +72,7 @@ __global__ void k_wbar_transpose(const unsigned char* __restrict__ codes, const 
 
 __global__ void __launch_bounds__(YT_THREADS, 1)
     k_yw_tc(float* __restrict__ Yw, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-            int rows, int d, int seg, int ng, int n_units) {
+            int rows, int d, int seg, int ng, int n_units, int hunits, int rows_per_hunit) {
   extern __shared__ unsigned char yt_raw[];
   const uint32_t raw = smem_u32(yt_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -116,7 +116,10 @@ __global__ void __launch_bounds__(YT_THREADS, 1)
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
 
-  const int m_tiles = (rows + YT_BM - 1) / YT_BM, n_tilesN = (d + YT_BN - 1) / YT_BN;
+  // hunits > 1: every block of rows_per_hunit rows (a head; a multiple of 128) has its own H_in, whose
+  // pieces are stacked [piece][head][k]; the units then also run over the heads
+  const int m_tiles = (rows_per_hunit + YT_BM - 1) / YT_BM, n_tilesN = (d + YT_BN - 1) / YT_BN;
+  const int units_per_head = ng * n_tilesN;
   const int khalves = seg / 64;  // 1 or 2 boxes of 64 contraction steps per group
   // unit u -> (group g, column tile nj): the unit's slice of H_in stays in shared memory while
   // the row tiles stream through
@@ -124,7 +127,8 @@ __global__ void __launch_bounds__(YT_THREADS, 1)
     if (lane == 0) {
       uint32_t it = 0, unit_it = 0;
       for (int u = blockIdx.x; u < n_units && !*abort_flag; u += gridDim.x, ++unit_it) {
-        const int g = u / n_tilesN, nj = u % n_tilesN;
+        const int hu = u / units_per_head, ur = u % units_per_head;
+        const int g = ur / n_tilesN, nj = ur % n_tilesN;
         const int n0 = nj * YT_BN, k00 = g * seg;
         if (!mbar_wait(bempty_bar, (unit_it & 1u) ^ 1u, abort_flag, &g_yt_error)) break;
         mbar_expect_tx(bfull_bar, 3u * khalves * 2u * YT_BOX);
@@ -133,7 +137,8 @@ __global__ void __launch_bounds__(YT_THREADS, 1)
           for (int kh = 0; kh < khalves; ++kh)
 #pragma unroll
             for (int j = 0; j < 2; ++j)
-              tma_load_2d(sb + ((pc * 2 + kh) * 2 + j) * YT_BOX, &map_b, n0 + 64 * j, pc * d + k00 + 64 * kh, bfull_bar);
+              tma_load_2d(sb + ((pc * 2 + kh) * 2 + j) * YT_BOX, &map_b, n0 + 64 * j,
+                          (pc * hunits + hu) * d + k00 + 64 * kh, bfull_bar);
         bool ok = true;
         for (int mi = 0; mi < m_tiles; ++mi, ++it) {
           const int s = it % YT_STAGES;
@@ -147,7 +152,8 @@ __global__ void __launch_bounds__(YT_THREADS, 1)
           for (int kh = 0; kh < khalves; ++kh)
 #pragma unroll
             for (int j = 0; j < 2; ++j)
-              tma_load_2d(sa + (kh * 2 + j) * YT_BOX, &map_a, mi * YT_BM + 64 * j, k00 + 64 * kh, afull_bar(s));
+              tma_load_2d(sa + (kh * 2 + j) * YT_BOX, &map_a, hu * rows_per_hunit + mi * YT_BM + 64 * j, k00 + 64 * kh,
+                          afull_bar(s));
         }
         if (!ok) break;
       }
@@ -197,7 +203,8 @@ __global__ void __launch_bounds__(YT_THREADS, 1)
     float* st = stage + warp * (32 * 33);
     uint32_t it = 0;
     for (int u = blockIdx.x; u < n_units && !*abort_flag; u += gridDim.x) {
-      const int g = u / n_tilesN, nj = u % n_tilesN;
+      const int hu = u / units_per_head, ur = u % units_per_head;
+      const int g = ur / n_tilesN, nj = ur % n_tilesN;
       bool ok = true;
       for (int mi = 0; mi < m_tiles; ++mi, ++it) {
         const int b = it & 1;
@@ -214,7 +221,7 @@ __global__ void __launch_bounds__(YT_THREADS, 1)
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncwarp();
         if (lane == 0) mbar_arrive(acce_bar(b));   // the accumulator may be overwritten
-        const long long gr0 = (long long)mi * YT_BM + q * 32;
+        const long long gr0 = (long long)hu * rows_per_hunit + (long long)mi * YT_BM + q * 32;
         const int gc0 = nj * YT_BN + hf * 64;
 #pragma unroll
         for (int c = 0; c < 2; ++c) {
@@ -405,10 +412,12 @@ __global__ void __launch_bounds__(YT_THREADS, 1)
 // Yw (float, [rows][ng][d]) from the codes; WbT ([d][rows] bf16) and Hp ([3][d][d] bf16) are scratch.
 // Requires seg % 64 == 0, d % 8 == 0, rows % 8 == 0.
 tb_status yw_tensor(float* Yw, const unsigned char* codes, const int* zeros, const float* H_in, __nv_bfloat16* WbT,
-                    __nv_bfloat16* Hp, bool split_h, long long rows, int d, int seg, int ng, cudaStream_t st) {
+                    __nv_bfloat16* Hp, bool split_h, long long rows, int d, int seg, int ng, int hunits,
+                    cudaStream_t st) {
   const long long dd = (long long)d * d;
+  if (hunits > 1 && (seg > 128 || (rows / hunits) % YT_BM || rows % hunits)) return TB_ERR_UNSUPPORTED;
   if (split_h) {
-    k_split3<<<148 * 8, 256, 0, st>>>(H_in, Hp, dd);
+    k_split3<<<148 * 8, 256, 0, st>>>(H_in, Hp, dd * hunits);
     TB_LAUNCH_CHECK();
   }
   k_wbar_transpose<<<dim3(d / 32, (unsigned)((rows + 31) / 32)), dim3(32, 8), 0, st>>>(codes, zeros, WbT, rows, d, seg, ng);
@@ -416,11 +425,11 @@ tb_status yw_tensor(float* Yw, const unsigned char* codes, const int* zeros, con
   CUtensorMap map_a, map_b;
   TB_TRY(make_map_2d(&map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, WbT, (unsigned long long)rows, (unsigned long long)d,
                      64, 64, CU_TENSOR_MAP_SWIZZLE_128B));
-  TB_TRY(make_map_2d(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Hp, (unsigned long long)d, (unsigned long long)3 * d,
-                     64, 64, CU_TENSOR_MAP_SWIZZLE_128B));
+  TB_TRY(make_map_2d(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Hp, (unsigned long long)d,
+                     (unsigned long long)3 * hunits * d, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B));
   const int m_tiles = (int)((rows + YT_BM - 1) / YT_BM), n_tilesN = (d + YT_BN - 1) / YT_BN;
   const bool resident = (seg <= 128);  // the group's slice of H_in fits next to the Wbar^T ring
-  const long long n_tiles = resident ? (long long)n_tilesN * ng   // units: one (group, column tile) pair each
+  const long long n_tiles = resident ? (long long)n_tilesN * ng * hunits   // units: one (head, group, column tile) each
                                      : (long long)m_tiles * n_tilesN * ng;
   if (n_tiles > 0x7fffffffll) return TB_ERR_UNSUPPORTED;
   int dev = 0, sms = 0;
@@ -435,7 +444,8 @@ tb_status yw_tensor(float* Yw, const unsigned char* codes, const int* zeros, con
   }
   const int grid = (int)(n_tiles < sms ? n_tiles : sms);
   if (resident)
-    k_yw_tc<<<grid, YT_THREADS, YT_SMEM, st>>>(Yw, map_a, map_b, (int)rows, d, seg, ng, (int)n_tiles);
+    k_yw_tc<<<grid, YT_THREADS, YT_SMEM, st>>>(Yw, map_a, map_b, (int)rows, d, seg, ng, (int)n_tiles, hunits,
+                                               (int)(rows / hunits));
   else
     k_yw_tc_stream<<<grid, YT_THREADS, YS_SMEM, st>>>(Yw, map_a, map_b, (int)rows, d, seg, ng, (int)n_tiles);
   TB_LAUNCH_CHECK();
@@ -494,7 +504,8 @@ __global__ void k_split3_transpose(const TA* __restrict__ A, __nv_bfloat16* __re
 
 __global__ void __launch_bounds__(YT_THREADS, 1)
     k_gsplit_tc(double* __restrict__ C, long long ldc, const __grid_constant__ CUtensorMap map_a,
-                const __grid_constant__ CUtensorMap map_b, int M, int N, int K, int n_tiles, int accumulate) {
+                const __grid_constant__ CUtensorMap map_b, int M, int N, int K, int n_tiles, int accumulate, int hunits,
+                int rows_per_hunit) {
   extern __shared__ unsigned char gs_raw[];
   const uint32_t raw = smem_u32(gs_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -540,6 +551,7 @@ __global__ void __launch_bounds__(YT_THREADS, 1)
       uint32_t it = 0;
       for (int t = blockIdx.x; t < n_tiles && !*abort_flag; t += gridDim.x) {
         const int m0 = (t / n_tilesN) * GS_BM, n0 = (t % n_tilesN) * GS_BN;
+        const int hu = (hunits > 1) ? m0 / rows_per_hunit : 0;  // the block of rows (head) whose B this tile multiplies
         for (int st = 0; st < n_stages; ++st, ++it) {
           const int s = it % GS_STAGES;
           const uint32_t ph = (it / GS_STAGES) & 1u;
@@ -552,7 +564,7 @@ __global__ void __launch_bounds__(YT_THREADS, 1)
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
               tma_load_2d(sa + (pc * 2 + j) * GS_BOX, &map_a, m0 + 64 * j, pc * K + k0, full_bar(s));
-              tma_load_2d(sb + (pc * 2 + j) * GS_BOX, &map_b, n0 + 64 * j, pc * K + k0, full_bar(s));
+              tma_load_2d(sb + (pc * 2 + j) * GS_BOX, &map_b, n0 + 64 * j, (pc * hunits + hu) * K + k0, full_bar(s));
             }
         }
       }
@@ -653,13 +665,15 @@ __global__ void __launch_bounds__(YT_THREADS, 1)
 
 // C (+)= A B (double result) from operands already split: AT [3][K][M], Bp [3][K][N].
 // Requires M % 8 == 0, N % 8 == 0, K % 32 == 0.
+// hunits > 1: every block of M / hunits rows (a multiple of 128) multiplies its own B, Bp stacked [3][hunits][K][N].
 tb_status gemm_split_presplit(double* C, long long ldc, const __nv_bfloat16* AT, const __nv_bfloat16* Bp, long long M,
-                              int N, int K, bool accumulate, cudaStream_t st) {
+                              int N, int K, bool accumulate, cudaStream_t st, int hunits) {
+  if (hunits > 1 && (M % hunits || (M / hunits) % GS_BM)) return TB_ERR_UNSUPPORTED;
   CUtensorMap map_a, map_b;
   TB_TRY(make_map_2d(&map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, AT, (unsigned long long)M, (unsigned long long)3 * K,
                      64, 32, CU_TENSOR_MAP_SWIZZLE_128B));
-  TB_TRY(make_map_2d(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Bp, (unsigned long long)N, (unsigned long long)3 * K,
-                     64, 32, CU_TENSOR_MAP_SWIZZLE_128B));
+  TB_TRY(make_map_2d(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Bp, (unsigned long long)N,
+                     (unsigned long long)3 * hunits * K, 64, 32, CU_TENSOR_MAP_SWIZZLE_128B));
   const long long n_tiles = ((M + GS_BM - 1) / GS_BM) * (long long)((N + GS_BN - 1) / GS_BN);
   if (n_tiles > 0x7fffffffll) return TB_ERR_UNSUPPORTED;
   int dev = 0, sms = 0;
@@ -672,7 +686,8 @@ tb_status gemm_split_presplit(double* C, long long ldc, const __nv_bfloat16* AT,
     configured[dev] = true;
   }
   const int grid = (int)(n_tiles < sms ? n_tiles : sms);
-  k_gsplit_tc<<<grid, YT_THREADS, GS_SMEM, st>>>(C, ldc, map_a, map_b, (int)M, N, K, (int)n_tiles, accumulate ? 1 : 0);
+  k_gsplit_tc<<<grid, YT_THREADS, GS_SMEM, st>>>(C, ldc, map_a, map_b, (int)M, N, K, (int)n_tiles, accumulate ? 1 : 0,
+                                                 hunits, (int)(M / hunits));
   TB_LAUNCH_CHECK();
   return TB_OK;
 }
@@ -701,7 +716,7 @@ tb_status gemm_split_tensor(double* C, long long ldc, const float* A, const floa
                             __nv_bfloat16* Bp, long long M, int N, int K, cudaStream_t st) {
   TB_TRY(split3(B, Bp, (long long)K * N, st));
   TB_TRY(split3_transpose(A, AT, M, K, st));
-  return gemm_split_presplit(C, ldc, AT, Bp, M, N, K, false, st);
+  return gemm_split_presplit(C, ldc, AT, Bp, M, N, K, false, st, 1);
 }
 
 int yw_error_read_clear() {

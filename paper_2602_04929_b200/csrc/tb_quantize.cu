@@ -26,10 +26,11 @@ namespace cg = cooperative_groups;
 namespace tb {
 // tensor-core blockwise product of the scale refinement (tb_gemm_tc.cu)
 tb_status yw_tensor(float* Yw, const unsigned char* codes, const int* zeros, const float* H_in, __nv_bfloat16* WbT,
-                    __nv_bfloat16* Hp, bool split_h, long long rows, int d, int seg, int ng, cudaStream_t st);
+                    __nv_bfloat16* Hp, bool split_h, long long rows, int d, int seg, int ng, int hunits,
+                    cudaStream_t st);
 // C (+)= A B in double from operands split into three bf16 pieces each (tb_gemm_tc.cu)
 tb_status gemm_split_presplit(double* C, long long ldc, const __nv_bfloat16* AT, const __nv_bfloat16* Bp, long long M,
-                              int N, int K, bool accumulate, cudaStream_t st);
+                              int N, int K, bool accumulate, cudaStream_t st, int hunits = 1);
 tb_status split3_transpose(const double* A, __nv_bfloat16* AT, long long M, int K, cudaStream_t st);
 tb_status split3_transpose(const float* A, __nv_bfloat16* AT, long long M, int K, cudaStream_t st);
 tb_status split3(const float* B, __nv_bfloat16* Bp, long long n, cudaStream_t st);
@@ -1498,11 +1499,14 @@ static tb_status make_plan(const tb_layer_desc* D, bool has_hout, bool with_r, b
     p.cd_rows = rows;
     p.Yw = b.take<double>((size_t)rows * p.ng * dd);
     // blockwise product on the tensor cores (float result): one shared H_in, groups that are whole TMA boxes
-    p.yw_tensor = (p.n_hin == 1) && (p.seg % 64 == 0) && (rows % 8 == 0) && (p.d_out % 8 == 0) &&
+    // With one H_in per head the heads of a batch go through the same launches, each against its own
+    // pieces of H_in; that needs heads of whole 128-row tiles and groups of at most 128 columns.
+    const bool per_head_ok = (p.n_hin > 1) && (p.dh % 128 == 0) && (p.seg <= 128) && (rows % p.dh == 0);
+    p.yw_tensor = (p.n_hin == 1 || per_head_ok) && (p.seg % 64 == 0) && (rows % 8 == 0) && (p.d_out % 8 == 0) &&
                   (p.dh % 8 == 0 || rows == p.d_out);
     if (p.yw_tensor) {
       p.WbT = b.take<__nv_bfloat16>((size_t)rows * dd);
-      p.Hp = b.take<__nv_bfloat16>((size_t)3 * dd * dd);
+      p.Hp = b.take<__nv_bfloat16>((size_t)3 * dd * dd * (p.n_hin > 1 ? (size_t)(rows / p.dh) : 1));
       p.dm_tensor = (p.d % 32 == 0);
     }
     const long long lines = rows;  // one set of statistics per row (the column-parallel pass keeps them all)
@@ -1794,13 +1798,16 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
       const long long rows = (p.d_out - r0 < p.cd_rows) ? (p.d_out - r0) : p.cd_rows;
       // Dm = (Q - W) H_in (+ W R); Yw = blockwise Wbar H_in.  With one H_in per head the
       // batch is whole heads and the products run head by head.
-      const long long rows_per_prod = (units > 1) ? p.dh : rows;
+      const bool heads_together = p.yw_tensor && units > 1;   // per-head H_in on the tensor-core path
+      const int hunits = heads_together ? (int)(rows / p.dh) : 1;
+      const long long rows_per_prod = (units > 1 && !heads_together) ? p.dh : rows;
       for (long long q0 = 0; q0 < rows; q0 += rows_per_prod) {
         const long long rr = r0 + q0;
         const float* Hh = H_in + ((units > 1) ? (rr / p.dh) * dd : 0);
         if (p.yw_tensor)  // also splits H_in into its bf16 pieces on the first batch
-          TB_TRY(yw_tensor(reinterpret_cast<float*>(p.Yw), codes + rr * d, zeros + rr * p.ng, H_in, p.WbT, p.Hp,
-                           r0 == 0 || with_r, rows, d, p.seg, p.ng, st));  // with R the pieces of R replace H_in's below
+          TB_TRY(yw_tensor(reinterpret_cast<float*>(p.Yw), codes + rr * d, zeros + rr * p.ng, Hh, p.WbT, p.Hp,
+                           r0 == 0 || with_r || units > 1, rows, d, p.seg, p.ng, hunits,
+                           st));  // with R the pieces of R replace H_in's below
         GemmP g = gemm_params();
         g.A = p.Dq + rr * d;
         g.a_m = d;
@@ -1818,7 +1825,7 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
           // and overwritten by G = H_out Dm only after the product)
           __nv_bfloat16* DqT = reinterpret_cast<__nv_bfloat16*>(p.Wt + rr * d);
           TB_TRY(split3_transpose(p.Dq + rr * d, DqT, rows, d, st));
-          TB_TRY(gemm_split_presplit(p.Dm + rr * d, d, DqT, p.Hp, rows, d, d, false, st));
+          TB_TRY(gemm_split_presplit(p.Dm + rr * d, d, DqT, p.Hp, rows, d, d, false, st, hunits));
         } else {
           TB_TRY((gemm_launch<double, float, double, double, false, true>(g, st)));
         }
@@ -1826,8 +1833,8 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
           // Dm += W R through the same split-bf16 product; the pieces of R take the place of H_in's
           __nv_bfloat16* WT = reinterpret_cast<__nv_bfloat16*>(p.Wt + rr * d);
           TB_TRY(split3_transpose(W + rr * d, WT, rows, d, st));
-          TB_TRY(split3(R, p.Hp, dd, st));
-          TB_TRY(gemm_split_presplit(p.Dm + rr * d, d, WT, p.Hp, rows, d, d, true, st));
+          TB_TRY(split3(R + ((units > 1) ? (rr / p.dh) * dd : 0), p.Hp, dd * hunits, st));
+          TB_TRY(gemm_split_presplit(p.Dm + rr * d, d, WT, p.Hp, rows, d, d, true, st, hunits));
         } else if (with_r) {
           GemmP h = g;
           h.A = W + rr * d;
