@@ -487,6 +487,7 @@ struct RowSweepP {
   RowMap rm;
   int M, d, seg, ng, maxq, nblk;
   int units, rows_per_unit, ctas_per_unit;
+  int cs;                // CTAs that share a group of 8 rows (1, or a cluster of 2 or 4 when rows are few)
 };
 struct RowSweepStage {
   float Ub[RS_CHUNK][RS_LDB];   // 64 rows of U or P: 128 columns of the target block + 8 spare
@@ -505,6 +506,7 @@ struct RowSweepSmem {
   double Es[8][RS_LDW];         // normalised errors of the current block
   double As[WITH_P ? 8 : 1][RS_LDW];  // arrival values of the current block
   unsigned long long full_bar[STAGES], empty_bar[STAGES];
+  unsigned long long cfull_bar[8], cempty_bar[8];  // ring of the cluster form (more, smaller stages)
   int abort_flag;
 };
 __device__ int g_sweep_error = 0;
@@ -516,6 +518,7 @@ __device__ __forceinline__ void mma_f64(double (&c)[2], double a, double b) {
 }
 __device__ __forceinline__ void bar_all() { asm volatile("bar.sync 3, 512;" ::: "memory"); }
 
+
 template <bool WITH_P>
 __global__ void __launch_bounds__(RS_THREADS, 1)
     k_sweep_rows(RowSweepP p, const __grid_constant__ CUtensorMap map_u, const __grid_constant__ CUtensorMap map_e,
@@ -526,8 +529,28 @@ __global__ void __launch_bounds__(RS_THREADS, 1)
   constexpr int NOP = WITH_P ? 2 : 1;  // operand pairs per 64-row chunk: (Err, U) and (Arr, P)
   Smem& sm = *reinterpret_cast<Smem*>(rs_raw);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int unit = blockIdx.x / p.ctas_per_unit;
-  const int r_first = (blockIdx.x % p.ctas_per_unit) * 8;  // first row of this CTA inside its unit
+  // With few rows per launch a cluster of cs CTAs shares a group of 8 rows: each prepares 128 / cs
+  // columns of the next block (its share of the contraction work) and writes them into the shared
+  // memory of all; the panel runs in every CTA on the same values, so all of them hold the block's
+  // errors and write identical results.
+  cg::cluster_group cluster = cg::this_cluster();
+  const int cs = p.cs;
+  const int crank = (cs > 1) ? (int)cluster.block_rank() : 0;
+  const int grp = blockIdx.x / cs;
+  const int unit = grp / p.ctas_per_unit;
+  const int r_first = (grp % p.ctas_per_unit) * 8;  // first row of this group inside its unit
+  // arrival values of the blocks: with a cluster the buffers alternate (a fast CTA may write block b + 1
+  // while a slow one still reads block b); the second one sits in the part of ring stage 0 that the
+  // narrower boxes of a cluster leave free
+  // The cluster form cuts the ring's memory into more, smaller stages (its boxes of U are 128 / cs + 8
+  // floats wide), as many as fit beside the second arrival buffer, at most 8: with short chunks only
+  // the number of loads in flight hides their latency.
+  const int c_ldb = 128 / cs + 8;
+  const int c_stage_bytes = RS_CHUNK * c_ldb * (int)sizeof(float) + (int)sizeof(RowSweepStage::Eb);
+  const int c_nst = min(8, (int)((sizeof(sm.ring) - sizeof(sm.wblk)) / c_stage_bytes));
+  unsigned char* ring_base = reinterpret_cast<unsigned char*>(&sm.ring[0]);
+  double* wbuf0 = &sm.wblk[0][0];
+  double* wbuf1 = (cs > 1) ? reinterpret_cast<double*>(ring_base + (size_t)c_nst * c_stage_bytes) : wbuf0;
   const int d = p.d;
   const long long uoff = (long long)unit * d * d * (p.units > 1 ? 1 : 0);
   const float* U = p.U + uoff;
@@ -545,6 +568,10 @@ __global__ void __launch_bounds__(RS_THREADS, 1)
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(smem_u32(&sm.full_bar[s]), 1);
       mbar_init(smem_u32(&sm.empty_bar[s]), 8);  // one arrival per update warp
+    }
+    for (int s = 0; s < 8; ++s) {
+      mbar_init(smem_u32(&sm.cfull_bar[s]), 1);
+      mbar_init(smem_u32(&sm.cempty_bar[s]), (cs > 1) ? 16 / cs : 8);  // one arrival per working update warp
     }
     sm.abort_flag = 0;
     mbar_fence_init();
@@ -583,7 +610,7 @@ __global__ void __launch_bounds__(RS_THREADS, 1)
       double w[4], rs4[4], rd4[4];
 #pragma unroll
       for (int sb = 0; sb < 4; ++sb) {
-        w[sb] = sm.wblk[warp][sb * 32 + lane];
+        w[sb] = ((b & 1) ? wbuf1 : wbuf0)[warp * 128 + sb * 32 + lane];
         rs4[sb] = 1.0 / s4[sb];
         rd4[sb] = 1.0 / (double)sm.sU[tri_base(sb) + lane * (128 - 32 * sb) + lane];
       }
@@ -681,15 +708,18 @@ __global__ void __launch_bounds__(RS_THREADS, 1)
       // the histories are read back by TMA (async proxy): order these stores before it
       asm volatile("fence.proxy.async;" ::: "memory");
       bar_all();  // block b is quantized: its errors are in Es and in the history
-      bar_all();  // block b+1 has been handed over in wblk
+      if (cs > 1)
+        cluster.sync();  // block b+1 has been handed over by all CTAs of the cluster
+      else
+        bar_all();       // block b+1 has been handed over in wblk
     }
-    if (p.stats) {
+    if (p.stats && crank == 0) {
       n_near = __reduce_add_sync(0xffffffffu, n_near);
       n_clamp = __reduce_add_sync(0xffffffffu, n_clamp);
       if (lane == 0) {
         if (n_near) atomicAdd(&p.stats->near_tie_codes, (unsigned long long)n_near);
         if (n_clamp) atomicAdd(&p.stats->clamped_codes, (unsigned long long)n_clamp);
-        if (blockIdx.x == 0 && warp == 0) atomicAdd(&p.stats->column_steps, (unsigned long long)d);
+        if (grp == 0 && warp == 0) atomicAdd(&p.stats->column_steps, (unsigned long long)d);
       }
     }
     return;
@@ -713,6 +743,90 @@ __global__ void __launch_bounds__(RS_THREADS, 1)
   // ring positions: `c_*` of the consumers (all update warps), `p_*` of the producer thread
   int c_slot = 0, p_slot = 0;
   uint32_t c_phase = 0, p_phase = 0;
+  if (cs > 1) {
+    // ---- cluster form: this CTA prepares columns crank * wc .. + wc - 1 of the next block, one 8-column
+    // fragment per working warp; the boxes of U are wc + 8 floats wide ----
+    const int wc = 128 / cs, ldb = c_ldb, frags = 16 / cs;
+    const int ub_bytes = RS_CHUNK * ldb * (int)sizeof(float);
+    const bool working = uw < frags;
+    const int n_blk = crank * wc + uw * 8;   // first column of this warp's fragment inside the block
+    for (int b = 0; b < p.nblk; ++b) {
+      if (b + 1 >= p.nblk) {
+        bar_all();
+        cluster.sync();
+        break;
+      }
+      const int cn = (b + 1) * 128;
+      const int n_hist = 2 * b * NOP, n_all = n_hist + 2 * NOP;
+      double* wnext = ((b + 1) & 1) ? wbuf1 : wbuf0;
+      if (working) {
+        double acc[8][2];  // eight accumulators in turn: one fragment per warp has to cover the latency alone
+#pragma unroll
+        for (int i = 0; i < 16; ++i) (&acc[0][0])[i] = 0.0;
+        double w0[2];
+#pragma unroll
+        for (int e = 0; e < 2; ++e) w0[e] = fr_valid ? p.Wt[fr_grow * d + cn + n_blk + 2 * fk + e] : 0.0;
+        auto produce = [&](int c) {
+          if (c < n_all) {
+            if ((c % frags) == uw) {
+              unsigned char* stg = ring_base + (size_t)p_slot * c_stage_bytes;
+              const uint32_t fb = smem_u32(&sm.cfull_bar[p_slot]);
+              if (mbar_wait(smem_u32(&sm.cempty_bar[p_slot]), p_phase ^ 1u, abort_flag, &g_sweep_error)) {
+                const bool hist = c < n_hist;
+                const bool second = WITH_P && (c & 1);
+                const int kc = c / NOP;
+                mbar_expect_tx(fb, (uint32_t)(ub_bytes + (hist ? sizeof(RowSweepStage::Eb) : 0)));
+                tma_load_2d(smem_u32(stg), second ? &map_p : &map_u, cn + crank * wc, u_row0 + kc * RS_CHUNK, fb);
+                if (hist) tma_load_2d(smem_u32(stg + ub_bytes), second ? &map_a : &map_e, kc * RS_CHUNK, m_base, fb);
+              }
+            }
+            if (++p_slot == c_nst) {
+              p_slot = 0;
+              p_phase ^= 1u;
+            }
+          }
+        };
+        if (lane0)
+          for (int c = 0; c < c_nst - 1; ++c) produce(c);
+        for (int c = 0; c < n_all; ++c) {
+          if (c == n_hist) bar_all();
+          const unsigned char* stg = ring_base + (size_t)c_slot * c_stage_bytes;
+          const double* eb = reinterpret_cast<const double*>(stg + ub_bytes);  // [8][RS_LDE]
+          const bool ok = mbar_wait(smem_u32(&sm.cfull_bar[c_slot]), c_phase, abort_flag, &g_sweep_error);
+          if (ok) {
+            const int own = (c - n_hist) / NOP;
+            const double* ap;
+            if (c < n_hist)
+              ap = eb + fr * RS_LDE + fk;
+            else if (WITH_P && (c & 1))
+              ap = &sm.As[fr][own * RS_CHUNK + fk];
+            else
+              ap = &sm.Es[fr][own * RS_CHUNK + fk];
+            const float* bp = reinterpret_cast<const float*>(stg) + fk * ldb + uw * 8 + fr;
+#pragma unroll
+            for (int q = 0; q < 16; ++q) mma_f64(acc[q & 7], ap[4 * q], (double)bp[4 * q * ldb]);
+          }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&sm.cempty_bar[c_slot]));
+          if (++c_slot == c_nst) {
+            c_slot = 0;
+            c_phase ^= 1u;
+          }
+          if (lane0) produce(c + c_nst - 1);
+        }
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const double v = w0[e] - (((acc[0][e] + acc[1][e]) + (acc[2][e] + acc[3][e])) +
+                                    ((acc[4][e] + acc[5][e]) + (acc[6][e] + acc[7][e])));
+          for (int r = 0; r < cs; ++r) cluster.map_shared_rank(wnext, r)[fr * 128 + n_blk + 2 * fk + e] = v;
+        }
+      } else {
+        bar_all();  // the barrier the working warps pass once the panel has finished block b
+      }
+      cluster.sync();  // block b+1 handed over
+    }
+    return;
+  }
   for (int b = 0; b < p.nblk; ++b) {
     if (b + 1 >= p.nblk) {  // nothing left to prepare
       bar_all();
@@ -1602,8 +1716,25 @@ static tb_status launch_sweep_rows(const RowSweepP& sp, const CUtensorMap& mu, c
   auto kern = k_sweep_rows<WITH_P>;
   static bool configured[64] = {false};
   TB_TRY(allow_smem(kern, sizeof(RowSweepSmem<WITH_P>), configured));
-  const long long ctas = (long long)sp.ctas_per_unit * sp.units;
-  kern<<<(unsigned)ctas, RS_THREADS, sizeof(RowSweepSmem<WITH_P>), st>>>(sp, mu, me, mp, ma);
+  const long long ctas = (long long)sp.ctas_per_unit * sp.units * sp.cs;
+  if (sp.cs == 1) {
+    kern<<<(unsigned)ctas, RS_THREADS, sizeof(RowSweepSmem<WITH_P>), st>>>(sp, mu, me, mp, ma);
+    TB_LAUNCH_CHECK();
+    return TB_OK;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)ctas);
+  cfg.blockDim = dim3(RS_THREADS);
+  cfg.dynamicSmemBytes = sizeof(RowSweepSmem<WITH_P>);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)sp.cs;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  TB_CUDA_CHECK(cudaLaunchKernelEx(&cfg, kern, sp, mu, me, mp, ma));
   TB_LAUNCH_CHECK();
   return TB_OK;
 }
@@ -1630,8 +1761,13 @@ static tb_status run_sweep_rows(const Plan& p, const float* U_in, const float* P
   sp.units = (p.n_hin == 1) ? 1 : p.H;
   sp.rows_per_unit = M / sp.units;
   sp.ctas_per_unit = (sp.rows_per_unit + 7) / 8;
+  // few rows: a cluster of 2 or 4 CTAs per group of 8 rows shares the contraction work of the updates
+  const long long groups = (long long)sp.ctas_per_unit * sp.units;
+  sp.cs = (p.d >= 256 && groups * 4 <= 148) ? 4 : (p.d >= 256 && groups * 2 <= 148) ? 2 : 1;
   CUtensorMap map_u, map_e, map_p, map_a;
-  const unsigned box_u = (unsigned)((p.d >= RS_LDB) ? RS_LDB : p.d), box_e = (unsigned)((p.d >= RS_LDE) ? RS_LDE : p.d);
+  const unsigned box_full = (unsigned)((p.d >= RS_LDB) ? RS_LDB : p.d);
+  const unsigned box_u = (sp.cs > 1) ? (unsigned)(128 / sp.cs + 8) : box_full;
+  const unsigned box_e = (unsigned)((p.d >= RS_LDE) ? RS_LDE : p.d);
   const unsigned long long mat_rows = (unsigned long long)p.d * sp.units;
   TB_TRY(make_map_2d(&map_u, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, sizeof(float), U_in, (unsigned long long)p.d, mat_rows,
                      box_u, RS_CHUNK, CU_TENSOR_MAP_SWIZZLE_NONE));
