@@ -473,6 +473,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) k_grid_tri(GridP p) {
 // are bounded: when a bound runs out the kernel raises a device error word and
 // stops computing, but still passes every barrier, so it always terminates.
 // ---------------------------------------------------------------------------
+enum { RS_CCHUNK = 128, RS_CLDE = 132 };  // cluster form: contraction rows per chunk, row pitch of its history box
 enum { RS_THREADS = 512, RS_LDB = 136, RS_LDE = 68, RS_CHUNK = 64, RS_LDW = 132, RS_TRI = 10240 };
 struct RowSweepP {
   const double* Wt;      // [d_out][d] current W~ (rows of the step are read, never written)
@@ -546,7 +547,7 @@ __global__ void __launch_bounds__(RS_THREADS, 1)
   // floats wide), as many as fit beside the second arrival buffer, at most 8: with short chunks only
   // the number of loads in flight hides their latency.
   const int c_ldb = 128 / cs + 8;
-  const int c_stage_bytes = RS_CHUNK * c_ldb * (int)sizeof(float) + (int)sizeof(RowSweepStage::Eb);
+  const int c_stage_bytes = RS_CCHUNK * c_ldb * (int)sizeof(float) + 8 * RS_CLDE * (int)sizeof(double);
   const int c_nst = min(8, (int)((sizeof(sm.ring) - sizeof(sm.wblk)) / c_stage_bytes));
   unsigned char* ring_base = reinterpret_cast<unsigned char*>(&sm.ring[0]);
   double* wbuf0 = &sm.wblk[0][0];
@@ -747,7 +748,10 @@ __global__ void __launch_bounds__(RS_THREADS, 1)
     // ---- cluster form: this CTA prepares columns crank * wc .. + wc - 1 of the next block, one 8-column
     // fragment per working warp; the boxes of U are wc + 8 floats wide ----
     const int wc = 128 / cs, ldb = c_ldb, frags = 16 / cs;
-    const int ub_bytes = RS_CHUNK * ldb * (int)sizeof(float);
+    const int ub_bytes = RS_CCHUNK * ldb * (int)sizeof(float);
+    const int eb_bytes = 8 * RS_CLDE * (int)sizeof(double);
+    // chunks of 128 contraction rows (a whole block): with one fragment per warp a 64-row chunk is too
+    // little work beside the fixed cost of a ring step
     const bool working = uw < frags;
     const int n_blk = crank * wc + uw * 8;   // first column of this warp's fragment inside the block
     for (int b = 0; b < p.nblk; ++b) {
@@ -757,7 +761,7 @@ __global__ void __launch_bounds__(RS_THREADS, 1)
         break;
       }
       const int cn = (b + 1) * 128;
-      const int n_hist = 2 * b * NOP, n_all = n_hist + 2 * NOP;
+      const int n_hist = b * NOP, n_all = n_hist + NOP;
       double* wnext = ((b + 1) & 1) ? wbuf1 : wbuf0;
       if (working) {
         double acc[8][2];  // eight accumulators in turn: one fragment per warp has to cover the latency alone
@@ -775,9 +779,9 @@ __global__ void __launch_bounds__(RS_THREADS, 1)
                 const bool hist = c < n_hist;
                 const bool second = WITH_P && (c & 1);
                 const int kc = c / NOP;
-                mbar_expect_tx(fb, (uint32_t)(ub_bytes + (hist ? sizeof(RowSweepStage::Eb) : 0)));
-                tma_load_2d(smem_u32(stg), second ? &map_p : &map_u, cn + crank * wc, u_row0 + kc * RS_CHUNK, fb);
-                if (hist) tma_load_2d(smem_u32(stg + ub_bytes), second ? &map_a : &map_e, kc * RS_CHUNK, m_base, fb);
+                mbar_expect_tx(fb, (uint32_t)(ub_bytes + (hist ? eb_bytes : 0)));
+                tma_load_2d(smem_u32(stg), second ? &map_p : &map_u, cn + crank * wc, u_row0 + kc * RS_CCHUNK, fb);
+                if (hist) tma_load_2d(smem_u32(stg + ub_bytes), second ? &map_a : &map_e, kc * RS_CCHUNK, m_base, fb);
               }
             }
             if (++p_slot == c_nst) {
@@ -791,20 +795,19 @@ __global__ void __launch_bounds__(RS_THREADS, 1)
         for (int c = 0; c < n_all; ++c) {
           if (c == n_hist) bar_all();
           const unsigned char* stg = ring_base + (size_t)c_slot * c_stage_bytes;
-          const double* eb = reinterpret_cast<const double*>(stg + ub_bytes);  // [8][RS_LDE]
+          const double* eb = reinterpret_cast<const double*>(stg + ub_bytes);  // [8][RS_CLDE]
           const bool ok = mbar_wait(smem_u32(&sm.cfull_bar[c_slot]), c_phase, abort_flag, &g_sweep_error);
           if (ok) {
-            const int own = (c - n_hist) / NOP;
             const double* ap;
             if (c < n_hist)
-              ap = eb + fr * RS_LDE + fk;
+              ap = eb + fr * RS_CLDE + fk;
             else if (WITH_P && (c & 1))
-              ap = &sm.As[fr][own * RS_CHUNK + fk];
+              ap = &sm.As[fr][fk];
             else
-              ap = &sm.Es[fr][own * RS_CHUNK + fk];
+              ap = &sm.Es[fr][fk];
             const float* bp = reinterpret_cast<const float*>(stg) + fk * ldb + uw * 8 + fr;
 #pragma unroll
-            for (int q = 0; q < 16; ++q) mma_f64(acc[q & 7], ap[4 * q], (double)bp[4 * q * ldb]);
+            for (int q = 0; q < RS_CCHUNK / 4; ++q) mma_f64(acc[q & 7], ap[4 * q], (double)bp[4 * q * ldb]);
           }
           __syncwarp();
           if (lane == 0) mbar_arrive(smem_u32(&sm.cempty_bar[c_slot]));
@@ -1767,15 +1770,16 @@ static tb_status run_sweep_rows(const Plan& p, const float* U_in, const float* P
   CUtensorMap map_u, map_e, map_p, map_a;
   const unsigned box_full = (unsigned)((p.d >= RS_LDB) ? RS_LDB : p.d);
   const unsigned box_u = (sp.cs > 1) ? (unsigned)(128 / sp.cs + 8) : box_full;
-  const unsigned box_e = (unsigned)((p.d >= RS_LDE) ? RS_LDE : p.d);
+  const unsigned box_e = (sp.cs > 1) ? (unsigned)RS_CLDE : (unsigned)((p.d >= RS_LDE) ? RS_LDE : p.d);
+  const unsigned box_k = (sp.cs > 1) ? (unsigned)RS_CCHUNK : (unsigned)RS_CHUNK;
   const unsigned long long mat_rows = (unsigned long long)p.d * sp.units;
   TB_TRY(make_map_2d(&map_u, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, sizeof(float), U_in, (unsigned long long)p.d, mat_rows,
-                     box_u, RS_CHUNK, CU_TENSOR_MAP_SWIZZLE_NONE));
+                     box_u, box_k, CU_TENSOR_MAP_SWIZZLE_NONE));
   TB_TRY(make_map_2d(&map_e, CU_TENSOR_MAP_DATA_TYPE_FLOAT64, sizeof(double), sp.ErrG, (unsigned long long)p.d,
                      (unsigned long long)M, box_e, 8, CU_TENSOR_MAP_SWIZZLE_NONE));
   if (!P) return launch_sweep_rows<false>(sp, map_u, map_e, map_u, map_e, st);
   TB_TRY(make_map_2d(&map_p, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, sizeof(float), P, (unsigned long long)p.d, mat_rows,
-                     box_u, RS_CHUNK, CU_TENSOR_MAP_SWIZZLE_NONE));
+                     box_u, box_k, CU_TENSOR_MAP_SWIZZLE_NONE));
   TB_TRY(make_map_2d(&map_a, CU_TENSOR_MAP_DATA_TYPE_FLOAT64, sizeof(double), sp.ArrG, (unsigned long long)p.d,
                      (unsigned long long)M, box_e, 8, CU_TENSOR_MAP_SWIZZLE_NONE));
   return launch_sweep_rows<true>(sp, map_u, map_e, map_p, map_a, st);
