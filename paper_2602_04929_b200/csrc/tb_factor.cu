@@ -15,11 +15,15 @@
 //        k_chol_panel  every CTA factors the 64 x 64 diagonal block (one thread
 //                      per row, the row in registers, right-looking) and then
 //                      solves its 64 rows of the panel against it
-//        GEMM          trailing matrix -= panel panel^T  (tiles on/below the diagonal)
-//   3. inverses of the 64 x 64 diagonal blocks, all at once (k_inv_diag64)
+//                      (after applying the previous panel's update to its own columns)
+//        GEMM          trailing matrix -= panel panel^T from the panel after the next on
+//                      (tiles on/below the diagonal)
+//   3. inverses of the 64 x 64 diagonal blocks (k_inv_diag64)
 //   4. L^{-1} by recursive doubling: for block size s = 64, 128, ... every pair of
 //      neighbouring inverted blocks A, B with coupling C = L[B rows, A cols] gets
-//      its off-diagonal block -B^{-1} C A^{-1} from two batched GEMMs
+//      its off-diagonal block -B^{-1} C A^{-1} from two batched GEMMs.  Steps 3 and 4
+//      follow the factorisation block by block of 512 columns, so that with the
+//      look-ahead they run beside the later panels.
 //   5. U = J L^{-1} J, written as float with an explicit zero lower triangle.
 #include "tb_common.cuh"
 #include "tb_gemm.cuh"
@@ -76,8 +80,13 @@ __global__ void k_reverse_out(const double* __restrict__ Li, float* __restrict__
 // shared memory: the panel solve runs the same elimination on its rows (x_j = a_j / L_jj,
 // then a_c -= x_j / L_jj * col_j[c]), so neither L nor an inverse is stored in between.
 // Entries right of the diagonal go through the same updates and are never used.
+//
+// update_first: the previous panel's rank-64 update of these 64 columns has not been applied yet (the
+// trailing update after a panel leaves out the next panel's columns); the kernel applies it to the
+// diagonal block and to its own rows before it starts, from the previous panel's rows staged
+// k-major.  That keeps a GEMM launch per panel off the chain of dependent launches.
 enum { PLD = 66, PQ = 16, PANEL_THREADS = 256 };  // PLD: row pitch of the staged 64 x 64 tiles (doubles)
-static constexpr size_t PANEL_SMEM = (2 * 64 * PLD + 64 + 2 * PQ * 64) * sizeof(double);
+static constexpr size_t PANEL_SMEM = (4 * 64 * PLD + 64 + 2 * PQ * 64) * sizeof(double);
 
 __device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gsrc) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((unsigned)__cvta_generic_to_shared(smem_dst)), "l"(gsrc)
@@ -86,12 +95,14 @@ __device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gsrc) {
 
 __global__ void __launch_bounds__(PANEL_THREADS) k_chol_panel(double* __restrict__ A, double* __restrict__ Ldiag,
                                                               long long ldiag_batch, int* __restrict__ info, int dp,
-                                                              int k0, int d_fact) {
+                                                              int k0, int d_fact, int update_first) {
   extern __shared__ __align__(16) unsigned char panel_raw[];
   double* sA = reinterpret_cast<double*>(panel_raw);  // this CTA's 64 panel rows
   double* sC = sA + 64 * PLD;                         // the diagonal block, then its raw columns: sC[j * PLD + r]
   double* rsv = sC + 64 * PLD;                        // 1 / L_jj
   double* sY = rsv + 64;                              // multipliers of the panel solve, [2][16][64]
+  double* sPd = sY + 2 * PQ * 64;                     // previous panel, rows of the diagonal block: sPd[k * PLD + row]
+  double* sPr = sPd + 64 * PLD;                       // previous panel, this CTA's rows, same layout
   const int tid = threadIdx.x, r = tid & 63, q = tid >> 6, b = blockIdx.y;
   double* Ab = A + (long long)b * dp * dp;
   double* diag = Ab + (long long)k0 * dp + k0;
@@ -114,7 +125,25 @@ __global__ void __launch_bounds__(PANEL_THREADS) k_chol_panel(double* __restrict
       }
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
-    asm volatile("cp.async.wait_group 1;" ::: "memory");
+    if (update_first) {
+      const double* dprev = diag - FNB;
+      const double* pprev = pan - FNB;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int rr = 8 * i + rr0;
+        const double2 v = *reinterpret_cast<const double2*>(dprev + (long long)rr * dp + 2 * ch);
+        sPd[(2 * ch) * PLD + rr] = v.x;
+        sPd[(2 * ch + 1) * PLD + rr] = v.y;
+        if (has_rows) {
+          const double2 w = *reinterpret_cast<const double2*>(pprev + (long long)rr * dp + 2 * ch);
+          sPr[(2 * ch) * PLD + rr] = w.x;
+          sPr[(2 * ch + 1) * PLD + rr] = w.y;
+        }
+      }
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+    } else {
+      asm volatile("cp.async.wait_group 1;" ::: "memory");
+    }
   }
   __syncthreads();
   double a[PQ];
@@ -123,6 +152,34 @@ __global__ void __launch_bounds__(PANEL_THREADS) k_chol_panel(double* __restrict
     const double2 v = *reinterpret_cast<const double2*>(sC + r * PLD + q * PQ + i);
     a[i] = v.x;
     a[i + 1] = v.y;
+  }
+  if (update_first) {
+    // a[c] -= sum_k Pd[r][k] Pd[c][k], and the same for this CTA's rows against Pr[r][k]
+    double xr[PQ];
+#pragma unroll
+    for (int i = 0; i < PQ; i += 2) {
+      const double2 v = has_rows ? *reinterpret_cast<const double2*>(sA + r * PLD + q * PQ + i) : make_double2(0.0, 0.0);
+      xr[i] = v.x;
+      xr[i + 1] = v.y;
+    }
+#pragma unroll 2
+    for (int k = 0; k < FNB; ++k) {
+      const double pd = sPd[k * PLD + r];
+      const double pr = has_rows ? sPr[k * PLD + r] : 0.0;
+#pragma unroll
+      for (int i = 0; i < PQ; i += 2) {
+        const double2 c = *reinterpret_cast<const double2*>(sPd + k * PLD + q * PQ + i);
+        a[i] = fma(-pd, c.x, a[i]);
+        a[i + 1] = fma(-pd, c.y, a[i + 1]);
+        xr[i] = fma(-pr, c.x, xr[i]);
+        xr[i + 1] = fma(-pr, c.y, xr[i + 1]);
+      }
+    }
+    if (has_rows) {
+#pragma unroll
+      for (int i = 0; i < PQ; i += 2)
+        *reinterpret_cast<double2*>(sA + r * PLD + q * PQ + i) = make_double2(xr[i], xr[i + 1]);
+    }
   }
   __syncthreads();  // the block has been read: its storage now takes the columns
 #pragma unroll 1
@@ -214,10 +271,10 @@ __global__ void __launch_bounds__(PANEL_THREADS) k_chol_panel(double* __restrict
 // Inverse of every 64 x 64 diagonal block of L into the same block of Li (lower triangular):
 // forward substitution, one thread per column, the column in registers.
 __global__ void __launch_bounds__(64) k_inv_diag64(const double* __restrict__ Ldiag, long long ldiag_batch,
-                                                   int n_factored, double* __restrict__ Li, int dp) {
+                                                   int n_factored, double* __restrict__ Li, int dp, int blk0) {
   __shared__ double Ls[FNB][FNB + 1];
   __shared__ double rdiag[FNB];
-  const int blk = blockIdx.x, b = blockIdx.y, c = threadIdx.x;
+  const int blk = blk0 + blockIdx.x, b = blockIdx.y, c = threadIdx.x;
   const long long off = (long long)b * dp * dp + (long long)blk * FNB * (dp + 1);
   // blocks of the identity padding were never factored: their factor is the identity
   const double* src = Ldiag + (long long)b * ldiag_batch + (long long)blk * FNB * FNB;
@@ -247,10 +304,14 @@ __global__ void k_mask_strict_upper(const double* __restrict__ src, double* __re
   }
 }
 
+enum { INV_BLOCK = 512 };  // the inverse is completed block by block of this many columns (see factor_run)
+
 struct FactorWs {
   double *A, *Li, *tmp;
   int dp;
-  size_t tmp_per;  // doubles of tmp per matrix
+  size_t tmp_per;   // doubles of tmp per matrix
+  size_t low_off;   // products of the doubling levels inside one block of INV_BLOCK columns
+  size_t high_off;  // products of the levels above, one region per level (level s at high_off + sum of the lower s^2)
   size_t total;
 };
 
@@ -267,18 +328,32 @@ static FactorWs factor_ws(int n_batch, int d, void* ws) {
   const size_t n = (size_t)f.dp * f.dp;
   f.A = b.take<double>((size_t)n_batch * n);
   f.Li = b.take<double>((size_t)n_batch * n);
-  // tmp: the factored diagonal blocks during the Cholesky sweep (dp x 64 per matrix), then the
-  // intermediate products of the doubling steps (dp^2 / 4 per matrix)
-  f.tmp_per = (n / 4 > (size_t)f.dp * FNB) ? n / 4 : (size_t)f.dp * FNB;
+  // tmp per matrix: the factored diagonal blocks (dp x 64), then the intermediate products of the
+  // doubling steps.  The inverse proceeds while later panels are still being factored, and a product
+  // of a high level stays alive while lower levels run, so each gets a region of its own.
+  const size_t gdim = (f.dp < INV_BLOCK) ? (size_t)f.dp : (size_t)INV_BLOCK;
+  f.low_off = (size_t)f.dp * FNB;
+  f.high_off = f.low_off + gdim * gdim / 4;
+  f.tmp_per = f.high_off;
+  for (size_t sb = gdim; sb < (size_t)f.dp; sb <<= 1) f.tmp_per += sb * sb;
   f.tmp = b.take<double>((size_t)n_batch * f.tmp_per + 64);
   f.total = b.total();
   return f;
 }
 
 // Helper stream of the look-ahead (one per device, created on first use, kept until exit).
+// The panels with the update of their own 64 columns are the critical path: they get a stream of the
+// highest priority, so that their few CTAs are placed before the many tiles of a trailing update that
+// is still being dispatched.  The first products of the upper doubling levels are large, and nothing
+// needs them before the pair's second half has been factored and inverted: they get a stream of the
+// lowest priority of their own (one per level: a small product must not queue behind a large one of the
+// level above), so that the block-by-block part of the inverse does not wait for them needlessly.
 struct FactorSide {
-  cudaStream_t stream;
-  cudaEvent_t fork, panel, trail;
+  cudaStream_t crit;    // panels (each applies the previous panel's update to its own columns first)
+  cudaStream_t stream;  // trailing updates
+  cudaStream_t inv;     // the inverse of the blocks already factored
+  cudaStream_t inv2[8];  // first products of the doubling levels above one block, a stream per level
+  cudaEvent_t fork, panel, trail[2], block_done, inv_done, crit_done, half_done, first_done[8];
   bool ready;
 };
 
@@ -288,10 +363,24 @@ static FactorSide* factor_side() {
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
   FactorSide* s = &per_device[dev];
   if (!s->ready) {
-    if (cudaStreamCreateWithFlags(&s->stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+    int least = 0, greatest = 0;
+    if (cudaDeviceGetStreamPriorityRange(&least, &greatest) != cudaSuccess) return nullptr;
+    const int middle = (greatest < least) ? greatest + 1 : least;  // numerically lower = more urgent
+    if (cudaStreamCreateWithPriority(&s->crit, cudaStreamNonBlocking, greatest) != cudaSuccess) return nullptr;
+    if (cudaStreamCreateWithPriority(&s->stream, cudaStreamNonBlocking, middle) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&s->crit_done, cudaEventDisableTiming) != cudaSuccess) return nullptr;
     if (cudaEventCreateWithFlags(&s->fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
     if (cudaEventCreateWithFlags(&s->panel, cudaEventDisableTiming) != cudaSuccess) return nullptr;
-    if (cudaEventCreateWithFlags(&s->trail, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&s->trail[0], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&s->trail[1], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    if (cudaStreamCreateWithPriority(&s->inv, cudaStreamNonBlocking, middle) != cudaSuccess) return nullptr;
+    for (int i = 0; i < 8; ++i)
+      if (cudaStreamCreateWithPriority(&s->inv2[i], cudaStreamNonBlocking, least) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&s->half_done, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    for (int i = 0; i < 8; ++i)
+      if (cudaEventCreateWithFlags(&s->first_done[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&s->block_done, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&s->inv_done, cudaEventDisableTiming) != cudaSuccess) return nullptr;
     s->ready = true;
   }
   return s;
@@ -314,11 +403,11 @@ extern "C" tb_status tb_factor(const float* H, int n_batch, int d, float* U, flo
   return factor_run(H, n_batch, d, U, Hinv, info, ws, ws_bytes, stream, true);
 }
 
-// lookahead: the trailing update of a panel is split in two.  The part that the next panel needs (its
-// 64 columns) stays on the caller's stream, followed at once by the next panel; the rest runs on a
-// helper stream beside them.  Every entry still receives its updates in the same order, so the result
-// is the same bit for bit.  Without it (callers that must not create a stream) everything runs on the
-// caller's stream.
+// lookahead: the panels run on a stream of high priority, the trailing updates (which leave out the
+// next panel's columns: that panel applies its share itself) on a second stream beside the next panel,
+// the inverse of the blocks already factored on a third.  Every entry still receives its updates in
+// the same order and every product is the same launch, so the result is the same bit for bit.  Without
+// it (callers that must not create a stream) everything runs on the caller's stream.
 tb_status tb::factor_run(const float* H, int n_batch, int d, float* U, float* Hinv, int* info, void* ws,
                          size_t ws_bytes, void* stream, bool lookahead) {
   if (!H || !U || !info || n_batch <= 0 || n_batch > 65535 || d <= 0) return TB_ERR_INVALID_ARG;
@@ -344,118 +433,199 @@ tb_status tb::factor_run(const float* H, int n_batch, int d, float* U, float* Hi
     if (!side) return TB_ERR_CUDA;
     TB_CUDA_CHECK(cudaEventRecord(side->fork, st));
     TB_CUDA_CHECK(cudaStreamWaitEvent(side->stream, side->fork, 0));
+    TB_CUDA_CHECK(cudaStreamWaitEvent(side->crit, side->fork, 0));
   }
-  bool trail_pending = false;
+  // L^{-1} block by block of G columns.  Block j can be inverted as soon as its last panel is factored:
+  // its 64 x 64 diagonal inverses, the doubling levels inside the block, then every level above whose
+  // pair this block completes (second product), and the first product of the one pair whose first half
+  // it completes (that product needs only columns already final).  With the look-ahead all of this runs
+  // on a stream of its own beside the later panels, and little of the inverse is left after the last
+  // panel; without it the same launches follow the panels on the caller's stream.  Every product is
+  // the same launch either way, so the result is the same bit for bit.
+  const int G = (dp < INV_BLOCK) ? dp : INV_BLOCK;
+  const int n_inv_blocks = dp / G, n_panels = d_fact / FNB;
+  cudaStream_t inv_st = side ? side->inv : st;
+  cudaStream_t cs = side ? side->crit : st;  // stream of the panels
+  // first product of a pair at level sblk: T = C A^{-1}, C = L[s:2s, 0:s], A^{-1} = Li[0:s, 0:s] (lower triangular)
+  // Launched in pieces of at most 768 rows (96 tiles at 2048 columns): the tiles of the upper levels
+  // run for hundreds of microseconds, and a launch that fills every SM with them would keep the panels
+  // waiting.  A piece is the same set of tiles, so nothing changes in the result.
+  auto pair_first = [&](int sblk, long long off, long long pair_stride, int batch, double* tmp, long long tmp_stride,
+                        cudaStream_t stream_first) -> tb_status {
+    GemmP g = gemm_params();
+    g.A = f.A + off + (long long)sblk * dp;
+    g.a_m = dp;
+    g.a_k = 1;
+    g.a_batch = pair_stride;
+    g.B = f.Li + off;
+    g.b_k = dp;
+    g.b_n = 1;
+    g.b_batch = pair_stride;
+    g.C = tmp;
+    g.ldc = sblk;
+    g.c_batch = tmp_stride;
+    g.M = sblk;
+    g.N = sblk;
+    g.K = sblk;
+    g.n_batch = batch;
+    g.btrim = 2;
+    g.flags = GEMM_HEAVY_N_FIRST;
+    const int piece = (sblk > 1024) ? 768 : sblk;
+    for (int m0 = 0; m0 < sblk; m0 += piece) {
+      GemmP gp = g;
+      gp.A = g.A + (long long)m0 * dp;
+      gp.C = tmp + (long long)m0 * sblk;
+      gp.M = (sblk - m0 < piece) ? sblk - m0 : piece;
+      TB_TRY((gemm_launch<double, double, double, double, false, true>(gp, stream_first)));
+    }
+    return TB_OK;
+  };
+  // second product: Li[s:2s, 0:s] = -B^{-1} T, B^{-1} = Li[s:2s, s:2s] (lower triangular)
+  auto pair_second = [&](int sblk, long long off, long long pair_stride, int batch, double* tmp,
+                         long long tmp_stride) -> tb_status {
+    GemmP h = gemm_params();
+    h.A = f.Li + off + (long long)sblk * (dp + 1);
+    h.a_m = dp;
+    h.a_k = 1;
+    h.a_batch = pair_stride;
+    h.B = tmp;
+    h.b_k = sblk;
+    h.b_n = 1;
+    h.b_batch = tmp_stride;
+    h.C = f.Li + off + (long long)sblk * dp;
+    h.ldc = dp;
+    h.c_batch = pair_stride;
+    h.M = sblk;
+    h.N = sblk;
+    h.K = sblk;
+    h.n_batch = batch;
+    h.alpha = -1.0;
+    h.atrim = 1;
+    h.flags = GEMM_HEAVY_M_LAST;
+    return gemm_launch<double, double, double, double, false, true>(h, inv_st);
+  };
+  auto high_tmp = [&](int sblk) {  // region of the level-sblk product (first matrix of the batch)
+    size_t o = f.high_off;
+    for (size_t sb = (size_t)G; sb < (size_t)sblk; sb <<= 1) o += sb * sb;
+    return f.tmp + o;
+  };
+  auto invert_block = [&](int j) -> tb_status {
+    const long long boff = (long long)j * G * (dp + 1);
+    k_inv_diag64<<<dim3(G / FNB, n_batch), 64, 0, inv_st>>>(f.tmp, (long long)f.tmp_per, n_panels, f.Li, dp,
+                                                             j * (G / FNB));
+    TB_LAUNCH_CHECK();
+    for (int sblk = FNB; sblk < G; sblk <<= 1) {
+      const int pairs = G / (2 * sblk);
+      // one batched launch covers all pairs of one matrix's block, or (a single pair) all matrices
+      const int outer = (pairs == 1) ? 1 : n_batch;
+      for (int mb = 0; mb < outer; ++mb) {
+        const long long off = (long long)mb * pp + boff;
+        const long long pair_stride = (pairs == 1) ? pp : (long long)2 * sblk * (dp + 1);
+        const int batch = (pairs == 1) ? n_batch : pairs;
+        double* tmp = f.tmp + (size_t)mb * f.tmp_per + f.low_off;
+        const long long tmp_stride = (pairs == 1) ? (long long)f.tmp_per : (long long)sblk * sblk;
+        TB_TRY(pair_first(sblk, off, pair_stride, batch, tmp, tmp_stride, inv_st));
+        TB_TRY(pair_second(sblk, off, pair_stride, batch, tmp, tmp_stride));
+      }
+    }
+    int level = 0;
+    for (int sblk = G; sblk < dp; sblk <<= 1, ++level) {
+      const int mblk = sblk / G;  // blocks per half of a pair at this level
+      if ((j + 1) % mblk) break;
+      const int halves = (j + 1) / mblk;
+      if (halves & 1) {  // block j completes the first half of its pair
+        if (side) {
+          TB_CUDA_CHECK(cudaEventRecord(side->half_done, side->inv));
+          TB_CUDA_CHECK(cudaStreamWaitEvent(side->inv2[level & 7], side->half_done, 0));
+        }
+        TB_TRY(pair_first(sblk, (long long)(j + 1 - mblk) * G * (dp + 1), pp, n_batch, high_tmp(sblk),
+                          (long long)f.tmp_per, side ? side->inv2[level & 7] : inv_st));
+        if (side) TB_CUDA_CHECK(cudaEventRecord(side->first_done[level & 7], side->inv2[level & 7]));
+        break;
+      }
+      if (side) TB_CUDA_CHECK(cudaStreamWaitEvent(side->inv, side->first_done[level & 7], 0));
+      TB_TRY(pair_second(sblk, (long long)(j + 1 - 2 * mblk) * G * (dp + 1), pp, n_batch, high_tmp(sblk),
+                         (long long)f.tmp_per));
+    }
+    return TB_OK;
+  };
+  int next_inv_block = 0;
+
+  // Panel k applies the update of panel k-1 to its own 64 columns itself; the trailing update after
+  // panel k covers the columns from panel k+2 on.  With the look-ahead it runs on the helper stream
+  // beside panel k+1, and panel k+2 waits for it (two events in turn).
+  bool trail_set[2] = {false, false};
   for (int k0 = 0; k0 < d_fact; k0 += FNB) {
     const int r0 = k0 + FNB, m = d_fact - r0;
     const int xt = (m > 0) ? m / FNB : 1;
-    k_chol_panel<<<dim3(xt, n_batch), PANEL_THREADS, PANEL_SMEM, st>>>(f.A, f.tmp, (long long)f.tmp_per, info, dp, k0,
-                                                                       d_fact);
+    const int pi = k0 / FNB;
+    if (side && trail_set[pi & 1]) TB_CUDA_CHECK(cudaStreamWaitEvent(cs, side->trail[pi & 1], 0));
+    k_chol_panel<<<dim3(xt, n_batch), PANEL_THREADS, PANEL_SMEM, cs>>>(f.A, f.tmp, (long long)f.tmp_per, info, dp, k0,
+                                                                       d_fact, k0 > 0 ? 1 : 0);
     TB_LAUNCH_CHECK();
+    if (side) {
+      // blocks whose last factored panel this was (the identity padding needs no panel)
+      bool waited = false;
+      while (next_inv_block < n_inv_blocks) {
+        int last = (next_inv_block + 1) * (G / FNB) - 1;
+        if (last > n_panels - 1) last = n_panels - 1;
+        if (last != pi) break;
+        if (!waited) {
+          TB_CUDA_CHECK(cudaEventRecord(side->block_done, cs));
+          TB_CUDA_CHECK(cudaStreamWaitEvent(side->inv, side->block_done, 0));
+          waited = true;
+        }
+        TB_TRY(invert_block(next_inv_block));
+        ++next_inv_block;
+      }
+    }
     if (m <= 0) break;
-    GemmP s = gemm_params();  // trailing -= panel panel^T, tiles on or below the diagonal
-    s.A = f.A + (long long)r0 * dp + k0;
-    s.a_m = dp;
-    s.a_k = 1;
-    s.a_batch = pp;
-    s.B = f.A + (long long)r0 * dp + k0;  // B(k, n) = panel[n][k]
-    s.b_k = 1;
-    s.b_n = dp;
-    s.b_batch = pp;
-    s.C = f.A + (long long)r0 * dp + r0;
-    s.ldc = dp;
-    s.c_batch = pp;
-    s.M = m;
-    s.N = m;
-    s.K = FNB;
-    s.n_batch = n_batch;
-    s.alpha = -1.0;
-    s.beta = 1.0;
-    s.flags = GEMM_LOWER_TILES;
+    trail_set[pi & 1] = false;
+    if (m <= FNB) continue;  // only the next panel's columns are left, and that panel updates them itself
+    GemmP t = gemm_params();  // trailing -= panel panel^T from column r0 + 64 on, tiles on or below the diagonal
+    t.A = f.A + (long long)(r0 + FNB) * dp + k0;
+    t.a_m = dp;
+    t.a_k = 1;
+    t.a_batch = pp;
+    t.B = t.A;  // B(k, n) = panel[n][k]
+    t.b_k = 1;
+    t.b_n = dp;
+    t.b_batch = pp;
+    t.C = f.A + (long long)(r0 + FNB) * dp + (r0 + FNB);
+    t.ldc = dp;
+    t.c_batch = pp;
+    t.M = m - FNB;
+    t.N = m - FNB;
+    t.K = FNB;
+    t.n_batch = n_batch;
+    t.alpha = -1.0;
+    t.beta = 1.0;
+    t.flags = GEMM_LOWER_TILES;
     if (!side) {
-      TB_TRY((gemm_launch<double, double, double, double, false, false>(s, st)));
+      TB_TRY((gemm_launch<double, double, double, double, false, false>(t, st)));
       continue;
     }
-    // the rest of the trailing matrix (columns from r0 + 64 on, hence rows from r0 + 64 on): helper stream
-    if (m > FNB) {
-      TB_CUDA_CHECK(cudaEventRecord(side->panel, st));
-      TB_CUDA_CHECK(cudaStreamWaitEvent(side->stream, side->panel, 0));
-      GemmP t = s;
-      t.A = f.A + (long long)(r0 + FNB) * dp + k0;
-      t.B = t.A;
-      t.C = f.A + (long long)(r0 + FNB) * dp + (r0 + FNB);
-      t.M = m - FNB;
-      t.N = m - FNB;
-      TB_TRY((gemm_launch<double, double, double, double, false, false>(t, side->stream)));
-    }
-    // the next panel's 64 columns: caller's stream, after the helper's update of the previous panel,
-    // which touched the same entries
-    if (trail_pending) TB_CUDA_CHECK(cudaStreamWaitEvent(st, side->trail, 0));
-    if (m > FNB) {
-      TB_CUDA_CHECK(cudaEventRecord(side->trail, side->stream));
-      trail_pending = true;
-    } else {
-      trail_pending = false;
-    }
-    s.N = FNB;
-    s.flags = 0;
-    TB_TRY((gemm_launch<double, double, double, double, false, false>(s, st)));
+    TB_CUDA_CHECK(cudaEventRecord(side->panel, cs));
+    TB_CUDA_CHECK(cudaStreamWaitEvent(side->stream, side->panel, 0));
+    TB_TRY((gemm_launch<double, double, double, double, false, false>(t, side->stream)));
+    TB_CUDA_CHECK(cudaEventRecord(side->trail[pi & 1], side->stream));
+    trail_set[pi & 1] = true;
   }
-  if (side && trail_pending) TB_CUDA_CHECK(cudaStreamWaitEvent(st, side->trail, 0));
+  if (side) {
+    for (int i = 0; i < 2; ++i)
+      if (trail_set[i]) TB_CUDA_CHECK(cudaStreamWaitEvent(st, side->trail[i], 0));
+    TB_CUDA_CHECK(cudaEventRecord(side->crit_done, side->crit));
+    TB_CUDA_CHECK(cudaStreamWaitEvent(st, side->crit_done, 0));
+  }
 
-  // L^{-1}: diagonal blocks, then recursive doubling
-  k_inv_diag64<<<dim3(dp / FNB, n_batch), 64, 0, st>>>(f.tmp, (long long)f.tmp_per, d_fact / FNB, f.Li, dp);
-  TB_LAUNCH_CHECK();
-  for (int sblk = FNB; sblk < dp; sblk <<= 1) {
-    const int pairs = dp / (2 * sblk);
-    // one batched launch covers all pairs of one matrix, or (a single pair per matrix) all matrices
-    const int outer = (pairs == 1) ? 1 : n_batch;
-    for (int mb = 0; mb < outer; ++mb) {
-      const long long moff = (long long)mb * pp;
-      const long long pair_stride = (pairs == 1) ? pp : (long long)2 * sblk * (dp + 1);
-      const int batch = (pairs == 1) ? n_batch : pairs;
-      double* tmp = f.tmp + (long long)mb * (long long)f.tmp_per;
-      const long long tmp_stride = (pairs == 1) ? (long long)f.tmp_per : (long long)sblk * sblk;
-      GemmP g = gemm_params();  // T = C A^{-1}: C = L[s:2s, 0:s], A^{-1} = Li[0:s, 0:s] (lower triangular)
-      g.A = f.A + moff + (long long)sblk * dp;
-      g.a_m = dp;
-      g.a_k = 1;
-      g.a_batch = pair_stride;
-      g.B = f.Li + moff;
-      g.b_k = dp;
-      g.b_n = 1;
-      g.b_batch = pair_stride;
-      g.C = tmp;
-      g.ldc = sblk;
-      g.c_batch = tmp_stride;
-      g.M = sblk;
-      g.N = sblk;
-      g.K = sblk;
-      g.n_batch = batch;
-      g.btrim = 2;
-      g.flags = GEMM_HEAVY_N_FIRST;
-      TB_TRY((gemm_launch<double, double, double, double, false, true>(g, st)));
-      GemmP h = gemm_params();  // Li[s:2s, 0:s] = -B^{-1} T, B^{-1} = Li[s:2s, s:2s] (lower triangular)
-      h.A = f.Li + moff + (long long)sblk * (dp + 1);
-      h.a_m = dp;
-      h.a_k = 1;
-      h.a_batch = pair_stride;
-      h.B = tmp;
-      h.b_k = sblk;
-      h.b_n = 1;
-      h.b_batch = tmp_stride;
-      h.C = f.Li + moff + (long long)sblk * dp;
-      h.ldc = dp;
-      h.c_batch = pair_stride;
-      h.M = sblk;
-      h.N = sblk;
-      h.K = sblk;
-      h.n_batch = batch;
-      h.alpha = -1.0;
-      h.atrim = 1;
-      h.flags = GEMM_HEAVY_M_LAST;
-      TB_TRY((gemm_launch<double, double, double, double, false, true>(h, st)));
-    }
+  // what is left of the inverse (all of it without the look-ahead)
+  while (next_inv_block < n_inv_blocks) {
+    TB_TRY(invert_block(next_inv_block));
+    ++next_inv_block;
+  }
+  if (side) {
+    TB_CUDA_CHECK(cudaEventRecord(side->inv_done, side->inv));
+    TB_CUDA_CHECK(cudaStreamWaitEvent(st, side->inv_done, 0));
   }
   int eo = (int)(((long long)d * d + 255) / 256);
   if (eo > 148 * 8) eo = 148 * 8;
