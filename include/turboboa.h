@@ -146,9 +146,13 @@ tb_status tb_build_hout(float* H_out, const float* G, const float* Hsum, int n_h
  * info (device, [n_batch] int): 0, or the 1-based index (counted in the
  * elimination order, which runs from the last row to the first) of the first
  * pivot that was not positive; U of that matrix is then meaningless.
- * For matrices of 1024 columns or more part of the work runs on a helper
- * stream of the library (one per device, created at the first such call and
- * kept until exit), forked from and joined back into `stream` by events. */
+ * For matrices of 1024 columns or more the work is spread over helper streams
+ * of the library (per device, created at the first such call and kept until
+ * exit; the chain of panel factorisations on one of the highest priority,
+ * trailing updates and the inverse of the finished blocks beside it), forked
+ * from and joined back into `stream` by events.  All calls on a device share
+ * these streams and events: do not factor such sizes on one device from two
+ * host threads at once. */
 size_t tb_factor_workspace(int n_batch, int d);
 tb_status tb_factor(const float* H, int n_batch, int d, float* U, float* Hinv, int* info,
                     void* ws, size_t ws_bytes, void* stream);

@@ -310,7 +310,7 @@ struct FactorWs {
   double *A, *Li, *tmp;
   int dp;
   size_t tmp_per;   // doubles of tmp per matrix
-  size_t low_off;   // products of the doubling levels inside one block of INV_BLOCK columns
+  size_t low_off;   // products of the doubling levels inside one block of INV_BLOCK columns (two regions in turn)
   size_t high_off;  // products of the levels above, one region per level (level s at high_off + sum of the lower s^2)
   size_t total;
 };
@@ -333,7 +333,7 @@ static FactorWs factor_ws(int n_batch, int d, void* ws) {
   // of a high level stays alive while lower levels run, so each gets a region of its own.
   const size_t gdim = (f.dp < INV_BLOCK) ? (size_t)f.dp : (size_t)INV_BLOCK;
   f.low_off = (size_t)f.dp * FNB;
-  f.high_off = f.low_off + gdim * gdim / 4;
+  f.high_off = f.low_off + 2 * (gdim * gdim / 4);  // two regions: neighbouring blocks are inverted side by side
   f.tmp_per = f.high_off;
   for (size_t sb = gdim; sb < (size_t)f.dp; sb <<= 1) f.tmp_per += sb * sb;
   f.tmp = b.take<double>((size_t)n_batch * f.tmp_per + 64);
@@ -351,9 +351,10 @@ static FactorWs factor_ws(int n_batch, int d, void* ws) {
 struct FactorSide {
   cudaStream_t crit;    // panels (each applies the previous panel's update to its own columns first)
   cudaStream_t stream;  // trailing updates
-  cudaStream_t inv;     // the inverse of the blocks already factored
+  cudaStream_t inv;     // the inverse above the blocks: second products of the upper levels
+  cudaStream_t low[2];  // the inverse inside a block of 512 columns, blocks in turn
   cudaStream_t inv2[8];  // first products of the doubling levels above one block, a stream per level
-  cudaEvent_t fork, panel, trail[2], block_done, inv_done, crit_done, half_done, first_done[8];
+  cudaEvent_t fork, panel, trail[2], block_done, inv_done, crit_done, half_done, first_done[8], low_done[2];
   bool ready;
 };
 
@@ -377,6 +378,10 @@ static FactorSide* factor_side() {
     for (int i = 0; i < 8; ++i)
       if (cudaStreamCreateWithPriority(&s->inv2[i], cudaStreamNonBlocking, least) != cudaSuccess) return nullptr;
     if (cudaEventCreateWithFlags(&s->half_done, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    for (int i = 0; i < 2; ++i) {
+      if (cudaStreamCreateWithPriority(&s->low[i], cudaStreamNonBlocking, middle) != cudaSuccess) return nullptr;
+      if (cudaEventCreateWithFlags(&s->low_done[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    }
     for (int i = 0; i < 8; ++i)
       if (cudaEventCreateWithFlags(&s->first_done[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
     if (cudaEventCreateWithFlags(&s->block_done, cudaEventDisableTiming) != cudaSuccess) return nullptr;
@@ -481,8 +486,8 @@ tb_status tb::factor_run(const float* H, int n_batch, int d, float* U, float* Hi
     return TB_OK;
   };
   // second product: Li[s:2s, 0:s] = -B^{-1} T, B^{-1} = Li[s:2s, s:2s] (lower triangular)
-  auto pair_second = [&](int sblk, long long off, long long pair_stride, int batch, double* tmp,
-                         long long tmp_stride) -> tb_status {
+  auto pair_second = [&](int sblk, long long off, long long pair_stride, int batch, double* tmp, long long tmp_stride,
+                         cudaStream_t stream_second) -> tb_status {
     GemmP h = gemm_params();
     h.A = f.Li + off + (long long)sblk * (dp + 1);
     h.a_m = dp;
@@ -502,7 +507,7 @@ tb_status tb::factor_run(const float* H, int n_batch, int d, float* U, float* Hi
     h.alpha = -1.0;
     h.atrim = 1;
     h.flags = GEMM_HEAVY_M_LAST;
-    return gemm_launch<double, double, double, double, false, true>(h, inv_st);
+    return gemm_launch<double, double, double, double, false, true>(h, stream_second);
   };
   auto high_tmp = [&](int sblk) {  // region of the level-sblk product (first matrix of the batch)
     size_t o = f.high_off;
@@ -511,7 +516,12 @@ tb_status tb::factor_run(const float* H, int n_batch, int d, float* U, float* Hi
   };
   auto invert_block = [&](int j) -> tb_status {
     const long long boff = (long long)j * G * (dp + 1);
-    k_inv_diag64<<<dim3(G / FNB, n_batch), 64, 0, inv_st>>>(f.tmp, (long long)f.tmp_per, n_panels, f.Li, dp,
+    // inside the block: a stream per block parity, so that a block does not wait for its neighbour's
+    // upper levels; the caller has just recorded block_done
+    cudaStream_t low_st = side ? side->low[j & 1] : inv_st;
+    const size_t low_region = f.low_off + (size_t)(j & 1) * ((size_t)G * G / 4);
+    if (side) TB_CUDA_CHECK(cudaStreamWaitEvent(low_st, side->block_done, 0));
+    k_inv_diag64<<<dim3(G / FNB, n_batch), 64, 0, low_st>>>(f.tmp, (long long)f.tmp_per, n_panels, f.Li, dp,
                                                              j * (G / FNB));
     TB_LAUNCH_CHECK();
     for (int sblk = FNB; sblk < G; sblk <<= 1) {
@@ -522,11 +532,15 @@ tb_status tb::factor_run(const float* H, int n_batch, int d, float* U, float* Hi
         const long long off = (long long)mb * pp + boff;
         const long long pair_stride = (pairs == 1) ? pp : (long long)2 * sblk * (dp + 1);
         const int batch = (pairs == 1) ? n_batch : pairs;
-        double* tmp = f.tmp + (size_t)mb * f.tmp_per + f.low_off;
+        double* tmp = f.tmp + (size_t)mb * f.tmp_per + low_region;
         const long long tmp_stride = (pairs == 1) ? (long long)f.tmp_per : (long long)sblk * sblk;
-        TB_TRY(pair_first(sblk, off, pair_stride, batch, tmp, tmp_stride, inv_st));
-        TB_TRY(pair_second(sblk, off, pair_stride, batch, tmp, tmp_stride));
+        TB_TRY(pair_first(sblk, off, pair_stride, batch, tmp, tmp_stride, low_st));
+        TB_TRY(pair_second(sblk, off, pair_stride, batch, tmp, tmp_stride, low_st));
       }
+    }
+    if (side) {
+      TB_CUDA_CHECK(cudaEventRecord(side->low_done[j & 1], low_st));
+      TB_CUDA_CHECK(cudaStreamWaitEvent(side->inv, side->low_done[j & 1], 0));
     }
     int level = 0;
     for (int sblk = G; sblk < dp; sblk <<= 1, ++level) {
@@ -545,7 +559,7 @@ tb_status tb::factor_run(const float* H, int n_batch, int d, float* U, float* Hi
       }
       if (side) TB_CUDA_CHECK(cudaStreamWaitEvent(side->inv, side->first_done[level & 7], 0));
       TB_TRY(pair_second(sblk, (long long)(j + 1 - 2 * mblk) * G * (dp + 1), pp, n_batch, high_tmp(sblk),
-                         (long long)f.tmp_per));
+                         (long long)f.tmp_per, inv_st));
     }
     return TB_OK;
   };
