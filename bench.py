@@ -128,11 +128,20 @@ def count_launches(cfg, proj, n_tok: int, with_loss=True, cd_iters=1) -> int:
     g = cfg.out_block if has_hout else dh
     S = dh // g
 
-    def factor(dd):
-        blocks = -(-dd // 64)
-        dp_blocks = 1 << max(0, (blocks - 1).bit_length())
-        levels = dp_blocks.bit_length() - 1
-        return 1 + blocks + (blocks - 1) + 1 + 2 * levels + 1   # reverse, panels, trailing, block inverses, doubling, reverse
+    def factor(dd, n_batch=1):
+        panels = -(-dd // 64)
+        dp = 64 << max(0, (panels - 1).bit_length())
+        G = min(512, dp)                                 # the inverse goes block by block of G columns
+        n = 1 + panels + max(0, panels - 2)              # reverse, panels, trailing updates (from the panel after the next on)
+        s = 64
+        while s < G:                                     # inside a block: both products of every level
+            n += (dp // G) * 2 * (1 if G // (2 * s) == 1 else n_batch)
+            s *= 2
+        n += dp // G                                     # 64 x 64 diagonal inverses, one launch per block
+        while s < dp:                                    # above: first product (in row pieces when large), second product
+            n += (dp // (2 * s)) * ((-(-s // 768) if s > 1024 else 1) + 1)
+            s *= 2
+        return n + 1                                     # reverse
 
     d_out = proj.d_out
     seg = cfg.quant_group or d
@@ -141,7 +150,7 @@ def count_launches(cfg, proj, n_tok: int, with_loss=True, cd_iters=1) -> int:
     if has_hout:
         hout_tensor = d_out % 8 == 0 and d % 32 == 0    # G Hsum as a split-bf16 tensor-core product
         n += (3 if hout_tensor else 1) + 2              # (two splits +) product, per-head Gram, combine
-    n += factor(d) + (factor(dh) if has_hout else 0)
+    n += factor(d) + (factor(dh, H) if has_hout else 0)
     n += 1 + (1 if has_hout and S > 1 else 0)           # widen, compensation matrices
     n += (S if cfg.adaptive else 1) + S                 # grid search, one sweep launch per step
     n += 2 * (S - 1) if has_hout else 0                 # residual + compensation GEMM

@@ -452,9 +452,10 @@ tb_status tb::factor_run(const float* H, int n_batch, int d, float* U, float* Hi
   cudaStream_t inv_st = side ? side->inv : st;
   cudaStream_t cs = side ? side->crit : st;  // stream of the panels
   // first product of a pair at level sblk: T = C A^{-1}, C = L[s:2s, 0:s], A^{-1} = Li[0:s, 0:s] (lower triangular)
-  // Launched in pieces of at most 768 rows (96 tiles at 2048 columns): the tiles of the upper levels
+  // Launched in pieces of at most 768 columns (96 tiles at 2048 rows): the tiles of the upper levels
   // run for hundreds of microseconds, and a launch that fills every SM with them would keep the panels
-  // waiting.  A piece is the same set of tiles, so nothing changes in the result.
+  // waiting.  The first columns meet the longest part of the triangle, so the pieces get shorter.  A
+  // piece is the same set of tiles, so nothing changes in the result.
   auto pair_first = [&](int sblk, long long off, long long pair_stride, int batch, double* tmp, long long tmp_stride,
                         cudaStream_t stream_first) -> tb_status {
     GemmP g = gemm_params();
@@ -476,11 +477,12 @@ tb_status tb::factor_run(const float* H, int n_batch, int d, float* U, float* Hi
     g.btrim = 2;
     g.flags = GEMM_HEAVY_N_FIRST;
     const int piece = (sblk > 1024) ? 768 : sblk;
-    for (int m0 = 0; m0 < sblk; m0 += piece) {
+    for (int n0 = 0; n0 < sblk; n0 += piece) {
       GemmP gp = g;
-      gp.A = g.A + (long long)m0 * dp;
-      gp.C = tmp + (long long)m0 * sblk;
-      gp.M = (sblk - m0 < piece) ? sblk - m0 : piece;
+      gp.B = g.B + n0;  // B(k, n0 + n), zero for k < n0 + n
+      gp.boff = n0;
+      gp.C = tmp + n0;
+      gp.N = (sblk - n0 < piece) ? sblk - n0 : piece;
       TB_TRY((gemm_launch<double, double, double, double, false, true>(gp, stream_first)));
     }
     return TB_OK;
