@@ -479,7 +479,7 @@ tb_status tb::factor_run(const float* H, int n_batch, int d, float* U, float* Hi
     const int piece = (sblk > 1024) ? 768 : sblk;
     for (int n0 = 0; n0 < sblk; n0 += piece) {
       GemmP gp = g;
-      gp.B = g.B + n0;  // B(k, n0 + n), zero for k < n0 + n
+      gp.B = f.Li + off + n0;  // B(k, n0 + n), zero for k < n0 + n
       gp.boff = n0;
       gp.C = tmp + n0;
       gp.N = (sblk - n0 < piece) ? sblk - n0 : piece;

@@ -98,10 +98,15 @@ def test_build_hout(n_heads, g_heads, with_sum):
     assert err <= 2e-6
 
 
-@pytest.mark.parametrize("n_batch,d,cond", [(3, 200, 1e3), (1, 256, 1e5), (2, 64, 1e2), (1, 520, 1e4), (5, 128, 1e3)])
+@pytest.mark.parametrize("n_batch,d,cond", [(3, 200, 1e3), (1, 256, 1e5), (2, 64, 1e2), (1, 520, 1e4), (5, 128, 1e3),
+                                            (2, 1024, 1e3), (1, 1100, 1e4), (1, 2100, 1e4), (1, 4096, 1e4)])
 def test_factor_matches_definition(n_batch, d, cond):
     """U = chol(H^-1)^T (Eq. 2).  The GPU takes the reversed-Cholesky route in
-    double and rounds once to float; the oracle inverts and factors."""
+    double and rounds once to float; the oracle inverts and factors.  From 1024 columns on
+    the panels, the trailing updates and the inverse of the finished blocks run on streams
+    of their own: two matrices at once, a size whose last blocks are partly and wholly
+    padding (1100 in 2048), one that reaches the level whose first product is launched
+    in pieces (2100 in 4096), and the benchmark's own size."""
     import torch
     import paper_2602_04929_b200 as tb
     H = np.stack([tb_inputs.spd_matrix(11 + b, d, cond=cond) for b in range(n_batch)])
