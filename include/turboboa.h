@@ -186,9 +186,7 @@ tb_status tb_factor_static(const float* H, int n_batch, int d, float* U, int* in
  *   P = ((R U^T) masked to its strictly upper triangle) U   (Algorithm 2, line 2)
  *   C = R U^T U = R H_in^{-1}                               (Proposition 3.2)
  * All [n_batch][d][d] float.  U must have a zero strictly-lower triangle.
- * For d a multiple of 32 the three products run on the tensor cores through
- * exact bf16 splits with double sums of 128-step runs (relative error of P and
- * C about 1e-6, they are float outputs); otherwise in double. */
+ * The three products run in double; P and C are rounded to float once. */
 size_t tb_prepare_correction_workspace(int n_batch, int d);
 tb_status tb_prepare_correction(const float* R, const float* U_in, int n_batch, int d, float* P,
                                 float* C, void* ws, size_t ws_bytes, void* stream);

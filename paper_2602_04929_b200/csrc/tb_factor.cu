@@ -30,13 +30,6 @@
 
 namespace tb {
 
-// split-bf16 tensor-core product (tb_gemm_tc.cu): C (+)= A B in double from operands in three bf16 pieces
-tb_status gemm_split_presplit(double* C, long long ldc, const __nv_bfloat16* AT, const __nv_bfloat16* Bp, long long M,
-                              int N, int K, bool accumulate, cudaStream_t st, int hunits = 1);
-tb_status split3_transpose(const double* A, __nv_bfloat16* AT, long long M, int K, cudaStream_t st);
-tb_status split3_transpose(const float* A, __nv_bfloat16* AT, long long M, int K, cudaStream_t st);
-tb_status split3(const float* B, __nv_bfloat16* Bp, long long n, cudaStream_t st);
-
 enum { FNB = 64 };
 
 // A (dp x dp) <- J H J in the leading d x d block, identity elsewhere
@@ -674,30 +667,15 @@ tb_status tb::factor_run(const float* H, int n_batch, int d, float* U, float* Hi
   return TB_OK;
 }
 
-// P and C are rounded to float on output and enter the loop as float inputs, so their three products may
-// run on the tensor cores through exact bf16 splits (relative error of a few 1e-7) where the shapes fit.
-static bool correction_on_tensor(int d) { return d % 32 == 0; }
-
+// P and C: three products on the FP64 engine.  (Products from bf16 splits on the tensor cores were 3x
+// faster, but R U^T U cancels heavily at large widths: their error, a few 1e-7 of sum |a||b|, came to
+// 1.5e-5 of the result at 4096 columns.)
 extern "C" size_t tb_prepare_correction_workspace(int n_batch, int d) {
   if (n_batch <= 0 || d <= 0) return 0;
   Bump b(nullptr);
   b.take<double>((size_t)d * d);
   b.take<double>((size_t)d * d);
-  if (correction_on_tensor(d)) {
-    b.take<__nv_bfloat16>((size_t)3 * d * d);  // left operand, transposed, in three pieces
-    b.take<__nv_bfloat16>((size_t)3 * d * d);  // right operand in three pieces
-  }
   return b.total();
-}
-
-// dst = (float)src, or its strictly upper part (zero elsewhere)
-__global__ void k_to_float(const double* __restrict__ src, float* __restrict__ dst, int d, int strict_upper) {
-  const long long n = (long long)d * d;
-  for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < n;
-       idx += (long long)gridDim.x * blockDim.x) {
-    const int i = (int)(idx / d), j = (int)(idx % d);
-    dst[idx] = (!strict_upper || j > i) ? (float)src[idx] : 0.0f;
-  }
 }
 
 extern "C" tb_status tb_prepare_correction(const float* R, const float* U_in, int n_batch, int d,
@@ -713,32 +691,6 @@ extern "C" tb_status tb_prepare_correction(const float* R, const float* U_in, in
   const long long dd = (long long)d * d;
   int eb = (int)((dd + 255) / 256);
   if (eb > 148 * 8) eb = 148 * 8;
-  if (correction_on_tensor(d)) {
-    __nv_bfloat16* AT = b.take<__nv_bfloat16>((size_t)3 * d * d);
-    __nv_bfloat16* Bp = b.take<__nv_bfloat16>((size_t)3 * d * d);
-    for (int i = 0; i < n_batch; ++i) {
-      const float* Rb = R + i * dd;
-      const float* Ub = U_in + i * dd;
-      // T1 = R U^T: the right operand U^T, [k][n] = U[n][k], is U split and transposed
-      TB_TRY(split3_transpose(Rb, AT, d, d, st));
-      TB_TRY(split3_transpose(Ub, Bp, d, d, st));
-      TB_TRY(gemm_split_presplit(T1, d, AT, Bp, d, d, d, false, st));
-      // C = T1 U
-      TB_TRY(split3(Ub, Bp, dd, st));
-      TB_TRY(split3_transpose(T1, AT, d, d, st));
-      TB_TRY(gemm_split_presplit(T2, d, AT, Bp, d, d, d, false, st));
-      k_to_float<<<eb, 256, 0, st>>>(T2, C + i * dd, d, 0);
-      TB_LAUNCH_CHECK();
-      // P = (strictly upper part of T1) U, itself strictly upper
-      k_mask_strict_upper<<<eb, 256, 0, st>>>(T1, T2, d);
-      TB_LAUNCH_CHECK();
-      TB_TRY(split3_transpose(T2, AT, d, d, st));
-      TB_TRY(gemm_split_presplit(T1, d, AT, Bp, d, d, d, false, st));
-      k_to_float<<<eb, 256, 0, st>>>(T1, P + i * dd, d, 1);
-      TB_LAUNCH_CHECK();
-    }
-    return TB_OK;
-  }
   for (int i = 0; i < n_batch; ++i) {
     const float* Rb = R + i * dd;
     const float* Ub = U_in + i * dd;

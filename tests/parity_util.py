@@ -74,6 +74,17 @@ def make_problem(seed, d_in, n_heads, d_head, n_tok, *, with_r=False, hout="proj
     return prob
 
 
+_PROBLEMS = {}
+
+
+def cached_problem(*args, **kw):
+    """make_problem, kept for the tests of one process that share a large problem (read-only use)."""
+    key = (args, tuple(sorted(kw.items())))
+    if key not in _PROBLEMS:
+        _PROBLEMS[key] = make_problem(*args, **kw)
+    return _PROBLEMS[key]
+
+
 def oracle_desc(prob, bits, quant_group, out_block, flags, n_cand=16, cd_iters=1, n_heads=None):
     H = n_heads or prob["n_heads"]
     return oracle.OracleDesc(d_out=H * prob["d_head"], d_in=prob["d_in"], n_heads=H, d_head=prob["d_head"],

@@ -6,7 +6,7 @@ import pytest
 
 import oracle
 import tb_inputs
-from parity_util import f32, rel_fro
+from parity_util import cached_problem, f32, rel_fro
 
 pytestmark = pytest.mark.gpu
 
@@ -185,3 +185,44 @@ def test_prepare_correction(n_batch, d):
     assert np.all(np.tril(Pg) == 0.0)
     assert rel_fro(Pg, Po) <= 1e-5
     assert rel_fro(C.cpu().numpy(), Co) <= 1e-5
+
+
+def test_prerequisites_at_full_width():
+    """Every prerequisite at the benchmark's width (4096 columns, 32 heads of 128 rows), in the launch
+    shapes that size produces, against the oracle's float64 results for the same 8192 seeded tokens:
+    Hessian and its undamped sum, deviation correlation R, the factor of H_in (helper streams, all
+    doubling levels), the correction operands P and C on the tensor-core path, H_out from the partner
+    projection and its 32 small factors.  Each call gets the oracle's (float32-rounded) inputs, so the
+    stages are compared one by one."""
+    import torch
+    import paper_2602_04929_b200 as tb
+    d, H, dh, n_tok, alpha, damp = 4096, 32, 128, 8192, 0.25, 0.01
+    prob = cached_problem(0, d, H, dh, n_tok, with_r=True)
+    X, Xfp = tb_inputs.DeviationRecipe(tb_inputs.HeavyTailRecipe(d, seed=0)).chunk(0, n_tok)
+    Xd, Xfd = _t(X, torch.bfloat16), _t(Xfp, torch.bfloat16)
+    Hg = torch.zeros((d, d), dtype=torch.float32, device="cuda:0")
+    Rg = torch.zeros((d, d), dtype=torch.float32, device="cuda:0")
+    Hsum = torch.empty_like(Hg)
+    for t0, t1 in ((0, 6144), (6144, n_tok)):     # two launches, the second shorter
+        tb.tb_accumulate_hessian(Hg, Xd[t0:t1].contiguous())
+        tb.tb_accumulate_cross(Rg, Xd[t0:t1].contiguous(), Xfd[t0:t1].contiguous(), alpha)
+    tb.tb_finalize_hessian(Hg, Rg, n_tok, damp, Hsum_out=Hsum)
+    torch.cuda.synchronize()
+    assert tb.tb_device_error_flag() == 0
+    assert rel_fro(Hg.cpu().numpy(), prob["Hin"][0]) <= 1e-5
+    assert rel_fro(Hsum.cpu().numpy(), prob["Hsum"]) <= 1e-5
+    assert rel_fro(Rg.cpu().numpy(), prob["R"][0]) <= 1e-5
+    U, info = tb.tb_factor(_t(prob["Hin"]))
+    P, C = tb.tb_prepare_correction(_t(prob["R"]), _t(prob["Uin"]))
+    Hout = tb.tb_build_hout(_t(prob["G"]), _t(prob["Hsum"]), H, dh, damp)
+    Uout, info_out = tb.tb_factor(_t(prob["Hout"]))
+    torch.cuda.synchronize()
+    assert tb.tb_device_error_flag() == 0
+    assert int(info.max()) == 0 and int(info_out.max()) == 0
+    errs = {"U_in": rel_fro(U.cpu().numpy()[0], prob["Uin"][0]), "P": rel_fro(P.cpu().numpy(), prob["P"]),
+            "C": rel_fro(C.cpu().numpy(), prob["C"]), "H_out": rel_fro(Hout.cpu().numpy(), prob["Hout"]),
+            "U_out": max(rel_fro(Uout.cpu().numpy()[h], prob["Uout"][h]) for h in range(H))}
+    print("FULL-WIDTH PREREQUISITES rel errors", errs)
+    assert errs["U_in"] <= 1e-6 and errs["U_out"] <= 1e-6
+    assert errs["P"] <= 1e-5 and errs["C"] <= 1e-5
+    assert errs["H_out"] <= 2e-6

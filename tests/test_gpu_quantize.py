@@ -7,7 +7,7 @@ import numpy as np
 import pytest
 
 import tb_inputs
-from parity_util import compare, make_problem, run_gpu
+from parity_util import cached_problem, compare, make_problem, run_gpu
 
 pytestmark = pytest.mark.gpu
 
@@ -107,7 +107,7 @@ def test_llama7b_q_proj_shape_sampled_heads():
 def test_llama7b_q_proj_with_propagated_error_sampled_head():
     """Config 3's q_proj: 4096 x 4096, 32 heads, INT2, group 128, g = 32, adaptive grid + CD, with the
     propagated-error operands R, P, C (alpha = 0.25) from a synthetic input deviation."""
-    prob = make_problem(0, 4096, 32, 128, 8192, with_r=True)
+    prob = cached_problem(0, 4096, 32, 128, 8192, with_r=True)
     gpu = run_gpu(prob, 2, 128, 32, ADAPT | CD)
     compare(prob, gpu, 2, 128, 32, ADAPT | CD, heads=[9], label="7b-q with R, sampled head")
 
