@@ -44,11 +44,11 @@ typedef enum { TB_F32 = 0, TB_BF16 = 1 } tb_dtype;
 /* flags of tb_layer_desc */
 enum {
   TB_F_ADAPTIVE_GRID = 1, /* grid chosen per out-channel group just before it is
-                             quantized (Algorithm 1, line 9; Section 3.3).  Off:
+                             quantized (Algorithm 1, grid step; Section 3.3).  Off:
                              the grid of every row is chosen once from the
                              original weights (the fixed grid of BoA).         */
   TB_F_CD_REFINE = 2      /* coordinate-descent scale refinement after the loop
-                             (Algorithm 1, line 12; Proposition 3.3)           */
+                             (Algorithm 1, refinement; Proposition 3.3)        */
 };
 
 /* Problem description of one projection (Algorithm 1, inputs). */
@@ -82,7 +82,7 @@ typedef struct {
 const char* tb_status_string(tb_status st);
 
 /* --------------------------------------------------------------------------
- * Calibration Hessians (Table 1; Algorithm 1, lines 4-5).
+ * Calibration Hessians (Table 1; Algorithm 1, statistics steps).
  * -------------------------------------------------------------------------- */
 
 /* H += X^T X, the un-normalised running sum of the input Hessian X X^T of
@@ -101,7 +101,7 @@ tb_status tb_accumulate_hessian(float* H, const void* X, tb_dtype x_type,
 int tb_device_error_flag(void);
 
 /* R += alpha * (X - Xfp)^T X, the deviation correlation alpha (X - X~) X^T of
- * Algorithm 1 line 5 in the same un-normalised form: R[a][b] accumulates
+ * Algorithm 1 (deviation step) in the same un-normalised form: R[a][b] accumulates
  * alpha * sum_t (x_t[a] - xfp_t[a]) * x_t[b].  R: [d][d] float, not symmetric.
  * bf16 activations run on the tensor cores (same bounded waits and error word
  * as tb_accumulate_hessian): the deviation is split into two bf16 pieces held
@@ -183,7 +183,7 @@ size_t tb_factor_static_capacity(void);
 tb_status tb_factor_static(const float* H, int n_batch, int d, float* U, int* info, void* stream);
 
 /* Operands of the propagated-error terms from R and U_in:
- *   P = ((R U^T) masked to its strictly upper triangle) U   (Algorithm 2, line 2)
+ *   P = ((R U^T) masked to its strictly upper triangle) U   (Algorithm 2, masked operand)
  *   C = R U^T U = R H_in^{-1}                               (Proposition 3.2)
  * All [n_batch][d][d] float.  U must have a zero strictly-lower triangle.
  * The three products run in double; P and C are rounded to float once. */
@@ -192,16 +192,17 @@ tb_status tb_prepare_correction(const float* R, const float* U_in, int n_batch, 
                                 float* C, void* ws, size_t ws_bytes, void* stream);
 
 /* --------------------------------------------------------------------------
- * The quantizer (Algorithm 1, lines 6-13, for one projection W).
+ * The quantizer (Algorithm 1, the group loop and its closing steps, for one
+ * projection W).
  * -------------------------------------------------------------------------- */
 
 /* For every head, and for every group of out_block rows in turn: choose the
- * grid of the group's rows (line 9), run the column sweep with in-row error
- * feedback through U_in (line 10; Algorithm 2; Eq. 2), then update the rows of
+ * grid of the group's rows (grid step), run the column sweep with in-row error
+ * feedback through U_in (Algorithm 2; Eq. 2), then update the rows of
  * the head not yet quantized with the closed-form joint compensation
- * (line 11; Propositions 3.1 and 3.2).  After the loop optionally refine the
- * scales by coordinate descent (line 12; Proposition 3.3 / Algorithm 3) and
- * write Q = diag(s)(W_int - z) (line 13).
+ * (Propositions 3.1 and 3.2).  After the loop optionally refine the
+ * scales by coordinate descent (Proposition 3.3 / Algorithm 3) and
+ * write Q = diag(s)(W_int - z) (final step).
  *
  * Inputs
  *   W      [d_out][d_in] float

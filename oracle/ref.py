@@ -129,7 +129,7 @@ def hessian(X, damp: float = 0.0, return_sum: bool = False):
 
 
 def cross_correlation(X, Xfp, alpha: float):
-    """R = alpha (X - Xfp) X^T in the paper's layout (Algorithm 1, line 5), i.e.
+    """R = alpha (X - Xfp) X^T in the paper's layout (Algorithm 1, deviation step), i.e.
     R[a, b] = alpha / n * sum_t (x_t[a] - xfp_t[a]) x_t[b] for token-major X."""
     X, Xfp = _f64(X), _f64(Xfp)
     return alpha * ((X - Xfp).T @ X) / X.shape[0]
@@ -188,7 +188,7 @@ def factor_upper(H):
 
 def correction_operands(R, U):
     """P = ((R U^T) * M_U) U with M_U the strictly-upper mask (Algorithm 2,
-    line 2) and C = R H_in^{-1} = R U^T U (Proposition 3.2)."""
+    its masked operand) and C = R H_in^{-1} = R U^T U (Proposition 3.2)."""
     R, U = _f64(R), _f64(U)
     if R.ndim == 3:
         pc = [correction_operands(r, u) for r, u in zip(R, U)]

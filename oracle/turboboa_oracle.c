@@ -18,13 +18,13 @@
  *   H_out  [n_heads][d_head][d_head], U_out likewise; NULL = identity, i.e.
  *          the GPTQ / GPTAQ row of Table 1 (all rows quantized at once).
  *   U      upper triangular with H^{-1} = U^T U (Eq. 2).
- *   R      alpha * (X - Xfp) X^T, already scaled (Algorithm 1, line 5).
+ *   R      alpha * (X - Xfp) X^T, already scaled (Algorithm 1, deviation step).
  *
  * Readings of points the paper leaves open (stated once here, used below):
  *   - integer zero-point z per (row, column group): q = clamp(rne(w/s + z)),
  *     Q = s (q - z).  Every formula of the paper holds with W_int replaced by
  *     Wbar = W_int - z.
- *   - the scale search of Algorithm 1 line 9 is a search over n_cand clipped
+ *   - the scale search of Algorithm 1 (grid step) is a search over n_cand clipped
  *     min-max grids, p_k = 1 - k/32, scored by e H_in[G,G] e^T with
  *     round-to-nearest codes, lowest k on ties.
  *   - column groups of quant_group columns each own a (s, z) pair; the score
@@ -74,7 +74,7 @@ static double rne(double x) { return nearbyint(x); } /* default mode: half-to-ev
 static double clampd(double v, double lo, double hi) { return v < lo ? lo : (v > hi ? hi : v); }
 
 /* ------------------------------------------------------------------------- */
-/* Grid for one row segment (Algorithm 1, line 9).                            */
+/* Grid for one row segment (Algorithm 1, grid step).                         */
 /* w: n weights; H: the n x n diagonal block of H_in (leading dimension ldh). */
 /* Returns chosen candidate; writes s, z and (optionally) all scores.         */
 /* ------------------------------------------------------------------------- */
@@ -183,7 +183,7 @@ static void grid_row(const double *w, int d, int gq, const double *Hin, int maxq
 }
 
 /* ------------------------------------------------------------------------- */
-/* GPTAQ sweep of one row (Algorithm 2, lines 3-7).                           */
+/* GPTAQ sweep of one row (Algorithm 2, its column loop).                     */
 /* w: working copy, overwritten (on return w[j] is NOT meaningful).           */
 /* U: upper factor of H_in^{-1}; P: strictly upper correction or NULL.        */
 /* ------------------------------------------------------------------------- */
@@ -251,7 +251,7 @@ static void comp_matrix(const double *Uo, int dh, int i0, int nb, double *T) {
 }
 
 /* ------------------------------------------------------------------------- */
-/* Group loop of Algorithm 1 (lines 6-11) for one head.                       */
+/* Group loop of Algorithm 1 for one head.                                    */
 /* Wt: [dh][d] working weights W-tilde (in: original rows; out: Q rows).      */
 /* ------------------------------------------------------------------------- */
 static void group_loop_head(const tbo_desc *D, double *Wt, const double *Hin, const double *Uin,
@@ -335,7 +335,7 @@ static void group_loop_head(const tbo_desc *D, double *Wt, const double *Hin, co
 /* The numerator needs row j of Hout ((Q - W) Hin + W R).  The inner product  */
 /* Dm = (Q - W) Hin + W R is kept current: when Q's row changes by            */
 /* delta * Wbar[j,G], row j of Dm changes by delta * Wbar[j,G] Hin[G,:]       */
-/* (that is line 5 of Algorithm 3, "update quantized weights", carried        */
+/* (that is the weight-update step of Algorithm 3, carried                     */
 /* through the product).                                                      */
 /* ------------------------------------------------------------------------- */
 static void cd_head(const tbo_desc *D, const double *W, const unsigned char *codes,
@@ -446,7 +446,7 @@ static double loss_head(int dh, int d, const double *W, const double *Q, const d
 /* Entry points                                                               */
 /* ------------------------------------------------------------------------- */
 
-/* Full per-projection procedure (Algorithm 1 lines 2-13 for one W).
+/* Full per-projection procedure (Algorithm 1 for one W).
  * Returns 0, or a negative number for an invalid description.
  * scales_pre (optional) receives the scales before CD refinement. */
 int tbo_quantize_layer(const tbo_desc *D, const double *W, const double *Hin, const double *Uin,
@@ -484,7 +484,7 @@ int tbo_quantize_layer(const tbo_desc *D, const double *W, const double *Hin, co
     if (scales_pre) memcpy(scales_pre + ro * ng, scales + ro * ng, sizeof(double) * (size_t)dh * ng);
     if ((D->flags & TBO_F_CD_REFINE) && D->cd_iters > 0)
       cd_head(D, Wh, codes + ro * d, zeros + ro * ng, scales + ro * ng, Hin_h, Ho, Rh);
-    /* Q <- diag(s) W_int (Algorithm 1, line 13) */
+    /* Q <- diag(s) W_int (Algorithm 1, final step) */
     for (int r = 0; r < dh; ++r)
       for (int a = 0; a < d; ++a) {
         int g = a / seg;

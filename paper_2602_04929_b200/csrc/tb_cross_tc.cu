@@ -1,4 +1,4 @@
-// Deviation correlation R += alpha (X - Xfp)^T X (Algorithm 1 line 5) for bf16
+// Deviation correlation R += alpha (X - Xfp)^T X (Algorithm 1, deviation step) for bf16
 // activations on the 5th-generation tensor cores.
 //
 // D = X - Xfp is formed in float (exact whenever the two values differ by less than

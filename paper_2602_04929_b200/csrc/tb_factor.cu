@@ -1,5 +1,5 @@
 // tb_factor: U upper triangular with H^{-1} = U^T U (Eq. 2), batched, and
-// tb_prepare_correction: P and C of Algorithm 2 line 2 / Proposition 3.2.
+// tb_prepare_correction: P and C of Algorithm 2 (masked operand) / Proposition 3.2.
 //
 // Route taken for U (the positive-diagonal factor is unique, so any route to it
 // is the factor of Eq. 2): with J the index reversal, J H J = L L^T is an
@@ -287,7 +287,7 @@ __global__ void __launch_bounds__(64) k_inv_diag64(const double* __restrict__ Ld
   for (int r = 0; r < FNB; ++r) Li[off + (long long)r * dp + c] = x[r];
 }
 
-// strictly-upper mask of a square matrix (Algorithm 2 line 2: (R U^T) .* M_U)
+// strictly-upper mask of a square matrix (Algorithm 2: (R U^T) .* M_U)
 __global__ void k_mask_strict_upper(const double* __restrict__ src, double* __restrict__ dst, int d) {
   const long long n = (long long)d * d;
   for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < n;

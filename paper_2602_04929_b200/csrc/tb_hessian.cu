@@ -1,4 +1,4 @@
-// Calibration Hessians (Table 1; Algorithm 1 lines 4-5):
+// Calibration Hessians (Table 1; Algorithm 1, statistics steps):
 //   tb_accumulate_hessian  H += X^T X          (X token-major, so this is the paper's X X^T)
 //   tb_accumulate_cross    R += alpha (X - Xfp)^T X
 //   tb_finalize_hessian    normalisation by the token count and diagonal damping

@@ -1,12 +1,12 @@
-// tb_quantize_layer: the out-channel-group loop of Algorithm 1 (lines 6-13).
+// tb_quantize_layer: the out-channel-group loop of Algorithm 1 and its closing steps.
 //
 // Per step i (a group of g = out_block rows of every head, M = n_heads * g
 // rows in all, heads being independent):
-//   grid     k_grid           Algorithm 1 line 9    candidate search per (row, column group)
+//   grid     k_grid           Algorithm 1, grid     candidate search per (row, column group)
 //   sweep    k_sweep_rows     Algorithm 2 / Eq. 2   one launch, 8 rows per CTA for the whole sweep
 //   residual k_residual       E = W0 - Q_B          (Proposition 3.1)
 //            GEMM             E -= W0 C             (Proposition 3.2, only with R)
-//   update   GEMM             W~[rem] -= T_i E      (Algorithm 1 line 11)
+//   update   GEMM             W~[rem] -= T_i E      (Algorithm 1, update)
 // then, once: coordinate descent on the scales (Algorithm 3), Q = s (W_int - z),
 // and the loss of the proofs of Propositions 3.1 / 3.2.
 //
@@ -94,7 +94,7 @@ __global__ void k_comp_matrices(const float* __restrict__ Uout, double* __restri
 }
 
 // ---------------------------------------------------------------------------
-// Grid search (Algorithm 1 line 9).  For every (row, column group): n_cand
+// Grid search (Algorithm 1, grid step).  For every (row, column group): n_cand
 // clipped min-max grids, p_k = 1 - k/32; score e H_in[G,G] e^T with e the
 // round-to-nearest error on that grid; the lowest score wins, lowest k on ties.
 //
@@ -1478,7 +1478,7 @@ __global__ void k_axpy(double* __restrict__ y, const double* __restrict__ x, lon
     y[i] += x[i];
 }
 
-// Q = s (W_int - z) in float, and the scales in float (Algorithm 1, line 13).
+// Q = s (W_int - z) in float, and the scales in float (Algorithm 1, final step).
 __global__ void k_dequant(const unsigned char* __restrict__ codes, const double* __restrict__ sD,
                           const int* __restrict__ z, float* __restrict__ What,
                           float* __restrict__ s_out, long long rows, int d, int seg, int ng) {
@@ -1904,7 +1904,7 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
       TB_TRY((gemm_launch<double, float, double, double, false, true>(g, st)));
     }
     {
-      // W~[rem rows of every head] -= T_i E   (Propositions 3.1 / 3.2; Algorithm 1 line 11)
+      // W~[rem rows of every head] -= T_i E   (Propositions 3.1 / 3.2; Algorithm 1, update step)
       GemmP g = gemm_params();
       g.A = p.T + (long long)step * p.dh * p.g;
       g.a_m = p.g;

@@ -49,7 +49,7 @@ def test_hessian_accumulation(n_tok, d, bf16):
 @pytest.mark.parametrize("bf16,d,chunks", [(True, 264, (6000,)), (False, 264, (6000,)), (True, 512, (5000, 64, 3001)),
                                             (True, 128, (7,))])
 def test_cross_correlation(bf16, d, chunks):
-    """R = alpha (X - Xfp) X^T / n (Algorithm 1, line 5), not symmetric; several launches with
+    """R = alpha (X - Xfp) X^T / n (Algorithm 1, deviation step), not symmetric; several launches with
     ragged token counts and a width that is not a multiple of the tile.  bf16: the deviation is
     split into two bf16 pieces (exact here), every product is exact in float and the float
     accumulation is cut into runs of 2048 steps, so the error stays far below 1e-5."""
@@ -167,7 +167,7 @@ def test_factor_is_independent_of_other_work_on_the_gpu():
 
 @pytest.mark.parametrize("n_batch,d", [(1, 256), (2, 200)])
 def test_prepare_correction(n_batch, d):
-    """P = ((R U^T) masked strictly upper) U (Algorithm 2, line 2); C = R U^T U (Proposition 3.2)."""
+    """P = ((R U^T) masked strictly upper) U (Algorithm 2, its masked operand); C = R U^T U (Proposition 3.2)."""
     import torch
     import paper_2602_04929_b200 as tb
     Rs, Us = [], []
