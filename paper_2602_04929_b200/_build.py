@@ -15,7 +15,8 @@ LIB = os.path.join(HERE, "libturboboa.so")
 
 SOURCES = ["tb_api.cu", "tb_hessian.cu", "tb_syrk_tc.cu", "tb_cross_tc.cu", "tb_gemm_tc.cu", "tb_factor.cu", "tb_factor_static.cu", "tb_quantize.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "-Xcompiler", "-fPIC", "-I", INCLUDE, "-I", CSRC]
+              "-Xcompiler", "-fPIC", "-Xcompiler", "-Werror=pointer-arith",   # no arithmetic on untyped pointers
+              "-I", INCLUDE, "-I", CSRC]
 
 
 def _nvcc() -> str:
