@@ -1538,6 +1538,7 @@ struct Plan {
   bool yw_tensor;
   bool dm_tensor;  // (Q - W) H_in through the split-bf16 tensor-core product as well
   bool loss_tensor;  // the loss's own dW H_in (no scale refinement) through it too
+  int loss_heads;    // with one H_in per head: heads per launch of that product (their pieces of H_in fit 2 GiB)
   size_t ws_total;
 };
 
@@ -1631,8 +1632,17 @@ static tb_status make_plan(const tb_layer_desc* D, bool has_hout, bool with_r, b
     p.Amat = b.take<double>((size_t)lines * p.ng * p.ng);
   }
   // without the scale refinement the loss forms dW H_in itself: the same split-bf16 product
-  p.loss_tensor = with_loss && !p.cd && (p.n_hin == 1) && (p.d % 32 == 0) && (p.d_out % 8 == 0);
-  if (p.loss_tensor) p.Hp = b.take<__nv_bfloat16>((size_t)3 * dd * dd);
+  // (with one H_in per head the heads of a batch share the launch, each against its own pieces: that
+  // needs heads of whole 128-row tiles)
+  p.loss_tensor = with_loss && !p.cd && (p.n_hin == 1 || p.dh % 128 == 0) && (p.d % 32 == 0) && (p.d_out % 8 == 0);
+  p.loss_heads = 1;
+  if (p.loss_tensor && p.n_hin > 1) {
+    const size_t per_head = (size_t)3 * dd * dd * sizeof(__nv_bfloat16);
+    size_t fit = ((size_t)2 << 30) / per_head;
+    if (fit < 1) fit = 1;
+    p.loss_heads = (fit < (size_t)p.H) ? (int)fit : p.H;
+  }
+  if (p.loss_tensor) p.Hp = b.take<__nv_bfloat16>((size_t)3 * dd * dd * (size_t)p.loss_heads);
   if (with_loss) p.G2 = b.take<double>((size_t)p.H * p.dh * (has_hout ? p.dh : 1));  // Z dW^T, or partial sums
   p.ws_total = b.total();
   return TB_OK;
@@ -2195,11 +2205,21 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
     // dW H_in for the final scales (it was kept current through the pass), so the product is skipped.
     // With R the pass keeps Dm = dW H_in + W R, so only one more W R is missing.
     const bool dm_is_current = p.cd;
-    if (!dm_is_current && p.loss_tensor) {
+    if (!dm_is_current && p.loss_tensor && units == 1) {
       __nv_bfloat16* DqT = reinterpret_cast<__nv_bfloat16*>(p.Wt);  // W~ is no longer needed
       TB_TRY(split3_transpose(p.Dq, DqT, p.d_out, d, st));
       TB_TRY(split3(H_in, p.Hp, dd, st));
       TB_TRY(gemm_split_presplit(p.Dm, d, DqT, p.Hp, p.d_out, d, d, false, st));
+    } else if (!dm_is_current && p.loss_tensor) {
+      // one H_in per head: a batch of heads per launch, every head against its own pieces
+      for (int h0 = 0; h0 < p.H; h0 += p.loss_heads) {
+        const int nb = (p.H - h0 < p.loss_heads) ? (p.H - h0) : p.loss_heads;
+        const long long rr = (long long)h0 * p.dh, rows = (long long)nb * p.dh;
+        __nv_bfloat16* DqT = reinterpret_cast<__nv_bfloat16*>(p.Wt + rr * d);  // W~ is no longer needed
+        TB_TRY(split3_transpose(p.Dq + rr * d, DqT, rows, d, st));
+        TB_TRY(split3(H_in + (long long)h0 * dd, p.Hp, dd * nb, st));
+        TB_TRY(gemm_split_presplit(p.Dm + rr * d, d, DqT, p.Hp, rows, d, d, false, st, nb));
+      }
     } else if (!dm_is_current) {
       TB_TRY((gemm_launch<double, float, double, double, false, true>(g, st)));
     }

@@ -65,6 +65,13 @@ def test_per_head_input_hessians():
     _case(prob, 3, 128, 8, ADAPT | CD, label="per-head H_in")
 
 
+def test_per_head_input_hessians_without_scale_refinement():
+    """One H_in per head, heads of 128 rows, no coordinate descent: the loss then forms (Q - W) H_in
+    itself, the heads sharing one tensor-core launch, each against the pieces of its own H_in."""
+    prob = make_problem(12, 256, 3, 128, 1024, n_hin=3, hout="spd")
+    _case(prob, 3, 128, 32, ADAPT, label="per-head H_in, no CD")
+
+
 def test_ragged_rows_and_candidate_counts():
     """Row counts that fill neither a panel CTA (8 rows) nor a GEMM tile; 5 and 32 candidates."""
     prob = make_problem(7, 384, 5, 21, 1024)
