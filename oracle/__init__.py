@@ -15,7 +15,6 @@ from .ref import (  # noqa: F401
     hessian,
     cross_correlation,
     hout_from_projection,
-    hout_from_gram,
     factor_upper,
     correction_operands,
     quantize_layer,

@@ -168,12 +168,6 @@ def hout_from_projection(G, Hsum, n_heads: int, d_head: int, damp: float = 0.0):
     return out
 
 
-def hout_from_gram(G):
-    """H_out = G^T G for an explicit G (the unified loss ||G dW X||_F^2)."""
-    G = _f64(G)
-    return G.T @ G
-
-
 def factor_upper(H):
     """U = Chol(H^{-1})^T, upper triangular with H^{-1} = U^T U (Eq. 2).
     Written as the definition: invert, lower Cholesky, transpose."""

@@ -670,3 +670,100 @@ def test_hints_are_adopted_only_inside_the_band():
     hint = c0.copy(); hint[0, 0] = 1
     c1, _, _, cnt1 = oracle.sweep_rows(Wt, U, np.array([[s]]), np.array([[z]]), 0, 2, hint_codes=hint)
     assert c1[0, 0] == 1 and cnt1["adopted_codes"] == 1
+
+
+# --------------------------------------------------------------------------- one H_in per head (the W_V row of Table 1)
+@pytest.mark.parametrize("with_r", [False, True])
+def test_per_head_input_hessians_equal_head_by_head_runs(with_r):
+    """n_hin = n_heads: head h must see H_in[h], U_in[h] (and R, P, C [h]) and nothing else.
+    Three heads with three different input Hessians, run once as one layer and once head by head
+    with a shared-H_in description each."""
+    dh, d, H = 4, 8, 3
+    prs = [small_problem(300 + h, dh=dh, d=d, with_r=with_r) for h in range(H)]
+    W = np.concatenate([p["W"] for p in prs])
+    Hin = np.stack([p["Hin"] for p in prs])
+    Uin = np.stack([oracle.factor_upper(p["Hin"]) for p in prs])
+    Ho = np.stack([p["Hout"][0] for p in prs])
+    Uo = oracle.factor_upper(Ho)
+    R = P = C = None
+    if with_r:
+        R = np.stack([p["R"] for p in prs])
+        P, C = oracle.correction_operands(R, Uin)
+    flags = F_ADAPTIVE_GRID | F_CD_REFINE
+    desc = OracleDesc(H * dh, d, H, dh, bits=2, quant_group=4, out_block=2, n_hin=H, flags=flags)
+    full = oracle.quantize_layer(desc, W, Hin, Uin, Ho, Uo, R, P, C)
+    assert not np.allclose(Hin[0], Hin[1])
+    for h in range(H):
+        one_desc = OracleDesc(dh, d, 1, dh, bits=2, quant_group=4, out_block=2, n_hin=1, flags=flags)
+        sl = slice(h * dh, (h + 1) * dh)
+        one = oracle.quantize_layer(one_desc, W[sl], Hin[h], Uin[h], Ho[h:h + 1], Uo[h:h + 1],
+                                    None if R is None else R[h], None if P is None else P[h],
+                                    None if C is None else C[h])
+        assert np.array_equal(one.codes, full.codes[sl]) and np.array_equal(one.zeros, full.zeros[sl])
+        assert np.array_equal(one.cand, full.cand[sl])
+        assert np.allclose(one.scales, full.scales[sl], atol=0)
+        assert np.allclose(one.w_comp, full.w_comp[sl], atol=0)
+        assert np.isclose(one.loss[0], full.loss[h], rtol=1e-12)
+        # and the per-head loss is the loss under that head's own Hessians
+        ref = oracle.loss_head(W[sl], full.w_hat[sl], Hin[h], Ho[h], None if R is None else R[h])
+        assert np.isclose(full.loss[h], ref, rtol=1e-12)
+
+
+# --------------------------------------------------------------------------- H_out = NULL branches of CD and loss
+@pytest.mark.parametrize("with_r", [False, True])
+@pytest.mark.parametrize("gq", [0, 4])
+def test_cd_and_loss_without_hout_equal_identity_hout(gq, with_r):
+    """The GPTQ / GPTAQ row of Table 1 (H_out = I): the NULL branches of the scale refinement and of
+    the loss against Proposition 3.3 evaluated literally with H_out = I, against the explicit loss
+    ||dW X||^2 (+ cross term) with G = I, and against the dense-identity branch."""
+    dh, d = 5, 8
+    pr = small_problem(83, dh=dh, d=d, with_r=with_r)
+    W, Hin, R = pr["W"], pr["Hin"], pr.get("R")
+    eye = np.eye(dh)
+    g = np.random.default_rng(83)
+    seg = gq or d
+    ng = d // seg
+    codes = g.integers(0, 4, size=(dh, d)).astype(np.uint8)
+    zeros = g.integers(0, 4, size=(dh, ng)).astype(np.int32)
+    s0 = 0.02 * (1 + 0.2 * g.random((dh, ng)))
+    desc = OracleDesc(dh, d, 1, dh, bits=2, quant_group=gq, cd_iters=1)
+    s_null = oracle.cd_refine(desc, W, codes, zeros, s0, Hin, None, R)
+    s_eye = oracle.cd_refine(desc, W, codes, zeros, s0, Hin, eye, R)
+    assert np.allclose(s_null, s_eye, rtol=1e-13, atol=0)
+    Wb = codes.astype(float) - np.repeat(zeros, seg, axis=1)
+    s = s0.copy()
+    for j in range(dh):
+        for gi in range(ng):
+            cols = slice(gi * seg, (gi + 1) * seg)
+            if not Wb[j, cols].any():
+                continue
+            Q = np.repeat(s, seg, axis=1) * Wb
+            s[j, gi] += literal_cd_step(Wb, W, Q, Hin, eye, R, j, cols)
+    assert np.allclose(s_null, s, rtol=1e-10, atol=1e-15)
+    # rows are independent without H_out: refining one row alone gives that row's scales
+    one = OracleDesc(1, d, 1, 1, bits=2, quant_group=gq, cd_iters=1)
+    for j in range(dh):
+        sj = oracle.cd_refine(one, W[j:j + 1], codes[j:j + 1], zeros[j:j + 1], s0[j:j + 1], Hin, None, R)
+        assert np.allclose(sj, s_null[j:j + 1], rtol=1e-12, atol=0)
+    # loss
+    Q = np.repeat(s_null, seg, axis=1) * Wb
+    l_null = oracle.loss_head(W, Q, Hin, None, R)
+    assert np.isclose(l_null, oracle.loss_head(W, Q, Hin, eye, R), rtol=1e-13)
+    X, n = pr["X"], pr["n_tok"]
+    lam = 0.01 * np.mean(np.diag(X @ X.T / n))
+    ref = explicit_loss(eye, Q - W, X, W, pr.get("dX"), pr.get("alpha", 1.0), n, damp_term=lam)
+    assert np.isclose(l_null, ref, rtol=1e-10)
+
+
+def test_identity_mode_layer_reports_refined_scales_and_loss():
+    """Whole-layer run in the H_out = NULL mode with the scale refinement on: the scales equal
+    cd_refine on the pre-refinement scales, and the reported loss is the loss of w_hat."""
+    pr = small_problem(84, dh=6, d=16, with_r=True)
+    out = run_layer(pr, 3, 8, 6, F_ADAPTIVE_GRID | F_CD_REFINE, hout=False, with_r=True)
+    desc = OracleDesc(6, 16, 1, 6, bits=3, quant_group=8, cd_iters=1)
+    s1 = oracle.cd_refine(desc, pr["W"], out.codes, out.zeros, out.scales_pre_cd, pr["Hin"], None, pr["R"])
+    assert np.allclose(out.scales, s1, atol=0)
+    assert not np.allclose(out.scales, out.scales_pre_cd)
+    assert np.isclose(out.loss[0], oracle.loss_head(pr["W"], out.w_hat, pr["Hin"], None, pr["R"]), rtol=1e-13)
+    pre = np.repeat(out.scales_pre_cd, 8, axis=1) * (out.codes.astype(float) - np.repeat(out.zeros, 8, axis=1))
+    assert out.loss[0] <= oracle.loss_head(pr["W"], pre, pr["Hin"], None, pr["R"])
