@@ -189,8 +189,7 @@ def run_reference(args, cfg, proj, rank, world):
     import oracle
     d, dh = proj.d_in, proj.d_head
     n_tok = 4096
-    sys.path.insert(0, os.path.join(ROOT, "tests"))
-    import parity_util as pu
+    import oracle.problems as pu
     prob = pu.make_problem(0, d, 1, dh, n_tok, hout="proj" if proj.partner else None)
     flags = (FLAGS_ADAPT if cfg.adaptive else 0) | (FLAGS_CD if cfg.cd else 0)
     od = pu.oracle_desc(prob, cfg.bits, cfg.quant_group, cfg.out_block, flags)
@@ -221,8 +220,7 @@ def run_reference(args, cfg, proj, rank, world):
 def cpu_baseline(cfg, proj, budget_s: float = 20.0):
     """Oracle timed on the host cores on a bounded sample of the same workload."""
     import oracle
-    sys.path.insert(0, os.path.join(ROOT, "tests"))
-    import parity_util as pu
+    import oracle.problems as pu
     d, dh = proj.d_in, proj.d_head
     prob = pu.make_problem(0, d, 1, dh, 4096, hout="proj" if proj.partner else None)
     flags = (FLAGS_ADAPT if cfg.adaptive else 0) | (FLAGS_CD if cfg.cd else 0)

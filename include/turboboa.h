@@ -36,7 +36,8 @@ typedef enum {
   TB_ERR_WORKSPACE = 3,   /* workspace NULL, misaligned or too small            */
   TB_ERR_NOT_SPD = 4,     /* reserved for host-side checks of info words        */
   TB_ERR_CUDA = 5,        /* a CUDA runtime call failed (launch, attribute)     */
-  TB_ERR_TIMEOUT = 6      /* reserved: a bounded device-side wait ran out       */
+  TB_ERR_TIMEOUT = 6      /* a bounded device-side wait ran out (see
+                             tb_device_error_flag)                              */
 } tb_status;
 
 typedef enum { TB_F32 = 0, TB_BF16 = 1 } tb_dtype;
@@ -99,6 +100,14 @@ tb_status tb_accumulate_hessian(float* H, const void* X, tb_dtype x_type,
  * (TB_ERR_TIMEOUT), -1 = the word could not be read.  Synchronises the device.
  * No counterpart in the paper. */
 int tb_device_error_flag(void);
+
+/* Self-test of that mechanism, with no counterpart in the paper: launches one
+ * small CTA that waits, through the library's bounded wait, on a hardware barrier
+ * at which nothing ever arrives, with a budget of budget_cycles SM clock cycles
+ * (0 .. 2e8, i.e. at most about 0.1 s).  The wait gives up, the kernel returns
+ * normally, *gave_up (device int, may be NULL) becomes 1 and the next
+ * tb_device_error_flag() returns 1.  Nothing faults and the context stays usable. */
+tb_status tb_selftest_bounded_wait(long long budget_cycles, int* gave_up, void* stream);
 
 /* R += alpha * (X - Xfp)^T X, the deviation correlation alpha (X - X~) X^T of
  * Algorithm 1 (deviation step) in the same un-normalised form: R[a][b] accumulates
@@ -174,6 +183,12 @@ tb_status tb_factor(const float* H, int n_batch, int d, float* U, float* Hinv, i
  *
  * The first call on each device looks up the array's device address (the
  * device must be current); make that first call outside any stream capture.
+ * Under CUDA's lazy module loading the array may only come into existence at
+ * that first look-up, so make the first call at start-up, while the device
+ * still has 32 MiB free: a process that first fills the device and only then
+ * calls this for the first time can get TB_ERR_CUDA.  The address is kept per
+ * device ordinal for the life of the process (no lock: make the first call of
+ * a device from one thread).
  * All calls share the one array: it keeps whatever the previous call left
  * (the call clears what it needs zeroed), and two calls whose work overlaps on
  * the GPU -- different streams, or different host threads -- race on it.
@@ -222,6 +237,10 @@ tb_status tb_prepare_correction(const float* R, const float* U_in, int n_batch, 
  *          every formula holds with W_int replaced by W_int - z)
  *   cand   [d_out][n_g] unsigned char or NULL: index k of the chosen grid candidate
  *   W_hat  [d_out][d_in] float or NULL: Q
+ *   W_comp [d_out][d_in] double or NULL: the compensated weights, row r as it stood
+ *          when its group was taken for quantization (the rows W~_B that Algorithm 1
+ *          hands to the sweep: the original row plus every joint compensation it
+ *          received from the groups of its head quantized before it)
  *   loss   [n_heads] double or NULL: tr(dW H_in dW^T H_out) + 2 tr(H_out W R dW^T),
  *          dW = Q - W (the objective in the proofs of Propositions 3.1 / 3.2)
  *   stats  tb_stats (device) or NULL
@@ -233,7 +252,7 @@ tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W, const flo
                             const float* U_in, const float* H_out, const float* U_out,
                             const float* R, const float* P, const float* C,
                             unsigned char* codes, float* scales, int* zeros, unsigned char* cand,
-                            float* W_hat, double* loss, tb_stats* stats, void* ws,
+                            float* W_hat, double* W_comp, double* loss, tb_stats* stats, void* ws,
                             size_t ws_bytes, void* stream);
 
 /* Profiling aid with no counterpart in the paper.  While enabled, every
@@ -257,7 +276,12 @@ int tb_profile_read(double* ms_by_phase, int n);
  * the pieces that have arrived accumulates, and later runs the H_out build and
  * its factor beside the factor of H_in.  X_host is bf16 [n_tok][d_in]; G_host is the partner
  * projection [g_heads*d_head][d_in] float or NULL (then H_out = identity).
- * Returns TB_ERR_NOT_SPD if a factorisation met a non-positive pivot. */
+ * The description is validated in full before anything is enqueued.  If a step
+ * fails after that, the call still joins its helper stream and waits for every
+ * copy it started before it returns the error, so the host buffers are never
+ * in use on return.  Returns TB_ERR_NOT_SPD if a factorisation met a
+ * non-positive pivot and TB_ERR_TIMEOUT if a bounded wait of a tensor-core
+ * kernel ran out (it reads and clears the word of tb_device_error_flag). */
 size_t tb_quantize_from_host_workspace(const tb_layer_desc* desc, long long n_tok, int g_heads);
 tb_status tb_quantize_from_host(const tb_layer_desc* desc, const float* W_host,
                                 const void* X_host, long long n_tok, const float* G_host,

@@ -58,6 +58,7 @@ _SIGNATURES = {
     "tb_status_string": (ctypes.c_char_p, [_int]),
     "tb_accumulate_hessian": (_int, [_vp, _vp, _int, _ll, _int, _vp]),
     "tb_device_error_flag": (_int, []),
+    "tb_selftest_bounded_wait": (_int, [_ll, _vp, _vp]),
     "tb_accumulate_cross_workspace": (_sz, [_int, _ll, _int]),
     "tb_accumulate_cross": (_int, [_vp, _vp, _vp, _int, _ll, _int, _f, _vp, _sz, _vp]),
     "tb_finalize_hessian": (_int, [_vp, _vp, _vp, _int, _ll, _f, _vp]),
@@ -70,7 +71,7 @@ _SIGNATURES = {
     "tb_prepare_correction_workspace": (_sz, [_int, _int]),
     "tb_prepare_correction": (_int, [_vp, _vp, _int, _int, _vp, _vp, _vp, _sz, _vp]),
     "tb_quantize_layer_workspace": (_sz, [ctypes.POINTER(LayerDesc), _int, _int]),
-    "tb_quantize_layer": (_int, [ctypes.POINTER(LayerDesc)] + [_vp] * 15 + [_vp, _sz, _vp]),
+    "tb_quantize_layer": (_int, [ctypes.POINTER(LayerDesc)] + [_vp] * 16 + [_vp, _sz, _vp]),
     "tb_profile_enable": (None, [_int]),
     "tb_profile_read": (_int, [ctypes.POINTER(ctypes.c_double), _int]),
     "tb_quantize_from_host_workspace": (_sz, [ctypes.POINTER(LayerDesc), _ll, _int]),
@@ -152,6 +153,11 @@ def tb_accumulate_hessian(H, X) -> None:
 
 def tb_device_error_flag() -> int:
     return int(load().tb_device_error_flag())
+
+
+def tb_selftest_bounded_wait(budget_cycles: int, gave_up=None) -> None:
+    _check(load().tb_selftest_bounded_wait(int(budget_cycles), _ptr(gave_up, torch.int32, True), _stream()),
+           "tb_selftest_bounded_wait")
 
 
 def tb_accumulate_cross(R, X, Xfp, alpha: float) -> None:
@@ -242,6 +248,7 @@ class QuantizeResult:
     w_hat: torch.Tensor
     loss: torch.Tensor | None
     stats: torch.Tensor
+    w_comp: torch.Tensor | None = None   # float64 [d_out][d_in], the compensated weights (optional output)
 
     def stats_dict(self) -> dict:
         v = self.stats.cpu().tolist()
@@ -253,7 +260,8 @@ def tb_quantize_layer_workspace(desc: LayerDesc, with_r: bool, with_loss: bool) 
 
 
 def tb_quantize_layer(desc: LayerDesc, W, H_in, U_in, H_out=None, U_out=None, R=None, P=None, C=None,
-                      want_loss: bool = True, ws=None, out: QuantizeResult | None = None) -> QuantizeResult:
+                      want_loss: bool = True, ws=None, out: QuantizeResult | None = None,
+                      want_w_comp: bool = False) -> QuantizeResult:
     lib = load()
     dev = W.device
     ng = desc.n_groups
@@ -265,7 +273,8 @@ def tb_quantize_layer(desc: LayerDesc, W, H_in, U_in, H_out=None, U_out=None, R=
             cand=torch.empty((desc.d_out, ng), dtype=torch.uint8, device=dev),
             w_hat=torch.empty((desc.d_out, desc.d_in), dtype=torch.float32, device=dev),
             loss=torch.empty(desc.n_heads, dtype=torch.float64, device=dev) if want_loss else None,
-            stats=torch.zeros(8, dtype=torch.int64, device=dev))
+            stats=torch.zeros(8, dtype=torch.int64, device=dev),
+            w_comp=torch.empty((desc.d_out, desc.d_in), dtype=torch.float64, device=dev) if want_w_comp else None)
     if ws is None:
         ws = _workspace(tb_quantize_layer_workspace(desc, R is not None, out.loss is not None), dev)
     f32 = torch.float32
@@ -273,7 +282,7 @@ def tb_quantize_layer(desc: LayerDesc, W, H_in, U_in, H_out=None, U_out=None, R=
         ctypes.byref(desc), _ptr(W, f32), _ptr(H_in, f32), _ptr(U_in, f32), _ptr(H_out, f32, True),
         _ptr(U_out, f32, True), _ptr(R, f32, True), _ptr(P, f32, True), _ptr(C, f32, True),
         _ptr(out.codes), _ptr(out.scales), _ptr(out.zeros), _ptr(out.cand), _ptr(out.w_hat),
-        _ptr(out.loss, None, True), _ptr(out.stats), _ptr(ws), ws.numel(), _stream()), "tb_quantize_layer")
+        _ptr(out.w_comp, torch.float64, True), _ptr(out.loss, None, True), _ptr(out.stats), _ptr(ws), ws.numel(), _stream()), "tb_quantize_layer")
     return out
 
 

@@ -109,33 +109,22 @@ extern "C" size_t tb_quantize_from_host_workspace(const tb_layer_desc* desc, lon
   return host_plan(desc, n_tok, g_heads, nullptr).total;
 }
 
-extern "C" tb_status tb_quantize_from_host(const tb_layer_desc* desc, const float* W_host,
-                                           const void* X_host, long long n_tok,
-                                           const float* G_host, int g_heads, float damp_in,
-                                           float damp_out, unsigned char* codes_host,
-                                           float* scales_host, int* zeros_host, float* W_hat_host,
-                                           double* loss_host, void* dev_ws, size_t ws_bytes,
-                                           void* stream) {
-  if (!desc_ok(desc, n_tok, G_host ? g_heads : 0)) return TB_ERR_INVALID_ARG;
-  if (!W_host || !X_host || !codes_host || !scales_host || !zeros_host) return TB_ERR_INVALID_ARG;
-  if (desc->n_hin != 1) return TB_ERR_UNSUPPORTED;  // one shared H_in on this entry point
-  if (!G_host) g_heads = 0;
-  const HostPlan hs = host_plan(desc, n_tok, g_heads, nullptr);
-  if (!dev_ws || !aligned(dev_ws, 256) || ws_bytes < hs.total) return TB_ERR_WORKSPACE;
-  const HostPlan h = host_plan(desc, n_tok, g_heads, dev_ws);
+namespace {
+
+// Everything tb_quantize_from_host enqueues; returns at the first failure.  The caller joins the
+// helper stream and synchronises whatever the outcome, so no copy is in flight when it returns.
+tb_status from_host_enqueue(const tb_layer_desc* desc, const HostPlan& h, SideStream* ss, const float* W_host,
+                            const void* X_host, long long n_tok, const float* G_host, int g_heads, float damp_in,
+                            float damp_out, unsigned char* codes_host, float* scales_host, int* zeros_host,
+                            float* W_hat_host, double* loss_host, int* info_host, int n_info, void* stream) {
   cudaStream_t st = as_stream(stream);
   const size_t d = (size_t)desc->d_in, dout = (size_t)desc->d_out;
   const size_t ng = desc->quant_group > 0 ? d / (size_t)desc->quant_group : 1;
   const int H = desc->n_heads, dh = desc->d_head;
-
   // X is by far the largest transfer: it goes over in pieces on the helper stream while the Hessian
   // of the pieces that have arrived accumulates on the caller's stream.  Pieces are multiples of 2048
   // tokens, so the sums are those of a single accumulation over all tokens.
-  SideStream* ss = side_stream();
-  if (!ss) return TB_ERR_CUDA;
   long long piece = ((n_tok + COPY_CHUNKS_MAX / 2 - 1) / (COPY_CHUNKS_MAX / 2) + 2047) / 2048 * 2048;  // about 8 pieces
-  TB_CUDA_CHECK(cudaEventRecord(ss->fork, st));  // earlier work on the caller's stream may still use the buffers
-  TB_CUDA_CHECK(cudaStreamWaitEvent(ss->stream, ss->fork, 0));
   TB_CUDA_CHECK(cudaMemsetAsync(h.Hin, 0, d * d * sizeof(float), st));
   int n_pieces = 0;
   for (long long t0 = 0; t0 < n_tok; t0 += piece, ++n_pieces) {
@@ -169,7 +158,7 @@ extern "C" tb_status tb_quantize_from_host(const tb_layer_desc* desc, const floa
   if (g_heads > 0) TB_CUDA_CHECK(cudaStreamWaitEvent(st, ss->join, 0));
   TB_TRY(tb_quantize_layer(desc, h.W, h.Hin, h.Uin, h.Hout, h.Uout, nullptr, nullptr, nullptr,
                            h.codes, h.scales, h.zeros, nullptr, W_hat_host ? h.What : nullptr,
-                           loss_host ? h.loss : nullptr, nullptr, h.sub, h.sub_bytes, stream));
+                           nullptr, loss_host ? h.loss : nullptr, nullptr, h.sub, h.sub_bytes, stream));
   TB_CUDA_CHECK(cudaMemcpyAsync(codes_host, h.codes, dout * d, cudaMemcpyDeviceToHost, st));
   TB_CUDA_CHECK(cudaMemcpyAsync(scales_host, h.scales, dout * ng * sizeof(float), cudaMemcpyDeviceToHost, st));
   TB_CUDA_CHECK(cudaMemcpyAsync(zeros_host, h.zeros, dout * ng * sizeof(int), cudaMemcpyDeviceToHost, st));
@@ -177,10 +166,60 @@ extern "C" tb_status tb_quantize_from_host(const tb_layer_desc* desc, const floa
     TB_CUDA_CHECK(cudaMemcpyAsync(W_hat_host, h.What, dout * d * sizeof(float), cudaMemcpyDeviceToHost, st));
   if (loss_host)
     TB_CUDA_CHECK(cudaMemcpyAsync(loss_host, h.loss, sizeof(double) * (size_t)H, cudaMemcpyDeviceToHost, st));
+  TB_CUDA_CHECK(cudaMemcpyAsync(info_host, h.info, sizeof(int) * (size_t)n_info, cudaMemcpyDeviceToHost, st));
+  return TB_OK;
+}
+
+}  // namespace
+
+extern "C" tb_status tb_quantize_from_host(const tb_layer_desc* desc, const float* W_host,
+                                           const void* X_host, long long n_tok,
+                                           const float* G_host, int g_heads, float damp_in,
+                                           float damp_out, unsigned char* codes_host,
+                                           float* scales_host, int* zeros_host, float* W_hat_host,
+                                           double* loss_host, void* dev_ws, size_t ws_bytes,
+                                           void* stream) {
+  // The whole description is checked before anything is enqueued: the quantizer's own workspace
+  // query rejects every description tb_quantize_layer would reject (it returns 0), and the
+  // tensor-core Hessian needs a width that is a multiple of 8.
+  if (!desc_ok(desc, n_tok, G_host ? g_heads : 0)) return TB_ERR_INVALID_ARG;
+  if (!W_host || !X_host || !codes_host || !scales_host || !zeros_host) return TB_ERR_INVALID_ARG;
+  if (desc->n_hin != 1) return TB_ERR_UNSUPPORTED;  // one shared H_in on this entry point
+  if (desc->d_in % 8) return TB_ERR_INVALID_ARG;
+  if (tb_quantize_layer_workspace(desc, 0, 1) == 0) {
+    // tell an unsupported shape from an invalid one the way tb_quantize_layer does
+    return (desc->d_in % 128 || (desc->quant_group > 0 && desc->quant_group % 32)) ? TB_ERR_UNSUPPORTED
+                                                                                  : TB_ERR_INVALID_ARG;
+  }
+  if (!G_host) g_heads = 0;
+  const HostPlan hs = host_plan(desc, n_tok, g_heads, nullptr);
+  if (!dev_ws || !aligned(dev_ws, 256) || ws_bytes < hs.total) return TB_ERR_WORKSPACE;
+  const HostPlan h = host_plan(desc, n_tok, g_heads, dev_ws);
+  cudaStream_t st = as_stream(stream);
+  const int H = desc->n_heads;
+  SideStream* ss = side_stream();
+  if (!ss) return TB_ERR_CUDA;
+  // earlier work on the caller's stream may still use the buffers: the helper stream starts after it
+  TB_CUDA_CHECK(cudaEventRecord(ss->fork, st));
+  TB_CUDA_CHECK(cudaStreamWaitEvent(ss->stream, ss->fork, 0));
   int info_host[1 + 4096];
   const int n_info = 1 + (H < 4096 ? H : 4096);
-  TB_CUDA_CHECK(cudaMemcpyAsync(info_host, h.info, sizeof(int) * (size_t)n_info, cudaMemcpyDeviceToHost, st));
-  TB_CUDA_CHECK(cudaStreamSynchronize(st));
+  tb_status status = from_host_enqueue(desc, h, ss, W_host, X_host, n_tok, G_host, g_heads, damp_in, damp_out,
+                                       codes_host, scales_host, zeros_host, W_hat_host, loss_host, info_host,
+                                       n_info, stream);
+  // One way out, success or not: the helper stream joins the caller's, and the call waits until
+  // nothing it enqueued (copies from and to the caller's host buffers included) is still in flight.
+  bool sync_ok = cudaEventRecord(ss->join, ss->stream) == cudaSuccess &&
+                 cudaStreamWaitEvent(st, ss->join, 0) == cudaSuccess;
+  sync_ok = (cudaStreamSynchronize(st) == cudaSuccess) && sync_ok;
+  if (!sync_ok) {
+    (void)cudaGetLastError();
+    return status != TB_OK ? status : TB_ERR_CUDA;
+  }
+  if (status != TB_OK) return status;
+  // a bounded wait inside one of the tensor-core kernels ran out: the results are incomplete
+  const int flag = tb_device_error_flag();
+  if (flag != 0) return flag > 0 ? TB_ERR_TIMEOUT : TB_ERR_CUDA;
   for (int i = 0; i < n_info; ++i)
     if (info_host[i] != 0) return TB_ERR_NOT_SPD;
   return TB_OK;

@@ -8,18 +8,20 @@
 
 #include "turboboa.h"
 
+// A failed runtime call leaves its code in the runtime's last-error slot; it is cleared here so
+// that the next, unrelated launch check does not report it again.
 #define TB_CUDA_CHECK(expr)                      \
   do {                                           \
     cudaError_t tb_e_ = (expr);                  \
-    if (tb_e_ != cudaSuccess) return TB_ERR_CUDA; \
+    if (tb_e_ != cudaSuccess) {                  \
+      (void)cudaGetLastError();                  \
+      return TB_ERR_CUDA;                        \
+    }                                            \
   } while (0)
 
 #define TB_LAUNCH_CHECK()                                   \
   do {                                                      \
-    if (cudaPeekAtLastError() != cudaSuccess) {             \
-      (void)cudaGetLastError();                             \
-      return TB_ERR_CUDA;                                   \
-    }                                                       \
+    if (cudaGetLastError() != cudaSuccess) return TB_ERR_CUDA; \
   } while (0)
 
 #define TB_TRY(expr)                   \

@@ -636,11 +636,16 @@ __global__ void __launch_bounds__(RS_THREADS, 1)
         for (int j = 0; j < 32; ++j) {
           // e = (v - s (q - z)) / U_jj = (v / U_jj + s z / U_jj) - (s / U_jj) q, with q = clamp(rne(v / s + z)).
           // The fused multiply-add into z + 1.5 * 2^52 performs the rounding itself and leaves the
-          // integer in the low word of the result (|v / s + z| < 2^31 assumed), where the clamp is
-          // two integer instructions instead of two slow double-precision min / max.
+          // integer in the low word of the result, where the clamp is two integer instructions
+          // instead of two slow double-precision min / max.  The low word alone is the integer only
+          // for |v / s + z| < 2^31; the high word tells (it is the constant's, or one less for a
+          // negative integer, exactly when the low word's sign says the same), and beyond that
+          // range, infinities included, the code saturates like the clamp of the full value.
           const double ard = fma(v, rd_l, szrd_l);
-          int n = __double2loint(fma(v, rs_l, zm_l));
-          n = min(max(n, 0), p.maxq);
+          const double xm = fma(v, rs_l, zm_l);
+          const int lo = __double2loint(xm), hw = __double2hiint(xm) - 0x43380000;
+          int n = min(max(lo, 0), p.maxq);
+          n = (hw == (lo >> 31)) ? n : ((hw >= 0) ? p.maxq : 0);
           const double q = __hiloint2double(0x43380000, n) - magic;
           const double e = fma(-srd_l, q, ard);
           const double ej = shfl_d(e, j);
@@ -1835,7 +1840,7 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
                                        const float* U_in, const float* H_out, const float* U_out,
                                        const float* R, const float* P, const float* C,
                                        unsigned char* codes, float* scales, int* zeros,
-                                       unsigned char* cand, float* W_hat, double* loss,
+                                       unsigned char* cand, float* W_hat, double* W_comp, double* loss,
                                        tb_stats* stats, void* ws, size_t ws_bytes, void* stream) {
   if (!desc || !W || !H_in || !U_in || !codes || !scales || !zeros) return TB_ERR_INVALID_ARG;
   if ((H_out == nullptr) != (U_out == nullptr)) return TB_ERR_INVALID_ARG;
@@ -1936,6 +1941,11 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
       TB_TRY((gemm_launch<double, double, double, double, false, true>(g, st)));
     }
   }
+
+  // A group's rows are never written after they have been taken, and the rows of later groups only by
+  // the compensation of the groups before them: after the loop row r of W~ is what the sweep saw.
+  if (W_comp)
+    TB_CUDA_CHECK(cudaMemcpyAsync(W_comp, p.Wt, (size_t)n_all * sizeof(double), cudaMemcpyDeviceToDevice, st));
 
   // ---- coordinate descent on the scales (Algorithm 3) ----
   if (p.cd) {

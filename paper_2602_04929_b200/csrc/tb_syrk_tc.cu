@@ -246,6 +246,32 @@ int yw_error_read_clear();     // and of the tensor-core product of the scale re
 int cross_error_read_clear();  // and of the deviation correlation (tb_cross_tc.cu)
 }
 
+// One CTA waits on an mbarrier at which nothing ever arrives, through the same bounded wait the
+// tensor-core kernels use, with the given cycle budget: the wait must give up, raise the device
+// error word and let the kernel return.
+namespace tb {
+__global__ void k_bounded_wait_probe(long long budget_cycles, int* __restrict__ gave_up) {
+  __shared__ unsigned long long bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag = 0;
+    mbar_fence_init();
+  }
+  __syncthreads();
+  const bool ok = mbar_wait(smem_u32(&bar), 0u, &abort_flag, &g_tc_error, budget_cycles);
+  __syncthreads();
+  if (threadIdx.x == 0 && gave_up) *gave_up = ok ? 0 : 1;
+}
+}  // namespace tb
+
+extern "C" tb_status tb_selftest_bounded_wait(long long budget_cycles, int* gave_up, void* stream) {
+  if (budget_cycles < 0 || budget_cycles > 200000000ll) return TB_ERR_INVALID_ARG;  // at most ~0.1 s
+  tb::k_bounded_wait_probe<<<1, 64, 0, tb::as_stream(stream)>>>(budget_cycles, gave_up);
+  TB_LAUNCH_CHECK();
+  return TB_OK;
+}
+
 extern "C" int tb_device_error_flag(void) {
   int v = 0;
   if (cudaMemcpyFromSymbol(&v, tb::g_tc_error, sizeof(int)) != cudaSuccess) return -1;

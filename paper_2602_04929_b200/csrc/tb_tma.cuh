@@ -34,15 +34,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait: gives up after about two seconds (or as soon as another thread of the CTA has
-// given up), raises *abort_flag and the device error word, and reports failure.
+// Bounded wait: gives up after `budget` clock cycles (about two seconds by default), or as soon as
+// another thread of the CTA has given up, raises *abort_flag and the device error word, and
+// reports failure.
+enum : long long { MBAR_WAIT_BUDGET = 4000000000ll };
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          int* device_error_word) {
+                                          int* device_error_word, long long budget = MBAR_WAIT_BUDGET) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   while (!mbar_try_wait(bar, parity)) {
     if (*abort_flag) return false;
-    if (clock64() - t0 > 4000000000ll) {
+    if (clock64() - t0 > budget) {
       *abort_flag = 1;
       atomicExch(device_error_word, 1);
       return false;

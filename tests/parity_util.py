@@ -15,81 +15,12 @@ from __future__ import annotations
 import numpy as np
 
 import oracle
-import tb_inputs
+from oracle.problems import cached_problem, f32, make_problem, oracle_desc  # noqa: F401
 
 BAND = 1e-6        # code units; the band inside which a rounding decision may differ
 CAND_TOL = 1e-9    # relative score gap below which two grid candidates count as tied
-TOL_W = 1e-5       # relative Frobenius error on W_hat and on the scales
+TOL_W = 1e-5       # relative Frobenius error on W_hat, on the scales and on the compensated weights
 TOL_LOSS = 1e-4    # relative error on the Hessian-weighted loss
-
-
-def f32(a):
-    return None if a is None else np.ascontiguousarray(a, dtype=np.float32)
-
-
-def make_problem(seed, d_in, n_heads, d_head, n_tok, *, with_r=False, hout="proj", n_hin=1,
-                 g_heads=None, damp=0.01, alpha=0.25, gaussian_x=False, vmix_seq=None):
-    """float32 inputs of one projection, every derived tensor computed by the oracle."""
-    d_out = n_heads * d_head
-    W = tb_inputs.weight(seed, d_out, d_in)
-    Hin, Uin, Hsum, R, P, C = [], [], [], [], [], []
-    for u in range(n_hin):
-        if vmix_seq:
-            # value projection: head u sees the attention-weighted inputs A_u X of the same tokens
-            base = tb_inputs.HeavyTailRecipe(d_in, seed=seed).chunk(0, n_tok)
-            X, Xfp = tb_inputs.causal_decay_mix(base, tb_inputs.decay_rate(u), vmix_seq), None
-        elif gaussian_x:
-            X = tb_inputs.activations_gaussian(seed + 101 * u, n_tok, d_in)
-            Xfp = None
-        else:
-            rec = tb_inputs.HeavyTailRecipe(d_in, seed=seed, tid_shift=u)
-            if with_r:
-                X, Xfp = tb_inputs.DeviationRecipe(rec).chunk(0, n_tok)
-            else:
-                X, Xfp = rec.chunk(0, n_tok), None
-        H, Hs = oracle.hessian(X, damp=damp, return_sum=True)
-        H32 = f32(H)
-        Hin.append(H32)
-        Hsum.append(f32(Hs))
-        U32 = f32(oracle.factor_upper(H32))
-        Uin.append(U32)
-        if with_r:
-            R32 = f32(oracle.cross_correlation(X, Xfp, alpha))
-            Pm, Cm = oracle.correction_operands(R32, U32)
-            R.append(R32)
-            P.append(f32(Pm))
-            C.append(f32(Cm))
-    prob = dict(W=W, Hin=np.stack(Hin), Uin=np.stack(Uin), Hsum=Hsum[0], d_out=d_out, d_in=d_in,
-                n_heads=n_heads, d_head=d_head, n_hin=n_hin, R=None, P=None, C=None, Hout=None, Uout=None)
-    if with_r:
-        prob.update(R=np.stack(R), P=np.stack(P), C=np.stack(C))
-    if hout == "proj":
-        gh = g_heads or n_heads
-        G = tb_inputs.weight(seed, gh * d_head, d_in, tid=tb_inputs.T_WPARTNER)
-        Ho = f32(oracle.hout_from_projection(G, Hsum[0], n_heads, d_head, damp=damp))
-        prob.update(G=G, Hout=Ho, Uout=f32(oracle.factor_upper(Ho)))
-    elif hout == "spd":
-        Ho = np.stack([tb_inputs.spd_matrix(seed + h, d_head, cond=1e3) for h in range(n_heads)])
-        prob.update(Hout=Ho, Uout=f32(oracle.factor_upper(Ho)))
-    return prob
-
-
-_PROBLEMS = {}
-
-
-def cached_problem(*args, **kw):
-    """make_problem, kept for the tests of one process that share a large problem (read-only use)."""
-    key = (args, tuple(sorted(kw.items())))
-    if key not in _PROBLEMS:
-        _PROBLEMS[key] = make_problem(*args, **kw)
-    return _PROBLEMS[key]
-
-
-def oracle_desc(prob, bits, quant_group, out_block, flags, n_cand=16, cd_iters=1, n_heads=None):
-    H = n_heads or prob["n_heads"]
-    return oracle.OracleDesc(d_out=H * prob["d_head"], d_in=prob["d_in"], n_heads=H, d_head=prob["d_head"],
-                             bits=bits, quant_group=quant_group, out_block=out_block,
-                             n_hin=1 if prob["n_hin"] == 1 else H, n_cand=n_cand, cd_iters=cd_iters, flags=flags)
 
 
 def run_gpu(prob, bits, quant_group, out_block, flags, n_cand=16, cd_iters=1, want_loss=True):
@@ -104,11 +35,11 @@ def run_gpu(prob, bits, quant_group, out_block, flags, n_cand=16, cd_iters=1, wa
     desc = tb.layer_desc(prob["d_out"], prob["d_in"], prob["n_heads"], prob["d_head"], bits, quant_group,
                          out_block, n_hin=prob["n_hin"], n_cand=n_cand, cd_iters=cd_iters, flags=flags)
     res = tb.tb_quantize_layer(desc, t(prob["W"]), t(prob["Hin"]), t(prob["Uin"]), t(prob["Hout"]),
-                               t(prob["Uout"]), t(prob["R"]), t(prob["P"]), t(prob["C"]), want_loss=want_loss)
+                               t(prob["Uout"]), t(prob["R"]), t(prob["P"]), t(prob["C"]), want_loss=want_loss, want_w_comp=True)
     torch.cuda.synchronize()
     assert tb.tb_device_error_flag() == 0, "a bounded device-side wait ran out"
     return dict(codes=res.codes.cpu().numpy(), scales=res.scales.cpu().numpy(), zeros=res.zeros.cpu().numpy(),
-                cand=res.cand.cpu().numpy(), w_hat=res.w_hat.cpu().numpy(),
+                cand=res.cand.cpu().numpy(), w_hat=res.w_hat.cpu().numpy(), w_comp=res.w_comp.cpu().numpy(),
                 loss=None if res.loss is None else res.loss.cpu().numpy(), stats=res.stats_dict())
 
 
@@ -156,6 +87,8 @@ def compare(prob, gpu, bits, quant_group, out_block, flags, n_cand=16, cd_iters=
     rep["cand_mismatch"] = int(np.count_nonzero(gpu["cand"][rows] != res.cand))
     rep["scales_rel"] = rel_fro(gpu["scales"][rows], res.scales)
     rep["w_hat_rel"] = rel_fro(gpu["w_hat"][rows], res.w_hat)
+    # compensated weights: every row as it stood when its group was taken (the oracle's snapshot W0)
+    rep["w_comp_rel"] = rel_fro(gpu["w_comp"][rows], res.w_comp)
     if gpu["loss"] is not None:
         lg, lo = gpu["loss"][hsel], res.loss
         rep["loss_rel"] = float(np.max(np.abs(lg - lo) / np.maximum(np.abs(lo), 1e-300)))
@@ -169,6 +102,7 @@ def compare(prob, gpu, bits, quant_group, out_block, flags, n_cand=16, cd_iters=
     assert rep["cand_mismatch"] == 0, rep
     assert rep["scales_rel"] <= TOL_W, rep
     assert rep["w_hat_rel"] <= TOL_W, rep
+    assert rep["w_comp_rel"] <= TOL_W, rep
     if "loss_rel" in rep:
         assert rep["loss_rel"] <= TOL_LOSS, rep
     return rep

@@ -226,3 +226,26 @@ def test_prerequisites_at_full_width():
     assert errs["U_in"] <= 1e-6 and errs["U_out"] <= 1e-6
     assert errs["P"] <= 1e-5 and errs["C"] <= 1e-5
     assert errs["H_out"] <= 2e-6
+
+
+def test_bounded_wait_gives_up_and_leaves_the_context_usable():
+    """A wait on a hardware barrier at which nothing ever arrives, with a budget of about 1 ms: the
+    kernel must return by itself, the device error word must be raised (and cleared by reading it),
+    and the next real call must be clean."""
+    import torch
+    import paper_2602_04929_b200 as tb
+    assert tb.tb_device_error_flag() == 0
+    gave_up = torch.zeros(1, dtype=torch.int32, device="cuda:0")
+    tb.tb_selftest_bounded_wait(2_000_000, gave_up)
+    torch.cuda.synchronize()
+    assert int(gave_up.item()) == 1
+    assert tb.tb_device_error_flag() == 1
+    assert tb.tb_device_error_flag() == 0          # reading it cleared it
+    # the context is intact: a tensor-core Hessian right after it, against the oracle
+    X = tb_inputs.HeavyTailRecipe(128, seed=9).chunk(0, 4096)
+    H = torch.zeros((128, 128), dtype=torch.float32, device="cuda:0")
+    tb.tb_accumulate_hessian(H, _t(X, torch.bfloat16))
+    tb.tb_finalize_hessian(H, None, 4096, 0.01)
+    torch.cuda.synchronize()
+    assert tb.tb_device_error_flag() == 0
+    assert rel_fro(H.cpu().numpy(), oracle.hessian(X, damp=0.01)) <= 1e-5

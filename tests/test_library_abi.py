@@ -61,7 +61,7 @@ def test_bad_descriptions_are_rejected_on_the_host():
 
     def call(desc, ws=one, ws_bytes=1 << 40, H_out=None, U_out=None):
         return lib.tb_quantize_layer(ctypes.byref(desc), one, one, one, H_out, U_out, None, None, None,
-                                     one, one, one, None, None, None, None, ws, ws_bytes, None)
+                                     one, one, one, None, None, None, None, None, ws, ws_bytes, None)
 
     ok = dict(d_out=256, d_in=256, n_heads=2, d_head=128, bits=4, quant_group=128, out_block=8)
     bad = [dict(ok, n_heads=3), dict(ok, bits=1), dict(ok, bits=9), dict(ok, quant_group=100),
@@ -84,3 +84,29 @@ def test_bad_descriptions_are_rejected_on_the_host():
     assert lib.tb_factor(one, 0, 64, one, None, one, one, 1 << 40, None) == 1
     assert lib.tb_prepare_correction(one, one, 1, 64, one, one, one, 16, None) == 3
     assert lib.tb_build_hout(one, one, None, 3, 2, 64, 128, 0.0, one, 1 << 40, None) == 1
+
+
+def test_host_entry_point_validates_the_whole_description_first():
+    """tb_quantize_from_host must reject everything tb_quantize_layer would reject before it
+    enqueues a copy (the pointers below are never dereferenced)."""
+    lib = tb.load()
+    one = ctypes.c_void_p(256)
+
+    def call(desc, n_tok=4096, g_heads=2, G=one, ws=one, ws_bytes=1 << 40):
+        return lib.tb_quantize_from_host(ctypes.byref(desc), one, one, n_tok, G, g_heads, 0.01, 0.01,
+                                         one, one, one, None, None, ws, ws_bytes, None)
+
+    ok = dict(d_out=256, d_in=256, n_heads=2, d_head=128, bits=4, quant_group=128, out_block=8)
+    for kw in [dict(ok, bits=1), dict(ok, bits=9), dict(ok, out_block=7), dict(ok, out_block=0),
+               dict(ok, n_cand=0), dict(ok, n_cand=33), dict(ok, cd_iters=-1), dict(ok, n_heads=3),
+               dict(ok, quant_group=100)]:
+        assert call(tb.layer_desc(**kw)) == 1, kw
+    assert call(tb.layer_desc(**dict(ok, quant_group=16))) == 2
+    assert call(tb.layer_desc(**dict(ok, d_in=192, quant_group=0))) == 2
+    assert call(tb.layer_desc(**dict(ok, n_hin=2))) == 2
+    assert call(tb.layer_desc(**ok), n_tok=0) == 1
+    assert call(tb.layer_desc(**ok), g_heads=3) == 1
+    assert call(tb.layer_desc(**ok), ws=None) == 3
+    assert call(tb.layer_desc(**ok), ws_bytes=4096) == 3
+    assert lib.tb_selftest_bounded_wait(-1, None, None) == 1
+    assert lib.tb_selftest_bounded_wait(10 ** 10, None, None) == 1

@@ -50,6 +50,17 @@ def test_static_scratch_factor_matches_tb_factor_twice():
             assert _rel(U[b].cpu().numpy(), U_ref[b].cpu().numpy()) <= 1e-6
         assert torch.equal(U, U_ref)
         assert torch.equal(torch.tril(U, -1), torch.zeros_like(U))
+        # the array exists by now (the call above was at least the first on this device): one more call
+        # must leave the device's free memory exactly as it found it
+        free_before, _ = torch.cuda.mem_get_info(dev)
+        st = lib.tb_factor_static(ctypes.c_void_p(Hd.data_ptr()), n_batch, d, ctypes.c_void_p(U.data_ptr()),
+                                  ctypes.c_void_p(info.data_ptr()),
+                                  ctypes.c_void_p(torch.cuda.current_stream().cuda_stream))
+        assert st == 0, tb.status_string(st)
+        torch.cuda.synchronize()
+        free_after, _ = torch.cuda.mem_get_info(dev)
+        assert free_after == free_before
+        assert torch.equal(U, U_ref)
 
 
 def test_static_scratch_rejects_what_does_not_fit():
