@@ -255,12 +255,109 @@ tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W, const flo
                             float* W_hat, double* W_comp, double* loss, tb_stats* stats, void* ws,
                             size_t ws_bytes, void* stream);
 
+/* --------------------------------------------------------------------------
+ * Block level: Algorithm 1's outer loop over the projections of an attention
+ * layer.
+ * -------------------------------------------------------------------------- */
+
+/* One prepared projection: exactly the arguments of tb_quantize_layer. */
+typedef struct {
+  tb_layer_desc desc;
+  const float *W, *H_in, *U_in, *H_out, *U_out, *R, *P, *C;
+  unsigned char* codes;
+  float* scales;
+  int* zeros;
+  unsigned char* cand;
+  float* W_hat;
+  double* W_comp;
+  double* loss;
+  tb_stats* stats;
+  void* ws;
+  size_t ws_bytes;
+} tb_projection_job;
+
+/* Quantizes up to 5 prepared projections (Algorithm 1 loops over W_Q, W_K, W_V;
+ * heads and projections are independent problems).  concurrent = 0: one after
+ * the other on `stream`.  concurrent != 0: job 0 on `stream`, the others on
+ * helper streams of the library (per device, created at the first such call and
+ * kept until exit), forked from and joined back into `stream` by events, so that
+ * the latency-bound phases of one projection run beside the throughput-bound
+ * phases of another; every job then needs a workspace of its own.  Results are
+ * those of separate tb_quantize_layer calls, bit for bit.  All descriptions and
+ * workspaces are checked before the first launch. */
+tb_status tb_quantize_block(const tb_projection_job* jobs, int n_jobs, int concurrent, void* stream);
+
+/* A whole attention layer from its calibration activations (Algorithm 1 for
+ * W_Q, W_K, W_V, and the output projection in the H_out = I mode of Table 1's
+ * GPTQ row). */
+typedef struct {
+  int d_model;     /* width d of the attention input; W_Q, W_K, W_V have d columns  */
+  int n_q_heads;   /* W_Q is [n_q_heads * d_head][d]; W_O is [d][n_q_heads * d_head] */
+  int n_kv_heads;  /* W_K, W_V are [n_kv_heads * d_head][d]; divides n_q_heads
+                      (grouped-query attention when smaller)                        */
+  int d_head;
+  int bits, quant_group, out_block, n_cand, cd_iters; /* as in tb_layer_desc        */
+  unsigned flags;  /* TB_F_*                                                        */
+  long long n_tok; /* calibration tokens in every activation tensor                 */
+  float damp;      /* damping of every Hessian built here (see tb_finalize_hessian) */
+  float alpha;     /* stabilisation coefficient of R (Algorithm 1, deviation step)  */
+  int on_host;     /* 0: every pointer of tb_attention_io is device memory;
+                      1: every pointer is host memory (pinned memory makes the
+                      copies asynchronous) and the call synchronises `stream`      */
+  int concurrent;  /* != 0: independent parts on helper streams side by side        */
+} tb_attention_desc;
+
+typedef struct {
+  /* activations, bf16, token-major */
+  const void* X;      /* [n_tok][d]  input of W_Q, W_K, W_V on the quantized path                  */
+  const void* X_fp;   /* same shape or NULL: the full-precision path's input X~; when given,
+                         R = alpha (X - X~) X^T enters W_Q and W_K (and W_V if X_v is NULL)       */
+  const void* X_v;    /* [n_kv_heads][n_tok][d] or NULL: the attention-weighted inputs A_h X of
+                         the value projection, one H_in per head (Table 1, W_V row; no R then);
+                         NULL: W_V shares the Hessian of X                                        */
+  const void* X_o;    /* [n_tok][n_q_heads * d_head]  input of the output projection             */
+  const void* X_o_fp; /* same shape or NULL: its full-precision twin (R of the output projection) */
+  /* weights, float, in the order q, k, v, o */
+  const float* W[4];
+  /* results per projection, same order; W_hat and loss entries may be NULL */
+  unsigned char* codes[4];
+  float* scales[4];
+  int* zeros[4];
+  float* W_hat[4];
+  double* loss[4];    /* [n_heads] of that projection (1 for the output projection)               */
+  int* info;          /* tb_attention_layer_info_count ints or NULL: the info words of every
+                         factorisation (H_in of X, of X_o, of each X_v head, then H_out of the
+                         q, k, v heads); 0 = positive definite                                    */
+} tb_attention_io;
+
+/* H_out follows Table 1: W_Q against K_h^T K_h (from W_K and the Hessian of X),
+ * W_K against Q_h^T Q_h (from W_Q), W_V against W_out,h^T W_out,h (the head's
+ * columns of W_O); with grouped-query attention a query head takes the block of
+ * its key/value head and a key/value head the sum over its query heads.  The
+ * output projection runs with H_out = NULL (all rows at once, GPTAQ if X_o_fp
+ * is given).  The workspace query only looks at which optional pointers of io
+ * are non-NULL.  With on_host = 1 the activations cross to the device in pieces
+ * of 16384 tokens on a copy stream while the Hessian of the pieces already there
+ * accumulates (the Hessian's sums do not depend on the pieces; the deviation
+ * correlation adds its two bf16 pieces per call, so its float sums differ from a
+ * single call's in the last bits), results are copied back, and the call returns TB_ERR_NOT_SPD /
+ * TB_ERR_TIMEOUT like tb_quantize_from_host; with on_host = 0 it only enqueues
+ * and the caller reads `info`.  Helper streams as for tb_quantize_block. */
+int tb_attention_layer_info_count(const tb_attention_desc* desc, int per_head_v);
+size_t tb_attention_layer_workspace(const tb_attention_desc* desc, const tb_attention_io* io);
+tb_status tb_attention_layer(const tb_attention_desc* desc, const tb_attention_io* io, void* ws,
+                             size_t ws_bytes, void* stream);
+
 /* Profiling aid with no counterpart in the paper.  While enabled, every
  * tb_quantize_layer call records CUDA events on its stream around its phases;
  * tb_profile_read waits for them, adds the elapsed milliseconds per phase into
  * ms_by_phase[0..n) (host memory; order: setup, grid search, column sweep,
- * compensation, coordinate descent, output, loss), forgets them and returns the
- * number of phases (7).  Process-wide and not thread-safe; off by default. */
+ * compensation, coordinate descent, output, loss, then the prerequisites as
+ * tb_attention_layer runs them: Hessian accumulation, deviation correlation,
+ * H_out build, factorisations, propagated-error operands, result copies),
+ * forgets them and returns the number of phases (13).  Phases that ran side by
+ * side on different streams each count their own elapsed time.  Process-wide
+ * and not thread-safe; off by default. */
 void tb_profile_enable(int on);
 int tb_profile_read(double* ms_by_phase, int n);
 

@@ -72,6 +72,10 @@ _SIGNATURES = {
     "tb_prepare_correction": (_int, [_vp, _vp, _int, _int, _vp, _vp, _vp, _sz, _vp]),
     "tb_quantize_layer_workspace": (_sz, [ctypes.POINTER(LayerDesc), _int, _int]),
     "tb_quantize_layer": (_int, [ctypes.POINTER(LayerDesc)] + [_vp] * 16 + [_vp, _sz, _vp]),
+    "tb_quantize_block": (_int, [_vp, _int, _int, _vp]),
+    "tb_attention_layer_info_count": (_int, [_vp, _int]),
+    "tb_attention_layer_workspace": (_sz, [_vp, _vp]),
+    "tb_attention_layer": (_int, [_vp, _vp, _vp, _sz, _vp]),
     "tb_profile_enable": (None, [_int]),
     "tb_profile_read": (_int, [ctypes.POINTER(ctypes.c_double), _int]),
     "tb_quantize_from_host_workspace": (_sz, [ctypes.POINTER(LayerDesc), _ll, _int]),
@@ -312,7 +316,128 @@ def tb_quantize_from_host(desc: LayerDesc, W_host, X_host, G_host, damp_in: floa
         "tb_quantize_from_host")
 
 
-PHASES = ("setup", "grid", "sweep", "compensation", "cd", "output", "loss")
+class ProjectionJob(ctypes.Structure):
+    """tb_projection_job"""
+    _fields_ = ([("desc", LayerDesc)] +
+                [(n, ctypes.c_void_p) for n in ("W", "H_in", "U_in", "H_out", "U_out", "R", "P", "C", "codes", "scales",
+                                                "zeros", "cand", "W_hat", "W_comp", "loss", "stats", "ws")] +
+                [("ws_bytes", ctypes.c_size_t)])
+
+
+class AttentionDesc(ctypes.Structure):
+    """tb_attention_desc"""
+    _fields_ = [("d_model", ctypes.c_int), ("n_q_heads", ctypes.c_int), ("n_kv_heads", ctypes.c_int),
+                ("d_head", ctypes.c_int), ("bits", ctypes.c_int), ("quant_group", ctypes.c_int),
+                ("out_block", ctypes.c_int), ("n_cand", ctypes.c_int), ("cd_iters", ctypes.c_int),
+                ("flags", ctypes.c_uint), ("n_tok", ctypes.c_longlong), ("damp", ctypes.c_float),
+                ("alpha", ctypes.c_float), ("on_host", ctypes.c_int), ("concurrent", ctypes.c_int)]
+
+
+class AttentionIO(ctypes.Structure):
+    """tb_attention_io"""
+    _fields_ = [("X", ctypes.c_void_p), ("X_fp", ctypes.c_void_p), ("X_v", ctypes.c_void_p), ("X_o", ctypes.c_void_p),
+                ("X_o_fp", ctypes.c_void_p), ("W", ctypes.c_void_p * 4), ("codes", ctypes.c_void_p * 4),
+                ("scales", ctypes.c_void_p * 4), ("zeros", ctypes.c_void_p * 4), ("W_hat", ctypes.c_void_p * 4),
+                ("loss", ctypes.c_void_p * 4), ("info", ctypes.c_void_p)]
+
+
+def attention_desc(d_model, n_q_heads, n_kv_heads, d_head, bits, quant_group, out_block, n_tok, n_cand=16, cd_iters=1,
+                   flags=0, damp=0.01, alpha=0.25, on_host=False, concurrent=True) -> AttentionDesc:
+    return AttentionDesc(d_model, n_q_heads, n_kv_heads, d_head, bits, quant_group, out_block, n_cand, cd_iters, flags,
+                         int(n_tok), float(damp), float(alpha), int(on_host), int(concurrent))
+
+
+def projection_job(desc: LayerDesc, W, H_in, U_in, H_out, U_out, R, P, C, out: "QuantizeResult", ws) -> ProjectionJob:
+    """tb_projection_job from torch CUDA tensors (argument marshalling only; the caller keeps them alive)."""
+    f32 = torch.float32
+
+    def v(t, dt=None):
+        q = _ptr(t, dt, True)
+        return None if q is None else q.value
+
+    return ProjectionJob(desc, v(W, f32), v(H_in, f32), v(U_in, f32), v(H_out, f32), v(U_out, f32), v(R, f32), v(P, f32),
+                         v(C, f32), v(out.codes), v(out.scales), v(out.zeros), v(out.cand), v(out.w_hat),
+                         v(out.w_comp, torch.float64), v(out.loss), v(out.stats), v(ws), ws.numel())
+
+
+def tb_quantize_block(jobs: list, concurrent: bool = True) -> None:
+    arr = (ProjectionJob * len(jobs))(*jobs)
+    _check(load().tb_quantize_block(ctypes.cast(arr, ctypes.c_void_p), len(jobs), int(bool(concurrent)), _stream()),
+           "tb_quantize_block")
+
+
+def empty_result(desc: LayerDesc, device, want_loss=True, want_w_comp=False) -> "QuantizeResult":
+    ng = desc.n_groups
+    return QuantizeResult(
+        codes=torch.empty((desc.d_out, desc.d_in), dtype=torch.uint8, device=device),
+        scales=torch.empty((desc.d_out, ng), dtype=torch.float32, device=device),
+        zeros=torch.empty((desc.d_out, ng), dtype=torch.int32, device=device),
+        cand=torch.empty((desc.d_out, ng), dtype=torch.uint8, device=device),
+        w_hat=torch.empty((desc.d_out, desc.d_in), dtype=torch.float32, device=device),
+        loss=torch.empty(desc.n_heads, dtype=torch.float64, device=device) if want_loss else None,
+        stats=torch.zeros(8, dtype=torch.int64, device=device),
+        w_comp=torch.empty((desc.d_out, desc.d_in), dtype=torch.float64, device=device) if want_w_comp else None)
+
+
+def attention_io(desc: AttentionDesc, X, X_o, W, out, X_fp=None, X_v=None, X_o_fp=None, info=None) -> AttentionIO:
+    """tb_attention_io from torch tensors: all on the device (desc.on_host = 0) or all on the host.
+    W: the four weights q, k, v, o; out: four dicts with codes, scales, zeros and optionally w_hat, loss."""
+    host = bool(desc.on_host)
+
+    def v(t):
+        if t is None:
+            return None
+        if t.is_cuda == host or not t.is_contiguous():
+            raise ValueError("tensors must be contiguous and all on the %s" % ("host" if host else "device"))
+        return t.data_ptr()
+
+    io = AttentionIO()
+    io.X, io.X_fp, io.X_v, io.X_o, io.X_o_fp, io.info = v(X), v(X_fp), v(X_v), v(X_o), v(X_o_fp), v(info)
+    for i in range(4):
+        io.W[i] = v(W[i])
+        io.codes[i], io.scales[i], io.zeros[i] = v(out[i]["codes"]), v(out[i]["scales"]), v(out[i]["zeros"])
+        io.W_hat[i], io.loss[i] = v(out[i].get("w_hat")), v(out[i].get("loss"))
+    return io
+
+
+def attention_layer_shapes(desc: AttentionDesc):
+    """(d_out, d_in, n_heads) of the q, k, v, o projections."""
+    dq, dkv = desc.n_q_heads * desc.d_head, desc.n_kv_heads * desc.d_head
+    return [(dq, desc.d_model, desc.n_q_heads), (dkv, desc.d_model, desc.n_kv_heads),
+            (dkv, desc.d_model, desc.n_kv_heads), (desc.d_model, dq, 1)]
+
+
+def attention_outputs(desc: AttentionDesc, device=None, pin=False, w_hat=True, loss=True):
+    """Result buffers of tb_attention_layer, on `device` or (device None) on the host."""
+    outs = []
+    for d_out, d_in, heads in attention_layer_shapes(desc):
+        ng = 1 if desc.quant_group == 0 else d_in // desc.quant_group
+        o = {"codes": torch.empty((d_out, d_in), dtype=torch.uint8, device=device),
+             "scales": torch.empty((d_out, ng), dtype=torch.float32, device=device),
+             "zeros": torch.empty((d_out, ng), dtype=torch.int32, device=device)}
+        if w_hat:
+            o["w_hat"] = torch.empty((d_out, d_in), dtype=torch.float32, device=device)
+        if loss:
+            o["loss"] = torch.empty(heads, dtype=torch.float64, device=device)
+        outs.append({k: (t.pin_memory() if pin else t) for k, t in o.items()})
+    return outs
+
+
+def tb_attention_layer_info_count(desc: AttentionDesc, per_head_v: bool) -> int:
+    return int(load().tb_attention_layer_info_count(ctypes.byref(desc), int(bool(per_head_v))))
+
+
+def tb_attention_layer_workspace(desc: AttentionDesc, io: AttentionIO) -> int:
+    return int(load().tb_attention_layer_workspace(ctypes.byref(desc), ctypes.byref(io)))
+
+
+def tb_attention_layer(desc: AttentionDesc, io: AttentionIO, ws) -> None:
+    _check(load().tb_attention_layer(ctypes.byref(desc), ctypes.byref(io), _ptr(ws), ws.numel(), _stream()),
+           "tb_attention_layer")
+
+
+PHASES = ("setup", "grid", "sweep", "compensation", "cd", "output", "loss",
+          "hessian", "cross", "hout", "factor", "prep", "copy")
 
 
 def tb_profile_enable(on: bool) -> None:

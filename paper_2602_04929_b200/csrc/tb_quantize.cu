@@ -19,6 +19,7 @@
 
 #include "tb_common.cuh"
 #include "tb_gemm.cuh"
+#include "tb_profile.cuh"
 #include "tb_tma.cuh"
 
 namespace cg = cooperative_groups;
@@ -1660,39 +1661,6 @@ static int ew_blocks(long long n) {
   return (int)b;
 }
 
-// ---------------------------------------------------------------------------
-// Optional phase timing (tb_profile_enable / tb_profile_read): CUDA events on
-// the launching stream around each phase of tb_quantize_layer.
-// ---------------------------------------------------------------------------
-enum { PH_SETUP = 0, PH_GRID, PH_SWEEP, PH_COMP, PH_CD, PH_OUTPUT, PH_LOSS, PH_COUNT };
-struct PhaseSpan {
-  int phase;
-  cudaEvent_t a, b;
-};
-static bool g_profile_on = false;
-static PhaseSpan g_spans[4096];
-static int g_n_spans = 0;
-
-struct PhaseScope {
-  int idx;
-  cudaStream_t st;
-  PhaseScope(int phase, cudaStream_t s) : idx(-1), st(s) {
-    if (!g_profile_on || g_n_spans >= 4096) return;
-    PhaseSpan& sp = g_spans[g_n_spans];
-    if (cudaEventCreate(&sp.a) != cudaSuccess) return;
-    if (cudaEventCreate(&sp.b) != cudaSuccess) {
-      cudaEventDestroy(sp.a);
-      return;
-    }
-    sp.phase = phase;
-    idx = g_n_spans++;
-    cudaEventRecord(sp.a, st);
-  }
-  ~PhaseScope() {
-    if (idx >= 0) cudaEventRecord(g_spans[idx].b, st);
-  }
-};
-
 static tb_status run_grid(const Plan& p, const float* H_in, float* scales, int* zeros,
                           unsigned char* cand, RowMap rm, int M, cudaStream_t st) {
   GridP gp;
@@ -1803,6 +1771,12 @@ static tb_status run_sweep_rows(const Plan& p, const float* U_in, const float* P
 }  // namespace tb
 
 using namespace tb;
+
+namespace tb {
+bool g_profile_on = false;
+PhaseSpan g_spans[TB_MAX_SPANS];
+int g_n_spans = 0;
+}  // namespace tb
 
 extern "C" void tb_profile_enable(int on) {
   for (int i = 0; i < g_n_spans; ++i) {
