@@ -256,6 +256,42 @@ tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W, const flo
                             size_t ws_bytes, void* stream);
 
 /* --------------------------------------------------------------------------
+ * Bit-packed integer weights.  Section 2.1 writes the quantized weight as
+ * Q = diag(s) W_int with W_int in {0 .. 2^b - 1}: what is stored and shipped is
+ * W_int at b bits per weight, with the scales (and here the zero-points).
+ * -------------------------------------------------------------------------- */
+
+/* Packed format: every row is a little-endian bit stream; code j of the row
+ * occupies bits [j b, (j + 1) b), counted from the least significant bit of the
+ * row's first 32-bit word (a code may straddle two words when b does not divide
+ * 32).  A row takes d_in * b / 32 words; d_in must be a multiple of 32.
+ * tb_packed_bytes: size of the packed matrix, 0 for an invalid shape.
+ * tb_pack_codes: codes [d_out][d_in] unsigned char (16-byte aligned, values
+ * below 2^bits) -> packed.  bits in 2..8. */
+size_t tb_packed_bytes(int d_out, int d_in, int bits);
+tb_status tb_pack_codes(const unsigned char* codes, int d_out, int d_in, int bits,
+                        unsigned int* packed, void* stream);
+
+/* Unpacks, dequantizes and optionally compares in one pass over the packed
+ * matrix: Q[r][j] = scales[r][g] * (code - zeros[r][g]) in float, g = j /
+ * quant_group (the final step of Algorithm 1 from what a deployment holds:
+ * packed codes, float scales, integer zero-points).
+ *   codes_out, W_hat_out  [d_out][d_in], either may be NULL
+ *   codes_ref             or NULL: unpacked codes are compared byte for byte
+ *   W_hat_ref             or NULL: |Q - ref| <= tol * |ref| is checked per
+ *                         element (tb_quantize_layer forms W_hat from the scales
+ *                         in double and rounds once, so the two may differ by an
+ *                         ulp: tol = 2^-22 passes, 0 asks for equal bits)
+ *   mismatch              device, 2 words, required when a reference is given:
+ *                         [0] codes that differ, [1] values beyond tol; cleared
+ *                         by the call */
+tb_status tb_unpack_dequant(const unsigned int* packed, const float* scales, const int* zeros,
+                            int d_out, int d_in, int bits, int quant_group,
+                            unsigned char* codes_out, float* W_hat_out,
+                            const unsigned char* codes_ref, const float* W_hat_ref, float tol,
+                            unsigned long long* mismatch, void* stream);
+
+/* --------------------------------------------------------------------------
  * Block level: Algorithm 1's outer loop over the projections of an attention
  * layer.
  * -------------------------------------------------------------------------- */
@@ -360,6 +396,11 @@ tb_status tb_attention_layer(const tb_attention_desc* desc, const tb_attention_i
  * and not thread-safe; off by default. */
 void tb_profile_enable(int on);
 int tb_profile_read(double* ms_by_phase, int n);
+
+/* Number of kernels the library has launched in this process so far (every launch
+ * of one of its own kernels counts once; copies and memsets do not).  Not
+ * thread-safe.  No counterpart in the paper. */
+unsigned long long tb_launch_count(void);
 
 /* Whole path for one projection from HOST buffers: copies X (and G) to the
  * device, accumulates and finalises H_in, builds H_out, factors both, runs

@@ -25,6 +25,9 @@ from .ref import (  # noqa: F401
     loss_head,
     group_loop_trace,
     num_threads,
+    pack_codes,
+    unpack_codes,
+    dequantize,
     F_ADAPTIVE_GRID,
     F_CD_REFINE,
 )

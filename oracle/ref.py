@@ -314,3 +314,46 @@ def group_loop_trace(desc: OracleDesc, W, Hin, Uin, Uout=None, P=None, C=None):
                              _p(codes, ctypes.c_ubyte), _p(scales), _p(zeros, ctypes.c_int), _p(Q),
                              _p(w_comp), _p(trace))
     return dict(codes=codes, scales=scales, zeros=zeros, Q=Q, w_comp=w_comp, trace=trace)
+
+
+# ----------------------------------------------------------------------------
+# Packed integer weights (Section 2.1: Q = diag(s) W_int, W_int in {0 .. 2^b - 1})
+# ----------------------------------------------------------------------------
+
+def pack_codes(codes, bits: int):
+    """Row-wise little-endian bit stream: code j of a row in bits [j b, (j + 1) b) from the least
+    significant bit of the row's first 32-bit word.  Written bit by bit (one boolean per stream bit)."""
+    codes = np.ascontiguousarray(codes, np.uint8)
+    d_out, d_in = codes.shape
+    if (d_in * bits) % 32:
+        raise ValueError("a row must fill whole 32-bit words")
+    stream = np.zeros((d_out, d_in, bits), np.uint8)
+    for k in range(bits):
+        stream[:, :, k] = (codes >> k) & 1          # bit k of code j is stream bit j * bits + k
+    stream = stream.reshape(d_out, d_in * bits // 32, 32).astype(np.uint64)
+    words = np.zeros(stream.shape[:2], np.uint64)
+    for k in range(32):
+        words |= stream[:, :, k] << np.uint64(k)
+    return words.astype(np.uint32)
+
+
+def unpack_codes(packed, bits: int, d_in: int):
+    packed = np.ascontiguousarray(packed, np.uint32)
+    d_out = packed.shape[0]
+    stream = np.zeros((d_out, packed.shape[1], 32), np.uint8)
+    for k in range(32):
+        stream[:, :, k] = (packed >> np.uint32(k)) & np.uint32(1)
+    stream = stream.reshape(d_out, d_in, bits)
+    codes = np.zeros((d_out, d_in), np.uint8)
+    for k in range(bits):
+        codes |= stream[:, :, k] << k
+    return codes
+
+
+def dequantize(codes, scales, zeros, quant_group: int):
+    """Q = s (W_int - z) per (row, column group), float64 (Algorithm 1, final step)."""
+    codes = np.asarray(codes)
+    seg = quant_group or codes.shape[1]
+    s = np.repeat(np.asarray(scales, np.float64), seg, axis=1)
+    z = np.repeat(np.asarray(zeros, np.float64), seg, axis=1)
+    return s * (codes.astype(np.float64) - z)

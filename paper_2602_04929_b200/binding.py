@@ -76,6 +76,10 @@ _SIGNATURES = {
     "tb_attention_layer_info_count": (_int, [_vp, _int]),
     "tb_attention_layer_workspace": (_sz, [_vp, _vp]),
     "tb_attention_layer": (_int, [_vp, _vp, _vp, _sz, _vp]),
+    "tb_launch_count": (ctypes.c_ulonglong, []),
+    "tb_packed_bytes": (_sz, [_int, _int, _int]),
+    "tb_pack_codes": (_int, [_vp, _int, _int, _int, _vp, _vp]),
+    "tb_unpack_dequant": (_int, [_vp, _vp, _vp, _int, _int, _int, _int, _vp, _vp, _vp, _vp, _f, _vp, _vp]),
     "tb_profile_enable": (None, [_int]),
     "tb_profile_read": (_int, [ctypes.POINTER(ctypes.c_double), _int]),
     "tb_quantize_from_host_workspace": (_sz, [ctypes.POINTER(LayerDesc), _ll, _int]),
@@ -438,6 +442,37 @@ def tb_attention_layer(desc: AttentionDesc, io: AttentionIO, ws) -> None:
 
 PHASES = ("setup", "grid", "sweep", "compensation", "cd", "output", "loss",
           "hessian", "cross", "hout", "factor", "prep", "copy")
+
+
+def tb_pack_codes(codes, bits: int):
+    """codes [d_out, d_in] uint8 -> packed int32 [d_out, d_in * bits / 32] (bit stream per row)."""
+    d_out, d_in = codes.shape
+    nbytes = int(load().tb_packed_bytes(d_out, d_in, bits))
+    if nbytes == 0:
+        raise ValueError("unsupported shape or bit width for packing")
+    packed = torch.empty((d_out, nbytes // (4 * d_out)), dtype=torch.int32, device=codes.device)
+    _check(load().tb_pack_codes(_ptr(codes, torch.uint8), d_out, d_in, bits, _ptr(packed), _stream()), "tb_pack_codes")
+    return packed
+
+
+def tb_unpack_dequant(packed, scales, zeros, d_in: int, bits: int, quant_group: int, want_codes=True, want_w_hat=True,
+                      codes_ref=None, w_hat_ref=None, tol: float = 2.0 ** -22):
+    """Returns (codes, w_hat, mismatch): mismatch is None without a reference, else an int64 tensor
+    [code mismatches, values beyond tol]."""
+    d_out = packed.shape[0]
+    dev = packed.device
+    codes = torch.empty((d_out, d_in), dtype=torch.uint8, device=dev) if want_codes else None
+    w_hat = torch.empty((d_out, d_in), dtype=torch.float32, device=dev) if want_w_hat else None
+    mism = torch.zeros(2, dtype=torch.int64, device=dev) if (codes_ref is not None or w_hat_ref is not None) else None
+    _check(load().tb_unpack_dequant(_ptr(packed, torch.int32), _ptr(scales, torch.float32), _ptr(zeros, torch.int32),
+                                    d_out, d_in, bits, quant_group, _ptr(codes, None, True), _ptr(w_hat, None, True),
+                                    _ptr(codes_ref, torch.uint8, True), _ptr(w_hat_ref, torch.float32, True), float(tol),
+                                    _ptr(mism, None, True), _stream()), "tb_unpack_dequant")
+    return codes, w_hat, mism
+
+
+def tb_launch_count() -> int:
+    return int(load().tb_launch_count())
 
 
 def tb_profile_enable(on: bool) -> None:

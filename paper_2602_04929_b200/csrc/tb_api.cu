@@ -4,6 +4,12 @@
 
 using namespace tb;
 
+namespace tb {
+unsigned long long g_launch_count = 0;
+}
+
+extern "C" unsigned long long tb_launch_count(void) { return tb::g_launch_count; }
+
 extern "C" const char* tb_status_string(tb_status st) {
   switch (st) {
     case TB_OK: return "ok";

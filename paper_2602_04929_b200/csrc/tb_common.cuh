@@ -19,8 +19,10 @@
     }                                            \
   } while (0)
 
+// Follows every kernel launch of the library (one check per launch); also counts them.
 #define TB_LAUNCH_CHECK()                                   \
   do {                                                      \
+    ++tb::g_launch_count;                                   \
     if (cudaGetLastError() != cudaSuccess) return TB_ERR_CUDA; \
   } while (0)
 
@@ -31,6 +33,8 @@
   } while (0)
 
 namespace tb {
+
+extern unsigned long long g_launch_count;  // kernels launched by the library in this process (tb_api.cu)
 
 // Bump allocator over a caller-provided workspace.  With base == nullptr it
 // only measures (used by the *_workspace queries), so sizes and carving can

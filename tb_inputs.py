@@ -133,6 +133,67 @@ def causal_decay_mix(X: np.ndarray, rho: float, seq_len: int, bf16: bool = True)
     return bf16_bits_to_f32(to_bf16_bits(out)) if bf16 else out
 
 
+def causal_decay_matrix(rho: float, seq_len: int) -> np.ndarray:
+    """The explicit A_h of causal_decay_mix for one sequence: A[t, s] = rho^(t-s) / sum_{s' <= t} rho^(t-s')
+    for s <= t, 0 above the diagonal (float64)."""
+    t = np.arange(seq_len)
+    A = np.tril(rho ** np.maximum(t[:, None] - t[None, :], 0).astype(np.float64))
+    return A / A.sum(axis=1, keepdims=True)
+
+
+# ----------------------------------------------------------------------------
+# The same recipes drawn on a CUDA device with torch's seeded generator, for tensors too large to
+# draw with numpy in reasonable time (the benchmark's 128 x 2048 tokens of width 4096 or 8192).
+# Same distributions and structure as the numpy recipes above (the outlier channels and the common
+# factor are the numpy ones), not the same random numbers.
+# ----------------------------------------------------------------------------
+
+def heavy_tail_device(rec: "HeavyTailRecipe", n_tok: int, device, seed: int = 0, chunk: int = 16384):
+    """bf16 [n_tok, d] activations of HeavyTailRecipe on `device`."""
+    import torch
+    g = torch.Generator(device=device)
+    g.manual_seed((rec.seed << 20) + (rec.tid_shift << 10) + seed + 12345)
+    F = torch.from_numpy(rec.F).to(device)
+    sig = torch.from_numpy(rec.sigma_c).to(device)
+    out = torch.empty((n_tok, rec.d), dtype=torch.bfloat16, device=device)
+    for t0 in range(0, n_tok, chunk):
+        n = min(chunk, n_tok - t0)
+        noise = torch.randn((n, rec.d), generator=g, device=device)
+        f = torch.randn((n, rec.rank), generator=g, device=device)
+        tau = torch.exp(rec.tok_sigma * torch.randn((n, 1), generator=g, device=device))
+        out[t0:t0 + n] = ((noise + 2.0 * (f @ F)) * tau * sig[None, :]).to(torch.bfloat16)
+    return out
+
+
+def deviation_device(dev_rec: "DeviationRecipe", Xfp, seed: int = 0, chunk: int = 16384):
+    """Quantized-path twin of Xfp (bf16 on a device): X = Xfp + 0.1 Xfp A B + 0.03 sigma_c n'."""
+    import torch
+    device = Xfp.device
+    g = torch.Generator(device=device)
+    g.manual_seed((dev_rec.base.seed << 20) + (dev_rec.base.tid_shift << 10) + seed + 777)
+    A = torch.from_numpy(dev_rec.A).to(device)
+    B = torch.from_numpy(dev_rec.B).to(device)
+    sig = torch.from_numpy(dev_rec.base.sigma_c).to(device)
+    out = torch.empty_like(Xfp)
+    for t0 in range(0, Xfp.shape[0], chunk):
+        x = Xfp[t0:t0 + chunk].float()
+        noise = torch.randn(x.shape, generator=g, device=device)
+        out[t0:t0 + chunk] = (x + 0.1 * ((x @ A) @ B) + 0.03 * sig[None, :] * noise).to(torch.bfloat16)
+    return out
+
+
+def causal_decay_mix_device(X, rho: float, seq_len: int):
+    """causal_decay_mix on a device: A_h X per sequence through the explicit matrix (float32 product)."""
+    import torch
+    n, d = X.shape
+    A = torch.from_numpy(causal_decay_matrix(rho, seq_len).astype(np.float32)).to(X.device)
+    out = torch.empty_like(X)
+    for s0 in range(0, n, seq_len):
+        m = min(seq_len, n - s0)
+        out[s0:s0 + m] = (A[:m, :m] @ X[s0:s0 + m].float()).to(X.dtype)
+    return out
+
+
 def spd_matrix(seed: int, n: int, cond: float = 1e3, tid: int = T_HOUT) -> np.ndarray:
     """V diag(lambda) V^T with V the Q-factor of a Gaussian matrix and lambda
     log-spaced from 1 down to 1/cond.  float32 (the layout the library takes)."""

@@ -767,3 +767,33 @@ def test_identity_mode_layer_reports_refined_scales_and_loss():
     assert np.isclose(out.loss[0], oracle.loss_head(pr["W"], out.w_hat, pr["Hin"], None, pr["R"]), rtol=1e-13)
     pre = np.repeat(out.scales_pre_cd, 8, axis=1) * (out.codes.astype(float) - np.repeat(out.zeros, 8, axis=1))
     assert out.loss[0] <= oracle.loss_head(pr["W"], pre, pr["Hin"], None, pr["R"])
+
+
+# --------------------------------------------------------------------------- packed integer weights
+@pytest.mark.parametrize("bits", [2, 3, 4, 5, 8])
+def test_packing_is_the_little_endian_bit_stream(bits):
+    """The reference packer against a brute-force bit stream held in one Python integer per row, and
+    its round trip; for 3 bits, codes straddle word boundaries."""
+    g = np.random.default_rng(700 + bits)
+    codes = g.integers(0, 1 << bits, size=(5, 64)).astype(np.uint8)
+    packed = oracle.pack_codes(codes, bits)
+    assert packed.dtype == np.uint32 and packed.shape == (5, 64 * bits // 32)
+    for r in range(5):
+        big = 0
+        for j, c in enumerate(codes[r].tolist()):
+            big |= c << (j * bits)
+        words = [(big >> (32 * w)) & 0xFFFFFFFF for w in range(64 * bits // 32)]
+        assert packed[r].tolist() == words
+    assert np.array_equal(oracle.unpack_codes(packed, bits, 64), codes)
+    if bits == 3:   # hand example: codes 0..7 fill 24 bits: 0b111_110_101_100_011_010_001_000
+        row = np.array([[0, 1, 2, 3, 4, 5, 6, 7] + [0] * 24], np.uint8)
+        assert oracle.pack_codes(row, 3)[0].tolist() == [0b111110101100011010001000, 0, 0]
+
+
+def test_dequantize_is_s_times_code_minus_zero():
+    codes = np.array([[0, 3, 1, 2], [2, 2, 0, 1]], np.uint8)
+    s = np.array([[0.5, 2.0], [1.0, 0.25]])
+    z = np.array([[1, 2], [0, 1]])
+    want = np.array([[-0.5, 1.0, -2.0, 0.0], [2.0, 2.0, -0.25, 0.0]])
+    assert np.array_equal(oracle.dequantize(codes, s, z, 2), want)
+    assert np.array_equal(oracle.dequantize(codes, s[:, :1], z[:, :1], 0), s[:, :1] * (codes - z[:, :1]))
