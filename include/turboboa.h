@@ -48,8 +48,18 @@ enum {
                              quantized (Algorithm 1, grid step; Section 3.3).  Off:
                              the grid of every row is chosen once from the
                              original weights (the fixed grid of BoA).         */
-  TB_F_CD_REFINE = 2      /* coordinate-descent scale refinement after the loop
+  TB_F_CD_REFINE = 2,     /* coordinate-descent scale refinement after the loop
                              (Algorithm 1, refinement; Proposition 3.3)        */
+  TB_F_DYNAMIC_GRID = 4   /* variant for column groups (which the paper does not
+                             have): the (scale, zero) of a column group is searched
+                             when the column sweep arrives at the group, from the
+                             group's current values, i.e. after the error feedback
+                             of every earlier column of the row (same candidates,
+                             same score).  Overrides the two grid modes above; with
+                             quant_group = 0 it is TB_F_ADAPTIVE_GRID.  Groups of at
+                             most 128 columns.  Runs group by group (one grid
+                             search, one panel, one update per group), not through
+                             the fused sweep kernel.                            */
 };
 
 /* Problem description of one projection (Algorithm 1, inputs). */

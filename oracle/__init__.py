@@ -30,4 +30,5 @@ from .ref import (  # noqa: F401
     dequantize,
     F_ADAPTIVE_GRID,
     F_CD_REFINE,
+    F_DYNAMIC_GRID,
 )

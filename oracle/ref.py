@@ -13,6 +13,7 @@ import numpy as np
 
 F_ADAPTIVE_GRID = 1
 F_CD_REFINE = 2
+F_DYNAMIC_GRID = 4   # variant: a column group's grid is searched when the sweep arrives at it
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "turboboa_oracle.c")
@@ -246,11 +247,17 @@ def grid_rows(W0, Hin, gq: int, bits: int, n_cand: int = 16, with_scores: bool =
     return (s, z, cand, scores) if with_scores else (s, z, cand)
 
 
-def sweep_rows(W0, Uin, s, z, gq: int, bits: int, P=None, band: float = 1e-6, hint_codes=None):
+def sweep_rows(W0, Uin, s, z, gq: int, bits: int, P=None, band: float = 1e-6, hint_codes=None, Hin_dyn=None,
+               n_cand: int = 16):
+    """Hin_dyn given: the dynamic-grid variant; s and z may be None and the grids found in the sweep are
+    returned as two extra values."""
     lib = _load()
-    W0, Uin, P, s = _f64(W0), _f64(Uin), _f64(P), _f64(s)
-    z = np.ascontiguousarray(z, np.int32)
+    W0, Uin, P = _f64(W0), _f64(Uin), _f64(P)
     m, d = W0.shape
+    ng = 1 if gq == 0 else d // gq
+    Hin_dyn = _f64(Hin_dyn)
+    s = np.ones((m, ng)) if s is None else np.array(s, dtype=np.float64, copy=True)
+    z = np.zeros((m, ng), np.int32) if z is None else np.array(z, dtype=np.int32, copy=True)
     codes = np.zeros((m, d), np.uint8)
     Q = np.zeros((m, d))
     err = np.zeros((m, d))
@@ -259,8 +266,10 @@ def sweep_rows(W0, Uin, s, z, gq: int, bits: int, P=None, band: float = 1e-6, hi
         hint_codes = np.ascontiguousarray(hint_codes, np.uint8)
     lib.tbo_sweep_rows(_p(W0), m, d, gq, _p(Uin), _p(P), _p(s), _p(z, ctypes.c_int), bits,
                        ctypes.c_double(band), _p(hint_codes, ctypes.c_ubyte),
-                       _p(codes, ctypes.c_ubyte), _p(Q), _p(err), ctypes.byref(cnt))
+                       _p(codes, ctypes.c_ubyte), _p(Q), _p(err), ctypes.byref(cnt), _p(Hin_dyn), n_cand)
     counters = {k: int(getattr(cnt, k)) for k, _ in _Counters._fields_}
+    if Hin_dyn is not None:
+        return codes, Q, err, counters, s, z
     return codes, Q, err, counters
 
 

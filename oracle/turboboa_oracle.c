@@ -30,6 +30,11 @@
  *   - column groups of quant_group columns each own a (s, z) pair; the score
  *     uses the diagonal block of H_in of that group.
  *   - rounding is round-half-to-even of x = w/s + z.
+ *   - by default the grid of a row is fixed before its sweep starts (Algorithm 1
+ *     hands the scales to the sweep).  Variant TBO_F_DYNAMIC_GRID: the (s, z) of a
+ *     column group is searched when the sweep ARRIVES at the group's first column,
+ *     from the group's current values, i.e. after the error feedback of all earlier
+ *     columns of the row; same candidates, same score, same tie rule.
  *
  * Loop order: Algorithm 2 walks columns for all rows at once; rows never
  * interact inside the sweep, so this file walks one row at a time (the row
@@ -49,6 +54,7 @@
 
 #define TBO_F_ADAPTIVE_GRID 1u
 #define TBO_F_CD_REFINE 2u
+#define TBO_F_DYNAMIC_GRID 4u /* variant of the reading on column groups: see sweep_row */
 
 typedef struct {
   int d_out, d_in;
@@ -187,13 +193,29 @@ static void grid_row(const double *w, int d, int gq, const double *Hin, int maxq
 /* w: working copy, overwritten (on return w[j] is NOT meaningful).           */
 /* U: upper factor of H_in^{-1}; P: strictly upper correction or NULL.        */
 /* ------------------------------------------------------------------------- */
-static void sweep_row(double *w, int d, int gq, const double *U, const double *P, const double *s,
-                      const int *z, int maxq, double band, const unsigned char *hint,
-                      unsigned char *codes, double *Q, double *err, tbo_counters *cnt) {
+typedef struct { /* dynamic-grid variant: what the in-sweep search needs (Hin NULL = grid fixed beforehand) */
+  const double *Hin;
+  int n_cand;
+  double cand_tol;
+  const unsigned char *hint_cand;
+  const int *hint_zero;
+  unsigned char *cand;
+} tbo_dyn;
+
+static void sweep_row(double *w, int d, int gq, const double *U, const double *P, double *s, int *z,
+                      int maxq, double band, const unsigned char *hint, unsigned char *codes,
+                      double *Q, double *err, tbo_counters *cnt, const tbo_dyn *dyn) {
   int seg = gq > 0 ? gq : d;
   long long near = 0, adopted = 0;
   for (int j = 0; j < d; ++j) {
     int g = j / seg;
+    if (dyn && dyn->Hin && j % seg == 0) {
+      /* the group's grid from its values on arrival (all earlier columns' feedback applied) */
+      int k = grid_segment(w + j, seg, dyn->Hin + (size_t)j * d + j, d, maxq, dyn->n_cand, band,
+                           dyn->cand_tol, dyn->hint_cand ? (int)dyn->hint_cand[g] : -1,
+                           dyn->hint_zero ? dyn->hint_zero[g] : -1, &s[g], &z[g], NULL, cnt);
+      if (dyn->cand) dyn->cand[g] = (unsigned char)k;
+    }
     double sj = s[g], zj = (double)z[g];
     double wj = w[j]; /* value on arrival at column j */
     double x = wj / sj + zj;
@@ -265,10 +287,11 @@ static void group_loop_head(const tbo_desc *D, double *Wt, const double *Hin, co
   const int dh = D->d_head, d = D->d_in, gq = D->quant_group;
   const int seg = gq > 0 ? gq : d, ng = d / seg;
   const int maxq = (1 << D->bits) - 1;
-  const int adaptive = (D->flags & TBO_F_ADAPTIVE_GRID) != 0;
+  const int dynamic = (D->flags & TBO_F_DYNAMIC_GRID) != 0;
+  const int adaptive = (D->flags & TBO_F_ADAPTIVE_GRID) != 0 && !dynamic;
   const int N = Uo ? D->out_block : dh; /* H_out = I: every row at once */
 
-  if (!adaptive) {
+  if (!adaptive && !dynamic) {
     /* fixed grid: computed once from the original weights, all rows */
 #pragma omp parallel for schedule(dynamic)
     for (int r = 0; r < dh; ++r)
@@ -295,9 +318,13 @@ static void group_loop_head(const tbo_desc *D, double *Wt, const double *Hin, co
                  zeros + (size_t)r * ng, cand ? cand + (size_t)r * ng : NULL, cnt);
       double *w = (double *)malloc(sizeof(double) * (size_t)d);
       memcpy(w, w0, sizeof(double) * (size_t)d);
+      tbo_dyn dyn = {dynamic ? Hin : NULL, D->n_cand, cand_tol,
+                     hint_cand ? hint_cand + (size_t)r * ng : NULL,
+                     hint_zeros ? hint_zeros + (size_t)r * ng : NULL,
+                     cand ? cand + (size_t)r * ng : NULL};
       sweep_row(w, d, gq, Uin, P, scales + (size_t)r * ng, zeros + (size_t)r * ng, maxq, band,
                 hint_codes ? hint_codes + (size_t)r * d : NULL, codes + (size_t)r * d,
-                Q + (size_t)r * d, NULL, cnt);
+                Q + (size_t)r * d, NULL, cnt, &dyn);
       free(w);
       double *Er = E + (size_t)b * d;
       for (int k = 0; k < d; ++k) Er[k] = w0[k] - Q[(size_t)r * d + k];
@@ -525,19 +552,21 @@ void tbo_grid_rows(const double *W0, int m, int d, int gq, const double *Hin, in
     }
 }
 
+/* Hin_dyn != NULL selects the dynamic-grid variant: s and z are then outputs. */
 void tbo_sweep_rows(const double *W0, int m, int d, int gq, const double *Uin, const double *P,
-                    const double *s, const int *z, int bits, double band,
-                    const unsigned char *hint_codes, unsigned char *codes, double *Q, double *err,
-                    tbo_counters *cnt) {
+                    double *s, int *z, int bits, double band, const unsigned char *hint_codes,
+                    unsigned char *codes, double *Q, double *err, tbo_counters *cnt,
+                    const double *Hin_dyn, int n_cand) {
   int seg = gq > 0 ? gq : d, ng = d / seg, maxq = (1 << bits) - 1;
   if (cnt) memset(cnt, 0, sizeof(*cnt));
 #pragma omp parallel for schedule(dynamic)
   for (int r = 0; r < m; ++r) {
     double *w = (double *)malloc(sizeof(double) * (size_t)d);
     memcpy(w, W0 + (size_t)r * d, sizeof(double) * (size_t)d);
+    tbo_dyn dyn = {Hin_dyn, n_cand, 0.0, NULL, NULL, NULL};
     sweep_row(w, d, gq, Uin, P, s + (size_t)r * ng, z + (size_t)r * ng, maxq, band,
               hint_codes ? hint_codes + (size_t)r * d : NULL, codes + (size_t)r * d,
-              Q + (size_t)r * d, err ? err + (size_t)r * d : NULL, cnt);
+              Q + (size_t)r * d, err ? err + (size_t)r * d : NULL, cnt, &dyn);
     free(w);
   }
 }

@@ -16,7 +16,7 @@ from . import _build
 
 TB_OK = 0
 TB_F32, TB_BF16 = 0, 1
-TB_F_ADAPTIVE_GRID, TB_F_CD_REFINE = 1, 2
+TB_F_ADAPTIVE_GRID, TB_F_CD_REFINE, TB_F_DYNAMIC_GRID = 1, 2, 4
 
 _STATUS_NAMES = {0: "TB_OK", 1: "TB_ERR_INVALID_ARG", 2: "TB_ERR_UNSUPPORTED", 3: "TB_ERR_WORKSPACE",
                  4: "TB_ERR_NOT_SPD", 5: "TB_ERR_CUDA", 6: "TB_ERR_TIMEOUT"}

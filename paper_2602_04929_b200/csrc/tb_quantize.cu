@@ -114,6 +114,8 @@ struct GridP {
   RowMap rm;
   int M, d, seg, ng, maxq, n_cand, ncp, rt;
   int units, rows_per_unit, tiles_per_unit;
+  const double* Wloc;  // or nullptr: the step's rows as a contiguous [M][d] working copy, read instead of Wt
+  int grp0;            // column group of blockIdx.x = 0
 };
 
 __global__ void __launch_bounds__(GEMM_THREADS, 1) k_grid(GridP p) {
@@ -122,7 +124,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) k_grid(GridP p) {
   __shared__ long long c_row[128];  // global row of a candidate row, or -1
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int grp = blockIdx.x;
+  const int grp = p.grp0 + blockIdx.x;
   const int unit = blockIdx.y / p.tiles_per_unit;
   const int tile = blockIdx.y % p.tiles_per_unit;
   const int seg0 = grp * p.seg;
@@ -273,10 +275,12 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) k_grid_tri(GridP p) {
   float* Bs = reinterpret_cast<float*>(smem_raw + (size_t)128 * GT_LDE * sizeof(double));  // [k][n]
   __shared__ double c_s[128], c_rs[128], c_z[128], c_J[128];
   __shared__ long long c_row[128];  // global row of a candidate row, or -1
+  __shared__ long long c_src[128];  // element offset of that row's first column in the source matrix
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int grp = blockIdx.x;
+  const int grp = p.grp0 + blockIdx.x;
   const int unit = blockIdx.y / p.tiles_per_unit;
+  const double* Wsrc = p.Wloc ? p.Wloc : p.Wt;
   const int tile = blockIdx.y % p.tiles_per_unit;
   const int seg0 = grp * p.seg;
   const int d = p.d, seg = p.seg;
@@ -303,11 +307,12 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) k_grid_tri(GridP p) {
   for (int r = warp; r < p.rt; r += GEMM_THREADS / 32) {
     const int rloc = tile * p.rt + r;
     const bool valid = rloc < p.rows_per_unit;
-    long long grow = -1;
+    long long grow = -1, src = 0;
     double mn = 0.0, mx = 0.0;
     if (valid) {
       grow = p.rm.row(unit * p.rows_per_unit + rloc);
-      const double* w = p.Wt + grow * p.d + seg0;
+      src = (p.Wloc ? (long long)(unit * p.rows_per_unit + rloc) : grow) * p.d;
+      const double* w = Wsrc + src + seg0;
       for (int a = lane; a < p.seg; a += 32) {
         const double v = w[a];
         mn = fmin(mn, v);
@@ -334,6 +339,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) k_grid_tri(GridP p) {
       c_rs[cr] = 1.0 / s;
       c_z[cr] = z;
       c_row[cr] = (valid && k < p.n_cand) ? grow : -1;
+      c_src[cr] = src;
     }
   }
   __syncthreads();
@@ -345,7 +351,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) k_grid_tri(GridP p) {
     const double s = c_s[cr], rs = c_rs[cr], z = c_z[cr];
     const double magic = 6755399441055744.0;  // 1.5 * 2^52
     const double zm = z + magic;
-    const double* w = p.Wt + (grow < 0 ? 0 : grow) * d + seg0;
+    const double* w = Wsrc + (grow < 0 ? 0 : c_src[cr]) + seg0;
 #pragma unroll 8
     for (int i = 0; i < 64; ++i) {
       const int k = (tid >> 7) + 2 * i;
@@ -929,6 +935,98 @@ int sweep_error_read_clear() {
     cudaMemcpyToSymbol(g_sweep_error, &z, sizeof(int));
   }
   return v;
+}
+
+// ---------------------------------------------------------------------------
+// Dynamic-grid variant of the sweep (the grid of a column group is searched when
+// the sweep arrives at the group, from the group's current values).  Right-looking,
+// one column group at a time on a contiguous working copy Wk [M][d] of the step's
+// rows: k_grid_tri on the group's current values, this kernel for the group's
+// columns (Algorithm 2's column loop restricted to the group: one warp per row, a
+// lane per column of each 32-column sub-block, values in registers), then one GEMM
+// that applies the group's errors (and, with R, its arrival values) to all later
+// columns.  The group's errors only live until that GEMM has run.
+// ---------------------------------------------------------------------------
+struct GroupPanelP {
+  double* Wk;            // [M][d] working values of the step's rows
+  const float* U;        // [n_hin][d][d]
+  const float* P;        // or nullptr
+  double* Err;           // [M][seg] normalised errors of this group
+  double* Arr;           // [M][seg] arrival values of this group (with P)
+  unsigned char* codes;  // [d_out][d]
+  const double* sD;      // [d_out][ng]
+  const int* z;          // [d_out][ng]
+  tb_stats* stats;
+  RowMap rm;
+  int M, d, seg, ng, maxq, grp;
+  int units, rows_per_unit, ctas_per_unit;
+};
+
+__global__ void __launch_bounds__(256) k_group_panel(GroupPanelP p) {
+  extern __shared__ float gp_sm[];   // U[c0 + j][c0 + c] at gp_sm[j * seg + c], then P likewise
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int seg = p.seg, d = p.d, c0 = p.grp * seg, nsb = seg / 32;
+  // a CTA takes 8 rows of one unit (rows that share an H_in / U_in); the last CTA of a unit may hold fewer
+  const int unit = blockIdx.x / p.ctas_per_unit;
+  const int m0 = unit * p.rows_per_unit + (blockIdx.x % p.ctas_per_unit) * 8;
+  const long long uoff = (p.units > 1) ? (long long)unit * d * d : 0;
+  const float* U = p.U + uoff;
+  const float* Pm = p.P ? p.P + uoff : nullptr;
+  float* sU = gp_sm;
+  float* sP = gp_sm + seg * seg;
+  for (int i = tid; i < seg * seg; i += blockDim.x) {
+    const int j = i / seg, c = i % seg;
+    sU[i] = (c >= j) ? U[(long long)(c0 + j) * d + c0 + c] : 0.0f;
+    if (Pm) sP[i] = (c > j) ? Pm[(long long)(c0 + j) * d + c0 + c] : 0.0f;
+  }
+  __syncthreads();
+  const int m = m0 + warp;
+  if (m >= (unit + 1) * p.rows_per_unit) return;
+  const long long grow = p.rm.row(m);
+  const double s = p.sD[grow * p.ng + p.grp];
+  const double zz = (double)p.z[grow * p.ng + p.grp];
+  const double maxq = (double)p.maxq;
+  double* wrow = p.Wk + (long long)m * d + c0;
+  double v[4] = {0.0, 0.0, 0.0, 0.0};
+#pragma unroll
+  for (int t = 0; t < 4; ++t)
+    if (t < nsb) v[t] = wrow[t * 32 + lane];
+  unsigned int n_near = 0, n_clamp = 0;
+  for (int j = 0; j < seg; ++j) {
+    const int tj = j >> 5, lj = j & 31;
+    const double mine = (tj == 0) ? v[0] : (tj == 1) ? v[1] : (tj == 2) ? v[2] : v[3];
+    const double wj = shfl_d(mine, lj);   // value of column j on arrival
+    const double x = wj / s + zz;
+    const double q = fmin(fmax(rne(x), 0.0), maxq);
+    const double ej = (wj - s * (q - zz)) / (double)sU[j * seg + j];
+    if (lane == lj) {
+      p.codes[grow * d + c0 + j] = (unsigned char)(int)q;
+      p.Err[(long long)m * seg + j] = ej;
+      if (Pm) p.Arr[(long long)m * seg + j] = wj;
+      const double fl = floor(x);
+      const double a0 = fmin(fmax(fl, 0.0), maxq), a1 = fmin(fmax(fl + 1.0, 0.0), maxq);
+      if (fabs(x - (fl + 0.5)) < 1e-6 && a0 != a1) ++n_near;
+      if (rne(x) != q) ++n_clamp;
+    }
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      const int c = t * 32 + lane;
+      if (t < nsb && c > j) {
+        double nv = fma(-ej, (double)sU[j * seg + c], v[t]);
+        if (Pm) nv = fma(-wj, (double)sP[j * seg + c], nv);
+        v[t] = nv;
+      }
+    }
+  }
+  if (p.stats) {
+    n_near = __reduce_add_sync(0xffffffffu, n_near);
+    n_clamp = __reduce_add_sync(0xffffffffu, n_clamp);
+    if (lane == 0) {
+      if (n_near) atomicAdd(&p.stats->near_tie_codes, (unsigned long long)n_near);
+      if (n_clamp) atomicAdd(&p.stats->clamped_codes, (unsigned long long)n_clamp);
+      if (m == 0) atomicAdd(&p.stats->column_steps, (unsigned long long)seg);
+    }
+  }
 }
 
 // E[m][k] = W~[row(m)][k] - s (code - z): the quantization error of the group on
@@ -1534,7 +1632,8 @@ __global__ void k_loss_identity_final(const double* __restrict__ partial, double
 // ---------------------------------------------------------------------------
 struct Plan {
   int d_out, d, H, dh, n_hin, bits, seg, ng, g, S, maxq, n_cand, ncp, rt, cd_iters;
-  bool adaptive, cd, with_r, with_loss, has_hout;
+  bool adaptive, dynamic, cd, with_r, with_loss, has_hout;
+  double *dynErr, *dynArr;  // [Mmax][seg] errors / arrival values of the current column group (dynamic grid)
   int Mmax;
   long long cd_rows;  // rows per coordinate-descent batch
   // workspace
@@ -1585,7 +1684,10 @@ static tb_status make_plan(const tb_layer_desc* D, bool has_hout, bool with_r, b
   p.ncp = pow2_ceil(D->n_cand);
   p.rt = 128 / p.ncp;
   p.cd_iters = D->cd_iters;
-  p.adaptive = (D->flags & TB_F_ADAPTIVE_GRID) != 0;
+  // dynamic grid: with one group per row it IS the adaptive grid (the group arrives unchanged)
+  p.dynamic = (D->flags & TB_F_DYNAMIC_GRID) != 0 && p.ng > 1;
+  p.adaptive = (D->flags & TB_F_ADAPTIVE_GRID) != 0 || ((D->flags & TB_F_DYNAMIC_GRID) != 0 && !p.dynamic);
+  if (p.dynamic && p.seg > 128) return TB_ERR_UNSUPPORTED;
   p.cd = (D->flags & TB_F_CD_REFINE) != 0 && D->cd_iters > 0;
   p.with_r = with_r;
   p.with_loss = with_loss;
@@ -1600,6 +1702,8 @@ static tb_status make_plan(const tb_layer_desc* D, bool has_hout, bool with_r, b
   p.W0c = with_r ? b.take<double>((size_t)p.Mmax * dd) : nullptr;
   p.sD = b.take<double>((size_t)p.d_out * p.ng);
   p.T = (has_hout && p.S > 1) ? b.take<double>((size_t)p.H * p.S * p.dh * p.g) : nullptr;
+  p.dynErr = p.dynamic ? b.take<double>((size_t)p.Mmax * p.seg) : nullptr;
+  p.dynArr = (p.dynamic && with_r) ? b.take<double>((size_t)p.Mmax * p.seg) : nullptr;
   p.Dq = p.Dm = p.Yw = p.n0 = p.Amat = p.G2 = nullptr;
   p.Wb = nullptr;
   p.WbT = p.Hp = nullptr;
@@ -1682,6 +1786,8 @@ static tb_status run_grid(const Plan& p, const float* H_in, float* scales, int* 
   gp.units = (p.n_hin == 1) ? 1 : p.H;
   gp.rows_per_unit = M / gp.units;
   gp.tiles_per_unit = (gp.rows_per_unit + p.rt - 1) / p.rt;
+  gp.Wloc = nullptr;
+  gp.grp0 = 0;
   static bool configured[64] = {false}, configured_tri[64] = {false};
   TB_TRY(allow_smem(k_grid, GemmSmem<double>::bytes, configured));
   TB_TRY(allow_smem(k_grid_tri, GRID_TRI_SMEM, configured_tri));
@@ -1768,6 +1874,98 @@ static tb_status run_sweep_rows(const Plan& p, const float* U_in, const float* P
   return launch_sweep_rows<true>(sp, map_u, map_e, map_p, map_a, st);
 }
 
+// Dynamic-grid variant: group by group on the working copy Wk of the step's rows.
+static tb_status run_sweep_dynamic(const Plan& p, const float* H_in, const float* U_in, const float* P,
+                                   unsigned char* codes, float* scales, int* zeros, unsigned char* cand,
+                                   tb_stats* stats, RowMap rm, int M, cudaStream_t st) {
+  const int d = p.d, seg = p.seg;
+  const int units = (p.n_hin == 1) ? 1 : p.H;
+  const long long dd = (long long)d * d;
+  k_gather<<<ew_blocks((long long)M * d), 256, 0, st>>>(p.Wt, p.Wk, nullptr, rm, M, d);
+  TB_LAUNCH_CHECK();
+  GridP gp;
+  gp.Wt = p.Wt;
+  gp.Hin = H_in;
+  gp.sD = p.sD;
+  gp.s_out = scales;
+  gp.z_out = zeros;
+  gp.cand_out = cand;
+  gp.rm = rm;
+  gp.M = M;
+  gp.d = d;
+  gp.seg = seg;
+  gp.ng = p.ng;
+  gp.maxq = p.maxq;
+  gp.n_cand = p.n_cand;
+  gp.ncp = p.ncp;
+  gp.rt = p.rt;
+  gp.units = units;
+  gp.rows_per_unit = M / units;
+  gp.tiles_per_unit = (gp.rows_per_unit + p.rt - 1) / p.rt;
+  gp.Wloc = p.Wk;
+  const long long ytiles = (long long)gp.units * gp.tiles_per_unit;
+  if (ytiles > 65535) return TB_ERR_UNSUPPORTED;
+  static bool configured_tri[64] = {false}, configured_panel[64] = {false};
+  TB_TRY(allow_smem(k_grid_tri, GRID_TRI_SMEM, configured_tri));
+  const size_t panel_smem = (size_t)seg * seg * sizeof(float) * (P ? 2 : 1);
+  TB_TRY(allow_smem(k_group_panel, 2 * 128 * 128 * sizeof(float), configured_panel));
+  GroupPanelP pp;
+  pp.Wk = p.Wk;
+  pp.U = U_in;
+  pp.P = P;
+  pp.Err = p.dynErr;
+  pp.Arr = p.dynArr;
+  pp.codes = codes;
+  pp.sD = p.sD;
+  pp.z = zeros;
+  pp.stats = stats;
+  pp.rm = rm;
+  pp.M = M;
+  pp.d = d;
+  pp.seg = seg;
+  pp.ng = p.ng;
+  pp.maxq = p.maxq;
+  pp.units = units;
+  pp.rows_per_unit = M / units;
+  pp.ctas_per_unit = (pp.rows_per_unit + 7) / 8;
+  for (int grp = 0; grp < p.ng; ++grp) {
+    const int c0 = grp * seg, c1 = c0 + seg;
+    gp.grp0 = grp;
+    k_grid_tri<<<dim3(1, (unsigned)ytiles), GEMM_THREADS, GRID_TRI_SMEM, st>>>(gp);
+    TB_LAUNCH_CHECK();
+    pp.grp = grp;
+    k_group_panel<<<(unsigned)(pp.ctas_per_unit * units), 256, panel_smem, st>>>(pp);
+    TB_LAUNCH_CHECK();
+    if (c1 >= d) break;
+    // Wk[:, c1:] -= Err U[c0:c1, c1:]  (- Arr P[c0:c1, c1:])
+    GemmP g = gemm_params();
+    g.A = p.dynErr;
+    g.a_m = seg;
+    g.a_k = 1;
+    g.a_batch = (long long)pp.rows_per_unit * seg;
+    g.B = U_in + (long long)c0 * d + c1;
+    g.b_k = d;
+    g.b_n = 1;
+    g.b_batch = (units > 1) ? dd : 0;
+    g.C = p.Wk + c1;
+    g.ldc = d;
+    g.c_batch = (long long)pp.rows_per_unit * d;
+    g.M = pp.rows_per_unit;
+    g.N = d - c1;
+    g.K = seg;
+    g.n_batch = units;
+    g.alpha = -1.0;
+    g.beta = 1.0;
+    TB_TRY((gemm_launch<double, float, double, double, false, true>(g, st)));
+    if (P) {
+      g.A = p.dynArr;
+      g.B = P + (long long)c0 * d + c1;
+      TB_TRY((gemm_launch<double, float, double, double, false, true>(g, st)));
+    }
+  }
+  return TB_OK;
+}
+
 }  // namespace tb
 
 using namespace tb;
@@ -1841,7 +2039,7 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
       TB_LAUNCH_CHECK();
     }
   }
-  if (!p.adaptive) {
+  if (!p.adaptive && !p.dynamic) {
     // fixed grid: every row, once, from the original weights
     PhaseScope ph(PH_GRID, st);
     RowMap all{p.dh, p.dh, 0};
@@ -1861,7 +2059,10 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
         k_gather<<<ew_blocks((long long)M * d), 256, 0, st>>>(p.Wt, p.W0c, nullptr, rm, M, d);
         TB_LAUNCH_CHECK();
       }
-      TB_TRY(run_sweep_rows(p, U_in, P, codes, zeros, stats, rm, M, st));
+      if (p.dynamic)
+        TB_TRY(run_sweep_dynamic(p, H_in, U_in, P, codes, scales, zeros, cand, stats, rm, M, st));
+      else
+        TB_TRY(run_sweep_rows(p, U_in, P, codes, zeros, stats, rm, M, st));
     }
     const int nrem = p.dh - i0 - p.g;
     if (!p.has_hout || nrem <= 0) continue;

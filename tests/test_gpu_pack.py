@@ -29,7 +29,7 @@ def test_pack_matches_the_reference_packer_and_round_trips(bits, shape):
                                              d_in, bits, 32, codes_ref=cd)
     assert torch.equal(back, cd) and mism.tolist() == [0, 0]
     ref = oracle.dequantize(codes, scales, zeros, 32)
-    assert np.array_equal(w_hat.cpu().numpy(), (scales.repeat(32, axis=1) * (codes.astype(np.float32) - zeros.repeat(32, axis=1))))
+    assert np.array_equal(w_hat.cpu().numpy(), (scales.repeat(32, axis=1) * (codes.astype(np.int32) - zeros.repeat(32, axis=1)).astype(np.float32)))
     assert np.max(np.abs(w_hat.cpu().numpy() - ref)) <= 2.0 ** -23 * np.max(np.abs(ref))
     # a planted difference is found and counted: one code and the value it gives
     bad = cd.clone()

@@ -188,6 +188,42 @@ def test_scale_refinement_with_more_than_32_column_groups(d_in, gq, with_r):
     _case(prob, 2, gq, 16, ADAPT | CD, cd_iters=2, label=f"CD row walk, two passes, d_in={d_in}")
 
 
+DYN = 4
+
+
+@pytest.mark.parametrize("gq,with_r,n_hin", [(128, False, 1), (64, True, 1), (32, False, 1), (128, True, 2)])
+def test_dynamic_column_group_grid(gq, with_r, n_hin):
+    """Variant of the column-group reading: a group's (scale, zero) is searched when the sweep arrives at
+    the group, from the values the error feedback of the earlier columns has left there.  Same parity
+    bar as the default mode; with and without the propagated-error term, shared and per-head H_in,
+    with the scale refinement after it."""
+    prob = make_problem(15, 384, 2, 64, 1024, with_r=with_r, n_hin=n_hin)
+    _case(prob, 3, gq, 16, DYN | CD, label=f"dynamic grid gq={gq} R={with_r} n_hin={n_hin}")
+    _case(prob, 2, gq, 64, DYN, label=f"dynamic grid gq={gq}, g = d_head, no CD")
+
+
+def test_dynamic_grid_special_cases():
+    """One group per row: the variant is the adaptive grid, bit for bit.  H_out = NULL mode runs it too.
+    Groups wider than 128 columns are refused."""
+    import paper_2602_04929_b200 as tb
+    prob = make_problem(16, 256, 2, 32, 1024)
+    a = run_gpu(prob, 3, 0, 8, DYN | CD)
+    b = run_gpu(prob, 3, 0, 8, ADAPT | CD)
+    for k in ("codes", "scales", "zeros", "cand", "w_hat", "loss"):
+        assert np.array_equal(a[k], b[k]), k
+    prob_id = make_problem(16, 256, 2, 32, 1024, hout=None)
+    _case(prob_id, 3, 64, 32, DYN | CD, label="dynamic grid, GPTQ mode")
+    with pytest.raises(tb.TurboBoAError):
+        run_gpu(make_problem(16, 512, 1, 32, 1024), 3, 256, 8, DYN)
+
+
+def test_dynamic_grid_full_width_sampled_head():
+    """4096 wide, 32 heads, INT2, groups of 128, g = 32, dynamic grid + CD; one sampled head."""
+    prob = cached_problem(0, 4096, 32, 128, 8192, with_r=True)
+    gpu = run_gpu(prob, 2, 128, 32, DYN | CD)
+    compare(prob, gpu, 2, 128, 32, DYN | CD, heads=[17], label="7b-q dynamic grid with R, sampled head")
+
+
 def test_near_constant_segment_under_the_fixed_grid():
     """A row segment whose original range is tiny gets a tiny scale from the fixed grid; after the
     compensation of earlier groups its pre-rounding values lie far outside the code range (and outside

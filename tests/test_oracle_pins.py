@@ -797,3 +797,69 @@ def test_dequantize_is_s_times_code_minus_zero():
     want = np.array([[-0.5, 1.0, -2.0, 0.0], [2.0, 2.0, -0.25, 0.0]])
     assert np.array_equal(oracle.dequantize(codes, s, z, 2), want)
     assert np.array_equal(oracle.dequantize(codes, s[:, :1], z[:, :1], 0), s[:, :1] * (codes - z[:, :1]))
+
+
+# --------------------------------------------------------------------------- dynamic per-column-group grid (variant)
+from oracle import F_DYNAMIC_GRID  # noqa: E402
+
+
+def test_dynamic_grid_is_the_grid_search_on_the_arrival_values():
+    """Variant of the column-group reading: the (s, z) of a group is searched when the sweep arrives
+    at it.  Pinned by reconstruction: the arrival values of group G are W0[:, G] - Err[:, <G] U[<G, G]
+    (GPTQ identity), and the grid found in the sweep must be the plain grid search (exhaustively
+    re-evaluated in Python above) on exactly those values.  The first group sees the snapshot."""
+    pr = small_problem(400, dh=6, d=16)
+    W, Hin = pr["W"], pr["Hin"]
+    U = oracle.factor_upper(Hin)
+    gq, bits = 4, 3
+    codes, Q, err, _, s, z = oracle.sweep_rows(W, U, None, None, gq, bits, Hin_dyn=Hin)
+    s_static, z_static, _ = oracle.grid_rows(W, Hin, gq, bits)
+    assert np.allclose(s[:, 0], s_static[:, 0], atol=0) and np.array_equal(z[:, 0], z_static[:, 0])
+    assert not np.allclose(s[:, 1:], s_static[:, 1:])
+    for g in range(16 // gq):
+        c0 = g * gq
+        arrival = W[:, c0:c0 + gq] - err[:, :c0] @ U[:c0, c0:c0 + gq]
+        for r in range(6):
+            cands = py_grid(arrival[r], Hin[c0:c0 + gq, c0:c0 + gq], bits, 16)
+            best = min(range(16), key=lambda k: (cands[k][0], k))     # lowest score, lowest k on ties
+            # a runner-up within rounding of the best score may legitimately win: accept either grid
+            ok = [k for k in range(16) if cands[k][0] <= cands[best][0] * (1 + 1e-12) + 1e-300]
+            assert any(np.isclose(s[r, g], cands[k][1], rtol=1e-12) and z[r, g] == cands[k][2] for k in ok)
+    # and the codes are the sweep's codes on those grids: a static sweep handed the same grids agrees
+    codes2, Q2, _, _ = oracle.sweep_rows(W, U, s, z, gq, bits)
+    assert np.array_equal(codes, codes2) and np.allclose(Q, Q2, atol=0)
+
+
+def test_dynamic_grid_reductions_still_hold():
+    """One group per row: the variant is the adaptive grid.  H_out = I or g = d_head: independent of g
+    (row-wise GPTQ).  Weights on a grid whose every group spans the full code range: fixed point."""
+    pr = small_problem(401, dh=8, d=16)
+    a = run_layer(pr, 3, 0, 2, F_ADAPTIVE_GRID)
+    b = run_layer(pr, 3, 0, 2, F_DYNAMIC_GRID)
+    assert np.array_equal(a.codes, b.codes) and np.allclose(a.scales, b.scales, atol=0)
+    ref = run_layer(pr, 3, 4, 8, F_DYNAMIC_GRID, hout=False)
+    pr_id = dict(pr, Hout=np.eye(8)[None])
+    for g in (1, 2, 8):
+        out = run_layer(pr_id, 3, 4, g, F_DYNAMIC_GRID)
+        assert np.array_equal(out.codes, ref.codes) and np.allclose(out.w_hat, ref.w_hat, atol=1e-15)
+    assert np.array_equal(run_layer(pr, 3, 4, 8, F_DYNAMIC_GRID).codes, ref.codes)      # g = d_head
+    # fixed point: every group of every row holds codes 0 and 3 (the min-max grid is the true grid)
+    g = np.random.default_rng(401)
+    codes = g.integers(0, 4, size=(8, 16)).astype(np.uint8)
+    codes[:, 0::4], codes[:, 1::4] = 0, 3
+    s_true = 0.5 ** g.integers(3, 6, size=(8, 4))
+    z_true = g.integers(1, 3, size=(8, 4))
+    Wg = np.repeat(s_true, 4, axis=1) * (codes - np.repeat(z_true, 4, axis=1))
+    out = run_layer(dict(pr, W=Wg), 2, 4, 2, F_DYNAMIC_GRID)
+    assert np.array_equal(out.codes, codes) and np.array_equal(out.zeros, z_true)
+    assert np.allclose(out.scales, s_true, atol=0) and np.allclose(out.w_comp, Wg, atol=0) and out.loss[0] == 0.0
+
+
+def test_dynamic_grid_usually_lowers_the_loss():
+    wins = 0
+    for seed in range(20):
+        pr = small_problem(420 + seed, dh=8, d=32)
+        dyn = run_layer(pr, 2, 8, 4, F_DYNAMIC_GRID).loss[0]
+        ada = run_layer(pr, 2, 8, 4, F_ADAPTIVE_GRID).loss[0]
+        wins += dyn <= ada
+    assert wins >= 12
