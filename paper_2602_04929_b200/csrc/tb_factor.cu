@@ -347,7 +347,9 @@ struct FactorSide {
   cudaStream_t inv;     // the inverse above the blocks: second products of the upper levels
   cudaStream_t low[2];  // the inverse inside a block of 512 columns, blocks in turn
   cudaStream_t inv2[8];  // first products of the doubling levels above one block, a stream per level
+  cudaStream_t rest;    // the wide rank-256 updates beyond the next outer block's columns
   cudaEvent_t fork, panel, trail[2], block_done, inv_done, crit_done, half_done, first_done[8], low_done[2];
+  cudaEvent_t outer_panels, strip_done, rest_done;
   bool ready;
 };
 
@@ -379,6 +381,10 @@ static FactorSide* factor_side() {
       if (cudaEventCreateWithFlags(&s->first_done[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
     if (cudaEventCreateWithFlags(&s->block_done, cudaEventDisableTiming) != cudaSuccess) return nullptr;
     if (cudaEventCreateWithFlags(&s->inv_done, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    if (cudaStreamCreateWithPriority(&s->rest, cudaStreamNonBlocking, least) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&s->outer_panels, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&s->strip_done, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&s->rest_done, cudaEventDisableTiming) != cudaSuccess) return nullptr;
     s->ready = true;
   }
   return s;
@@ -432,6 +438,7 @@ tb_status tb::factor_run(const float* H, int n_batch, int d, float* U, float* Hi
     TB_CUDA_CHECK(cudaEventRecord(side->fork, st));
     TB_CUDA_CHECK(cudaStreamWaitEvent(side->stream, side->fork, 0));
     TB_CUDA_CHECK(cudaStreamWaitEvent(side->crit, side->fork, 0));
+    TB_CUDA_CHECK(cudaStreamWaitEvent(side->rest, side->fork, 0));
   }
   // L^{-1} block by block of G columns.  Block j can be inverted as soon as its last panel is factored:
   // its 64 x 64 diagonal inverses, the doubling levels inside the block, then every level above whose
@@ -560,14 +567,55 @@ tb_status tb::factor_run(const float* H, int n_batch, int d, float* U, float* Hi
   };
   int next_inv_block = 0;
 
-  // Panel k applies the update of panel k-1 to its own 64 columns itself; the trailing update after
-  // panel k covers the columns from panel k+2 on.  With the look-ahead it runs on the helper stream
-  // beside panel k+1, and panel k+2 waits for it (two events in turn).
+  // Two levels of blocking.  Outer blocks of OB = 256 columns (four panels).  Panel k applies the
+  // update of panel k-1 to its own 64 columns itself; the rank-64 update after panel k covers the
+  // columns from panel k+2 on up to ZL = 128 columns past the end of its outer block (a strip at most
+  // 256 columns wide), so that the first two panels of the next block never wait for anything wide.
+  // After a block's last panel its 256 columns update everything further right in one rank-256
+  // product, in two launches: the columns up to ZL past the next block's end ("near": the next block's
+  // third panel is the first to need it), then the rest ("far").  A rank-64 update of the whole
+  // trailing matrix moves the matrix through memory once per panel and is bound by that traffic;
+  // rank-256 updates move it a quarter as often and run at the GEMM engine's large-K efficiency.
+  // With the look-ahead: panels on the high-priority stream, the rank-64 strips and the near updates
+  // in order on the trailing stream, the far updates on a low-priority stream beside the next block's
+  // panels.  The far update of block J and the near update of block J+1 overlap in their columns, so
+  // the latter waits for the former: every entry receives its updates in the same order as in the
+  // single-stream schedule, and the results agree bit for bit.
+  enum { OB = 4 * FNB, ZL = 2 * FNB };
   bool trail_set[2] = {false, false};
+  bool strip_set = false, rest_set = false;
+  auto rank_update = [&](int k_lo, int k_cnt, int c_lo, int c_hi, cudaStream_t stream_u) -> tb_status {
+    // A[r][c] -= sum_k L[r][k_lo + k] L[c][k_lo + k] for c in [c_lo, c_hi), r >= c (tiles on or below the diagonal)
+    if (c_hi <= c_lo) return TB_OK;
+    GemmP t = gemm_params();
+    t.A = f.A + (long long)c_lo * dp + k_lo;
+    t.a_m = dp;
+    t.a_k = 1;
+    t.a_batch = pp;
+    t.B = t.A;  // B(k, n) = L[c_lo + n][k_lo + k]
+    t.b_k = 1;
+    t.b_n = dp;
+    t.b_batch = pp;
+    t.C = f.A + (long long)c_lo * dp + c_lo;
+    t.ldc = dp;
+    t.c_batch = pp;
+    t.M = d_fact - c_lo;
+    t.N = c_hi - c_lo;
+    t.K = k_cnt;
+    t.n_batch = n_batch;
+    t.alpha = -1.0;
+    t.beta = 1.0;
+    t.flags = GEMM_LOWER_TILES;
+    return gemm_launch<double, double, double, double, false, false>(t, stream_u);
+  };
   for (int k0 = 0; k0 < d_fact; k0 += FNB) {
     const int r0 = k0 + FNB, m = d_fact - r0;
     const int xt = (m > 0) ? m / FNB : 1;
     const int pi = k0 / FNB;
+    const int j0 = (k0 / OB) * OB;                               // first column of this outer block
+    const int j1 = (j0 + OB < d_fact) ? j0 + OB : d_fact;        // one past its last column
+    const bool last_in_block = (r0 >= j1);
+    auto clip = [&](int c) { return c < d_fact ? c : d_fact; };
     if (side && trail_set[pi & 1]) TB_CUDA_CHECK(cudaStreamWaitEvent(cs, side->trail[pi & 1], 0));
     k_chol_panel<<<dim3(xt, n_batch), PANEL_THREADS, PANEL_SMEM, cs>>>(f.A, f.tmp, (long long)f.tmp_per, info, dp, k0,
                                                                        d_fact, k0 > 0 ? 1 : 0);
@@ -590,39 +638,47 @@ tb_status tb::factor_run(const float* H, int n_batch, int d, float* U, float* Hi
     }
     if (m <= 0) break;
     trail_set[pi & 1] = false;
-    if (m <= FNB) continue;  // only the next panel's columns are left, and that panel updates them itself
-    GemmP t = gemm_params();  // trailing -= panel panel^T from column r0 + 64 on, tiles on or below the diagonal
-    t.A = f.A + (long long)(r0 + FNB) * dp + k0;
-    t.a_m = dp;
-    t.a_k = 1;
-    t.a_batch = pp;
-    t.B = t.A;  // B(k, n) = panel[n][k]
-    t.b_k = 1;
-    t.b_n = dp;
-    t.b_batch = pp;
-    t.C = f.A + (long long)(r0 + FNB) * dp + (r0 + FNB);
-    t.ldc = dp;
-    t.c_batch = pp;
-    t.M = m - FNB;
-    t.N = m - FNB;
-    t.K = FNB;
-    t.n_batch = n_batch;
-    t.alpha = -1.0;
-    t.beta = 1.0;
-    t.flags = GEMM_LOWER_TILES;
+    // rank-64 strip: the columns from panel k+2 on, up to ZL past the end of the outer block
+    const int t_lo = clip(r0 + FNB), t_hi = clip(j1 + ZL);
+    if (side && (t_hi > t_lo || last_in_block)) {
+      TB_CUDA_CHECK(cudaEventRecord(side->panel, cs));
+      TB_CUDA_CHECK(cudaStreamWaitEvent(side->stream, side->panel, 0));
+    }
+    if (t_hi > t_lo) {
+      TB_TRY(rank_update(k0, FNB, t_lo, t_hi, side ? side->stream : st));
+      if (side) {
+        TB_CUDA_CHECK(cudaEventRecord(side->trail[pi & 1], side->stream));
+        trail_set[pi & 1] = true;
+      }
+    }
+    if (!last_in_block) continue;
+    // the block is factored: rank-(j1 - j0) update of everything further right
+    const int n_lo = clip(j1 + ZL), n_hi = clip(j1 + OB + ZL);
     if (!side) {
-      TB_TRY((gemm_launch<double, double, double, double, false, false>(t, st)));
+      TB_TRY(rank_update(j0, j1 - j0, n_lo, n_hi, st));
+      TB_TRY(rank_update(j0, j1 - j0, n_hi, d_fact, st));
       continue;
     }
-    TB_CUDA_CHECK(cudaEventRecord(side->panel, cs));
-    TB_CUDA_CHECK(cudaStreamWaitEvent(side->stream, side->panel, 0));
-    TB_TRY((gemm_launch<double, double, double, double, false, false>(t, side->stream)));
-    TB_CUDA_CHECK(cudaEventRecord(side->trail[pi & 1], side->stream));
-    trail_set[pi & 1] = true;
+    if (n_hi > n_lo) {
+      // near: overlaps the previous block's far update in these columns, so after it
+      if (rest_set) TB_CUDA_CHECK(cudaStreamWaitEvent(side->stream, side->rest_done, 0));
+      TB_TRY(rank_update(j0, j1 - j0, n_lo, n_hi, side->stream));
+      // later strips of this stream follow it in order; the panels that need it wait for those strips
+      TB_CUDA_CHECK(cudaEventRecord(side->strip_done, side->stream));
+      strip_set = true;
+    }
+    if (n_hi < d_fact) {
+      TB_CUDA_CHECK(cudaStreamWaitEvent(side->rest, side->panel, 0));
+      TB_TRY(rank_update(j0, j1 - j0, n_hi, d_fact, side->rest));
+      TB_CUDA_CHECK(cudaEventRecord(side->rest_done, side->rest));
+      rest_set = true;
+    }
   }
   if (side) {
     for (int i = 0; i < 2; ++i)
       if (trail_set[i]) TB_CUDA_CHECK(cudaStreamWaitEvent(st, side->trail[i], 0));
+    if (strip_set) TB_CUDA_CHECK(cudaStreamWaitEvent(st, side->strip_done, 0));
+    if (rest_set) TB_CUDA_CHECK(cudaStreamWaitEvent(st, side->rest_done, 0));
     TB_CUDA_CHECK(cudaEventRecord(side->crit_done, side->crit));
     TB_CUDA_CHECK(cudaStreamWaitEvent(st, side->crit_done, 0));
   }
