@@ -27,6 +27,7 @@
 //   5. U = J L^{-1} J, written as float with an explicit zero lower triangle.
 #include "tb_common.cuh"
 #include "tb_gemm.cuh"
+#include "tb_gemm64.cuh"
 
 namespace tb {
 
@@ -483,7 +484,7 @@ tb_status tb::factor_run(const float* H, int n_batch, int d, float* U, float* Hi
       gp.boff = n0;
       gp.C = tmp + n0;
       gp.N = (sblk - n0 < piece) ? sblk - n0 : piece;
-      TB_TRY((gemm_launch<double, double, double, double, false, true>(gp, stream_first)));
+      TB_TRY((gemm64_launch<true>(gp, stream_first)));
     }
     return TB_OK;
   };
@@ -509,7 +510,7 @@ tb_status tb::factor_run(const float* H, int n_batch, int d, float* U, float* Hi
     h.alpha = -1.0;
     h.atrim = 1;
     h.flags = GEMM_HEAVY_M_LAST;
-    return gemm_launch<double, double, double, double, false, true>(h, stream_second);
+    return gemm64_launch<true>(h, stream_second);
   };
   auto high_tmp = [&](int sblk) {  // region of the level-sblk product (first matrix of the batch)
     size_t o = f.high_off;
@@ -606,7 +607,7 @@ tb_status tb::factor_run(const float* H, int n_batch, int d, float* U, float* Hi
     t.alpha = -1.0;
     t.beta = 1.0;
     t.flags = GEMM_LOWER_TILES;
-    return gemm_launch<double, double, double, double, false, false>(t, stream_u);
+    return gemm64_launch<false>(t, stream_u);
   };
   for (int k0 = 0; k0 < d_fact; k0 += FNB) {
     const int r0 = k0 + FNB, m = d_fact - r0;
