@@ -19,7 +19,6 @@
 
 #include "tb_common.cuh"
 #include "tb_gemm.cuh"
-#include "tb_gemm64.cuh"
 #include "tb_profile.cuh"
 #include "tb_tma.cuh"
 
@@ -2114,7 +2113,7 @@ extern "C" tb_status tb_quantize_layer(const tb_layer_desc* desc, const float* W
       g.n_batch = p.H;
       g.alpha = -1.0;
       g.beta = 1.0;
-      TB_TRY((gemm64_launch<true>(g, st)));
+      TB_TRY((gemm_launch<double, double, double, double, false, true>(g, st)));
     }
   }
 
