@@ -518,6 +518,8 @@ def main(argv=None):
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(tb_inputs.CONFIGS))
     ap.add_argument("--tokens", type=int, default=0, help="override the token count (default: the config's)")
+    ap.add_argument("--heads", type=int, default=0,
+                    help="single-projection workloads: keep only this many heads (small captures under a profiler)")
     ap.add_argument("--no-configs", action="store_true", help="skip the other four configurations")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -529,6 +531,11 @@ def main(argv=None):
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     cfg = tb_inputs.CONFIGS[args.workload]
+    if args.heads and not is_block(cfg) and cfg.projections[0].partner:
+        import dataclasses
+        p0 = cfg.projections[0]
+        cfg = dataclasses.replace(cfg, projections=(dataclasses.replace(p0, n_heads=args.heads,
+                                                                       d_out=args.heads * p0.d_head),))
     if args.impl == "reference":
         run_reference(args, cfg, rank)
         return
