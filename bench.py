@@ -47,7 +47,17 @@ FP32_FFMA_MEASURED_TFLOPS = 71.5
 FP64_KIND = "FP64 FMA / FP64 tensor pipe, 148 SM x 64 lanes x 2 x 1.965 GHz"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (bytes), keyed by (workload, kernel); absent where the kernel has changed since its capture
-NCU_TRAFFIC = {}
+# (the mean over the launches of that kernel in one layer; the Hessian kernel's figure holds for the
+# default 262 144 tokens only)
+NCU_TRAFFIC = {
+    ("l2_70b_block", "k_sweep_rows"): 755.0e6,     # 13 launches per layer, 9.8 GB in all
+    ("l2_70b_block", "k_grid_tri"): 314.1e6,       # 4 launches per layer
+    ("l2_70b_block", "k_syrk_tc"): 51.9e9,         # 10 launches per layer, 42.7 .. 58.7 GB read each
+    ("l2_7b_q", "k_sweep_rows"): 77.9e6,           # 4 launches per layer
+    ("l2_7b_q", "k_grid_tri"): 34.9e6,             # 4 launches per layer
+    ("l2_7b_q", "k_syrk_tc"): 6.91e9,
+}
+NCU_TRAFFIC_TOKENS = 262144
 
 
 # --------------------------------------------------------------------------------------------
@@ -473,7 +483,7 @@ def rooflines(cfg, n_tok, m, peaks):
         ach = hessian_flops(cfg, n_tok) / (ph["hessian"] * 1e-3) / 1e12
         out["hessian"] = {"kernel": "k_syrk_tc (+ mirror, finalize)", "bound": "tensor", "achieved": ach, "peak": bf16_peak,
                           "unit": "TFLOP/s", "frac": ach / bf16_peak, "peak_kind": bf16_kind, "ms": ph["hessian"],
-                          "traffic": NCU_TRAFFIC.get((cfg.name, "k_syrk_tc"))}
+                          "traffic": NCU_TRAFFIC.get((cfg.name, "k_syrk_tc")) if n_tok == NCU_TRAFFIC_TOKENS else None}
     return out, loop_ms
 
 
@@ -534,8 +544,9 @@ def main(argv=None):
     if args.heads and not is_block(cfg) and cfg.projections[0].partner:
         import dataclasses
         p0 = cfg.projections[0]
-        cfg = dataclasses.replace(cfg, projections=(dataclasses.replace(p0, n_heads=args.heads,
-                                                                       d_out=args.heads * p0.d_head),))
+        cfg = dataclasses.replace(cfg, name=f"{cfg.name}[{args.heads} heads]",
+                                  projections=(dataclasses.replace(p0, n_heads=args.heads,
+                                                                   d_out=args.heads * p0.d_head),))
     if args.impl == "reference":
         run_reference(args, cfg, rank)
         return
