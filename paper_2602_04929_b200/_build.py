@@ -13,7 +13,7 @@ INCLUDE = os.path.join(ROOT, "include")
 OBJ_DIR = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libturboboa.so")
 
-SOURCES = ["tb_api.cu", "tb_hessian.cu", "tb_syrk_tc.cu", "tb_cross_tc.cu", "tb_gemm_tc.cu", "tb_factor.cu", "tb_factor_static.cu", "tb_quantize.cu", "tb_block.cu", "tb_pack.cu"]
+SOURCES = ["tb_api.cu", "tb_hessian.cu", "tb_syrk_tc.cu", "tb_syrk_tc2.cu", "tb_cross_tc.cu", "tb_gemm_tc.cu", "tb_factor.cu", "tb_factor_static.cu", "tb_quantize.cu", "tb_block.cu", "tb_pack.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-Werror=pointer-arith",   # no arithmetic on untyped pointers
               "-I", INCLUDE, "-I", CSRC]
