@@ -50,9 +50,9 @@ FP64_KIND = "FP64 FMA / FP64 tensor pipe, 148 SM x 64 lanes x 2 x 1.965 GHz"
 # (the mean over the launches of that kernel in one layer; the Hessian kernel's figure holds for the
 # default 262 144 tokens only)
 NCU_TRAFFIC = {
-    ("l2_70b_block", "k_sweep_rows"): 755.0e6,     # 13 launches per layer, 9.8 GB in all
+    ("l2_70b_block", "k_sweep_rows"): 759.0e6,     # 13 launches per layer, 9.9 GB in all
     ("l2_70b_block", "k_grid_tri"): 314.1e6,       # 4 launches per layer
-    ("l2_70b_block", "k_syrk_tc"): 51.9e9,         # 10 launches per layer, 42.7 .. 58.7 GB read each
+    ("l2_70b_block", "k_syrk_tc"): 58.1e9,         # 10 launches per layer (pair form), 54.8 .. 59.0 GB read each
     ("l2_7b_q", "k_sweep_rows"): 77.9e6,           # 4 launches per layer
     ("l2_7b_q", "k_grid_tri"): 34.9e6,             # 4 launches per layer
     ("l2_7b_q", "k_syrk_tc"): 6.91e9,
@@ -481,7 +481,7 @@ def rooflines(cfg, n_tok, m, peaks):
     alu("loop", "grid + sweep + compensation", loop_flops(cfg), loop_ms)
     if ph.get("hessian"):
         ach = hessian_flops(cfg, n_tok) / (ph["hessian"] * 1e-3) / 1e12
-        out["hessian"] = {"kernel": "k_syrk_tc (+ mirror, finalize)", "bound": "tensor", "achieved": ach, "peak": bf16_peak,
+        out["hessian"] = {"kernel": "k_syrk_tc / k_syrk_tc_pair from 6144 columns on (+ mirror, finalize)", "bound": "tensor", "achieved": ach, "peak": bf16_peak,
                           "unit": "TFLOP/s", "frac": ach / bf16_peak, "peak_kind": bf16_kind, "ms": ph["hessian"],
                           "traffic": NCU_TRAFFIC.get((cfg.name, "k_syrk_tc")) if n_tok == NCU_TRAFFIC_TOKENS else None}
     return out, loop_ms
