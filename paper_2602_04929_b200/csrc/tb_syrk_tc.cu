@@ -218,8 +218,8 @@ tb_status syrk_bf16_tensor_pair(float* H, const __nv_bfloat16* X, long long n_to
 
 tb_status syrk_bf16_tensor(float* H, const __nv_bfloat16* X, long long n_tok, int d, cudaStream_t st) {
   if (n_tok > 0x7fffffffll) return TB_ERR_UNSUPPORTED;
-  // From 6144 columns on, 256 x 256 tiles on CTA pairs are faster (measured: 3 % at 6144, 15 % at 8192; below
-  // that the single-CTA tiles win by 2-10 %).
+  // From 6144 columns on, 256 x 256 tiles on CTA pairs (measured: 11 % faster at 8192 columns, level at 5120
+  // and 6144; below that the single-CTA tiles win by 3-10 %).
   if (d >= 6144) return syrk_bf16_tensor_pair(H, X, n_tok, d, st);
   CUtensorMap map;
   TB_TRY(make_map_2d(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, sizeof(__nv_bfloat16), X, (unsigned long long)d,
@@ -236,7 +236,9 @@ tb_status syrk_bf16_tensor(float* H, const __nv_bfloat16* X, long long n_tok, in
     TB_CUDA_CHECK(cudaFuncSetAttribute(k_syrk_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM));
     configured[dev] = true;
   }
-  const int grid = n_tiles < sms ? n_tiles : sms;
+  // as many CTAs as fill the rounds of tiles evenly (the same number of rounds as with every SM)
+  const int rounds = (n_tiles + sms - 1) / (sms > 0 ? sms : 1);
+  const int grid = (n_tiles + rounds - 1) / rounds;
   k_syrk_tc<<<grid, TC_THREADS, TC_SMEM, st>>>(H, map, (int)n_tok, d, n_tiles);
   TB_LAUNCH_CHECK();
   return TB_OK;

@@ -309,7 +309,11 @@ tb_status syrk_bf16_tensor_pair(float* H, const __nv_bfloat16* X, long long n_to
     TB_CUDA_CHECK(cudaFuncSetAttribute(k_syrk_tc_pair, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)T2_SMEM));
     configured[dev] = true;
   }
-  const int pairs = n_tiles < sms / 2 ? n_tiles : sms / 2;
+  // as many pairs as fill the rounds evenly: 528 tiles on 74 pairs take 8 rounds, the last one with 10 tiles;
+  // 66 pairs take the same 8 rounds and leave 16 SMs (and their share of the power budget) to other work
+  const int max_pairs = sms / 2 > 0 ? sms / 2 : 1;
+  const int rounds = (n_tiles + max_pairs - 1) / max_pairs;
+  const int pairs = (n_tiles + rounds - 1) / rounds;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(2 * pairs));
   cfg.blockDim = dim3(T2_THREADS);
