@@ -233,7 +233,10 @@ tb_status cross_bf16_tensor(float* R, const __nv_bfloat16* X, const __nv_bfloat1
     TB_CUDA_CHECK(cudaFuncSetAttribute(k_cross_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)XC_SMEM));
     configured[dev] = true;
   }
-  const int grid = n_tiles < sms ? n_tiles : sms;
+  // as many CTAs as fill the rounds of tiles evenly (the same number of rounds as with every SM: fewer CTAs
+  // asking L2 at once, and less power, for the same time or less)
+  const int rounds_of_tiles = (int)((n_tiles + sms - 1) / (sms > 0 ? sms : 1));
+  const int grid = (int)((n_tiles + rounds_of_tiles - 1) / (rounds_of_tiles > 0 ? rounds_of_tiles : 1));
   k_cross_tc<<<grid, XC_THREADS, XC_SMEM, st>>>(R, dmap, xmap, (int)ntp, d, n_tiles, alpha);
   TB_LAUNCH_CHECK();
   return TB_OK;

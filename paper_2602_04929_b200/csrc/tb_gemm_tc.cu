@@ -442,7 +442,10 @@ tb_status yw_tensor(float* Yw, const unsigned char* codes, const int* zeros, con
     TB_CUDA_CHECK(cudaFuncSetAttribute(k_yw_tc_stream, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)YS_SMEM));
     configured[dev] = true;
   }
-  const int grid = (int)(n_tiles < sms ? n_tiles : sms);
+  // as many CTAs as fill the rounds of tiles evenly (the same number of rounds as with every SM: fewer CTAs
+  // asking L2 at once, and less power, for the same time or less)
+  const int rounds_of_tiles = (int)((n_tiles + sms - 1) / (sms > 0 ? sms : 1));
+  const int grid = (int)((n_tiles + rounds_of_tiles - 1) / (rounds_of_tiles > 0 ? rounds_of_tiles : 1));
   if (resident)
     k_yw_tc<<<grid, YT_THREADS, YT_SMEM, st>>>(Yw, map_a, map_b, (int)rows, d, seg, ng, (int)n_tiles, hunits,
                                                (int)(rows / hunits));
@@ -685,7 +688,10 @@ tb_status gemm_split_presplit(double* C, long long ldc, const __nv_bfloat16* AT,
     TB_CUDA_CHECK(cudaFuncSetAttribute(k_gsplit_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GS_SMEM));
     configured[dev] = true;
   }
-  const int grid = (int)(n_tiles < sms ? n_tiles : sms);
+  // as many CTAs as fill the rounds of tiles evenly (the same number of rounds as with every SM: fewer CTAs
+  // asking L2 at once, and less power, for the same time or less)
+  const int rounds_of_tiles = (int)((n_tiles + sms - 1) / (sms > 0 ? sms : 1));
+  const int grid = (int)((n_tiles + rounds_of_tiles - 1) / (rounds_of_tiles > 0 ? rounds_of_tiles : 1));
   k_gsplit_tc<<<grid, YT_THREADS, GS_SMEM, st>>>(C, ldc, map_a, map_b, (int)M, N, K, (int)n_tiles, accumulate ? 1 : 0,
                                                  hunits, (int)(M / hunits));
   TB_LAUNCH_CHECK();
