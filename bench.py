@@ -52,7 +52,7 @@ FP64_KIND = "FP64 FMA / FP64 tensor pipe, 148 SM x 64 lanes x 2 x 1.965 GHz"
 NCU_TRAFFIC = {
     ("l2_70b_block", "k_sweep_rows"): 759.0e6,     # 13 launches per layer, 9.9 GB in all
     ("l2_70b_block", "k_grid_tri"): 314.1e6,       # 4 launches per layer
-    ("l2_70b_block", "k_syrk_tc"): 58.1e9,         # 10 launches per layer (pair form), 54.8 .. 59.0 GB read each
+    ("l2_70b_block", "k_syrk_tc"): 55.2e9,         # 10 launches per layer (pair form, 66 pairs), 49.4 .. 58.7 GB read each
     ("l2_7b_q", "k_sweep_rows"): 77.9e6,           # 4 launches per layer
     ("l2_7b_q", "k_grid_tri"): 34.9e6,             # 4 launches per layer
     ("l2_7b_q", "k_syrk_tc"): 6.91e9,
