@@ -230,6 +230,39 @@ def test_prerequisites_at_full_width():
     assert errs["H_out"] <= 2e-6
 
 
+def test_hessian_at_the_benchmark_size_on_sampled_entries():
+    """The Hessian of the headline benchmark (262 144 bf16 tokens, 8192 columns: one call, the launch the
+    benchmark times, CTA pairs on 256 x 256 tiles) against the oracle on sampled entries: the oracle gets
+    the sampled columns of the same seeded activations and returns their block of X^T X / n in float64.
+    The columns are chosen around tile edges (127 | 128, 255 | 256), in the first and the last tile and
+    across distant tiles, so that every kind of tile (diagonal, below the diagonal, last round) and the
+    mirrored half are hit.  Tolerance as in the small cases: 1e-5 of sqrt(H_ii H_jj) per entry."""
+    import torch
+    import paper_2602_04929_b200 as tb
+    d, n_tok = 8192, 262144
+    rec = tb_inputs.HeavyTailRecipe(d, seed=5)
+    X = tb_inputs.heavy_tail_device(rec, n_tok, "cuda:0", seed=1)
+    H = torch.zeros((d, d), dtype=torch.float32, device="cuda:0")
+    Hsum = torch.empty_like(H)
+    tb.tb_accumulate_hessian(H, X)
+    tb.tb_finalize_hessian(H, None, n_tok, 0.0, Hsum_out=Hsum)
+    torch.cuda.synchronize()
+    assert tb.tb_device_error_flag() == 0
+    cols = sorted({0, 1, 63, 64, 127, 128, 129, 255, 256, 257, 511, 512, 1000, 2047, 2048, 3071, 4095, 4096, 4097,
+                   5000, 6143, 6144, 7000, 7935, 7936, 8063, 8064, 8190, 8191})
+    idx = torch.tensor(cols, device="cuda:0")
+    Xs = X[:, idx].float().cpu().numpy()                 # bf16 values are exact in float
+    Ho = oracle.hessian(Xs, damp=0.0)                    # [len(cols)]^2 block of X^T X / n in float64
+    Hg = Hsum[idx][:, idx].cpu().numpy().astype(np.float64)
+    scale = np.sqrt(np.outer(np.diag(Ho), np.diag(Ho)))
+    err = np.max(np.abs(Hg - Ho) / scale)
+    print("FULL-SIZE HESSIAN sampled entries:", len(cols) ** 2, "max scaled error", err)
+    assert err <= 1e-5
+    assert np.array_equal(Hg, Hg.T)                      # the mirrored half is a copy
+    del X, H, Hsum
+    torch.cuda.empty_cache()
+
+
 def test_bounded_wait_gives_up_and_leaves_the_context_usable():
     """A wait on a hardware barrier at which nothing ever arrives, with a budget of about 1 ms: the
     kernel must return by itself, the device error word must be raised (and cleared by reading it),
