@@ -16,7 +16,7 @@ using namespace tb;
 
 namespace {
 
-enum { N_HELPERS = 4, STAGE_SLOTS = 2 };
+enum { N_HELPERS = 4, STAGE_SLOTS = 8 };
 
 // Helper streams and events of the block level, one set per device, created on first use and
 // kept for the life of the process.
@@ -34,8 +34,13 @@ BlockSide* block_side() {
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
   BlockSide* s = &per_device[dev];
   if (!s->ready) {
+    int prio_low = 0, prio_high = 0;
+    if (cudaDeviceGetStreamPriorityRange(&prio_low, &prio_high) != cudaSuccess) return nullptr;
     for (int i = 0; i < N_HELPERS; ++i) {
-      if (cudaStreamCreateWithFlags(&s->helper[i], cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+      // the last helper is the ingest stream of the host mode: its short Hessian launches go first when SMs
+      // fall free, so that the staging slots drain while long quantizer launches hold the GPU
+      const int prio = (i == N_HELPERS - 1) ? prio_high : prio_low;
+      if (cudaStreamCreateWithPriority(&s->helper[i], cudaStreamNonBlocking, prio) != cudaSuccess) return nullptr;
       if (cudaEventCreateWithFlags(&s->join[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
     }
     if (cudaStreamCreateWithFlags(&s->copy, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
@@ -277,7 +282,7 @@ tb_status make_layer_plan(const tb_attention_desc* D, const tb_attention_io* io,
 }
 
 // H (+ R) of one activation tensor [n_tok][width], un-normalised sums then finalised.
-// Device-resident tensors go through in one call; host tensors in pieces through the two staging
+// Device-resident tensors go through in one call; host tensors in pieces through the staging
 // slots on the copy stream, each piece accumulated as soon as it has arrived.
 tb_status accumulate_input(const LayerPlan& p, BlockSide* bs, const void* X, const void* Xfp, int width, float* H,
                            float* R, float* Hsum, float damp, float alpha, cudaStream_t st) {
@@ -347,8 +352,25 @@ tb_status layer_enqueue(const tb_attention_desc* D, const tb_attention_io* io, L
   info_out[2] = info_out[1] + p.hkv;
   TB_CUDA_CHECK(cudaMemsetAsync(p.info, 0, sizeof(int) * (size_t)p.info_count, st));
 
+  // With host buffers the Hessians accumulate on a stream of their own ("ingest"), piece by piece as the
+  // copies land, and everything that is not a Hessian (factors, correction operands, the quantizer) runs on
+  // the caller's stream behind an event per finished Hessian: the copy engine then never waits for a factor
+  // or for the quantizer, and the order of the inputs is chosen so that as much as possible of that work
+  // has run by the time the last activation has crossed: attention input, output projection's input, then
+  // the value heads (each factored alone as soon as its Hessian is complete, which gives the batched
+  // factor's numbers bit for bit), the value projection last.
+  cudaStream_t in = p.on_host ? bs->helper[N_HELPERS - 1] : st;
+  auto hessian_ready = [&]() -> tb_status {   // work enqueued on st from here on sees what `in` has done so far
+    if (in == st) return TB_OK;
+    TB_CUDA_CHECK(cudaEventRecord(bs->dep[N_HELPERS + 1], in));
+    TB_CUDA_CHECK(cudaStreamWaitEvent(st, bs->dep[N_HELPERS + 1], 0));
+    return TB_OK;
+  };
+  if (in != st) TB_CUDA_CHECK(cudaStreamWaitEvent(in, bs->fork, 0));  // after the caller's earlier work
+
   // ---- the attention input: H_in of W_Q, W_K (and of W_V without per-head inputs), and R ----
-  TB_TRY(accumulate_input(p, bs, io->X, io->X_fp, p.d, p.attn.H, p.attn.R, p.attn.Hsum, D->damp, D->alpha, st));
+  TB_TRY(accumulate_input(p, bs, io->X, io->X_fp, p.d, p.attn.H, p.attn.R, p.attn.Hsum, D->damp, D->alpha, in));
+  TB_TRY(hessian_ready());
 
   // ---- out-channel Hessians of Table 1 and their factors: they need Hsum and the partner weights
   // only, so with `concurrent` they run on helper streams beside the factor of H_in ----
@@ -397,25 +419,41 @@ tb_status layer_enqueue(const tb_attention_desc* D, const tb_attention_io* io, L
   }
 
   // ---- the value projection's own input Hessians, one per key/value head (Table 1, W_V row) ----
-  if (p.per_head_v) {
+  auto value_side = [&]() -> tb_status {
+    if (!p.per_head_v) return TB_OK;
     for (int h = 0; h < p.hkv; ++h) {
       const __nv_bfloat16* Xh = static_cast<const __nv_bfloat16*>(io->X_v) + (size_t)h * p.n_tok * p.d;
-      TB_TRY(accumulate_input(p, bs, Xh, nullptr, p.d, p.vhead.H + (size_t)h * dd, nullptr, nullptr, D->damp, 0.0f, st));
+      TB_TRY(accumulate_input(p, bs, Xh, nullptr, p.d, p.vhead.H + (size_t)h * dd, nullptr, nullptr, D->damp, 0.0f, in));
+      if (in != st) {
+        // host buffers: this head's factor runs while the next head's activations cross
+        TB_TRY(hessian_ready());
+        PhaseScope ph(PH_FACTOR, st);
+        TB_TRY(tb_factor(p.vhead.H + (size_t)h * dd, 1, p.d, p.vhead.U + (size_t)h * dd, nullptr, info_v + h, p.ws_factor,
+                         p.factor_bytes, st));
+      }
     }
+    if (in != st) return TB_OK;
     PhaseScope ph(PH_FACTOR, st);
-    TB_TRY(tb_factor(p.vhead.H, p.hkv, p.d, p.vhead.U, nullptr, info_v, p.ws_factor, p.factor_bytes, st));
-  }
+    return tb_factor(p.vhead.H, p.hkv, p.d, p.vhead.U, nullptr, info_v, p.ws_factor, p.factor_bytes, st);
+  };
 
   // ---- the output projection's input ----
-  TB_TRY(accumulate_input(p, bs, io->X_o, io->X_o_fp, p.dq, p.oin.H, p.oin.R, nullptr, D->damp, D->alpha, st));
-  {
-    PhaseScope ph(PH_FACTOR, st);
-    TB_TRY(tb_factor(p.oin.H, 1, p.dq, p.oin.U, nullptr, info_o, p.ws_factor, p.factor_bytes, st));
-  }
-  if (p.with_ro) {
-    PhaseScope ph(PH_PREP, st);
-    TB_TRY(tb_prepare_correction(p.oin.R, p.oin.U, 1, p.dq, p.oin.P, p.oin.C, p.ws_prep, p.prep_bytes, st));
-  }
+  auto output_side = [&]() -> tb_status {
+    TB_TRY(accumulate_input(p, bs, io->X_o, io->X_o_fp, p.dq, p.oin.H, p.oin.R, nullptr, D->damp, D->alpha, in));
+    TB_TRY(hessian_ready());
+    {
+      PhaseScope ph(PH_FACTOR, st);
+      TB_TRY(tb_factor(p.oin.H, 1, p.dq, p.oin.U, nullptr, info_o, p.ws_factor, p.factor_bytes, st));
+    }
+    if (p.with_ro) {
+      PhaseScope ph(PH_PREP, st);
+      TB_TRY(tb_prepare_correction(p.oin.R, p.oin.U, 1, p.dq, p.oin.P, p.oin.C, p.ws_prep, p.prep_bytes, st));
+    }
+    return TB_OK;
+  };
+  const bool value_last = p.on_host && p.per_head_v;   // host buffers: the value heads cross last
+  if (!value_last) TB_TRY(value_side());
+  TB_TRY(output_side());
   if (p.concurrent) {
     TB_CUDA_CHECK(cudaStreamWaitEvent(st, bs->join[0], 0));
     TB_CUDA_CHECK(cudaStreamWaitEvent(st, bs->join[1], 0));
@@ -447,27 +485,40 @@ tb_status layer_enqueue(const tb_attention_desc* D, const tb_attention_io* io, L
     j.ws = p.ws_quant[i];
     j.ws_bytes = p.quant_bytes[i];
   }
-  // the two large projections first: their launches then fill the GPU while the small ones run beside them
-  const tb_projection_job order[4] = {jobs[0], jobs[3], jobs[1], jobs[2]};
-  TB_TRY(tb_quantize_block(order, 4, p.concurrent ? 1 : 0, st));
-
-  // ---- results ----
-  if (p.on_host) {
+  // results of projection i back to the host (host buffers only)
+  auto results_home = [&](int i) -> tb_status {
+    if (!p.on_host) return TB_OK;
     PhaseScope ph(PH_COPY, st);
-    for (int i = 0; i < 4; ++i) {
-      const size_t n = (size_t)p.desc[i].d_out * p.desc[i].d_in;
-      const size_t ng = D->quant_group > 0 ? (size_t)p.desc[i].d_in / D->quant_group : 1;
-      const size_t ns = (size_t)p.desc[i].d_out * ng;
-      TB_CUDA_CHECK(cudaMemcpyAsync(io->codes[i], p.codes[i], n, cudaMemcpyDeviceToHost, st));
-      TB_CUDA_CHECK(cudaMemcpyAsync(io->scales[i], p.scales[i], ns * sizeof(float), cudaMemcpyDeviceToHost, st));
-      TB_CUDA_CHECK(cudaMemcpyAsync(io->zeros[i], p.zeros[i], ns * sizeof(int), cudaMemcpyDeviceToHost, st));
-      if (io->W_hat[i])
-        TB_CUDA_CHECK(cudaMemcpyAsync(io->W_hat[i], p.What[i], n * sizeof(float), cudaMemcpyDeviceToHost, st));
-      if (io->loss[i])
-        TB_CUDA_CHECK(cudaMemcpyAsync(io->loss[i], p.loss[i], sizeof(double) * (size_t)p.desc[i].n_heads,
-                                      cudaMemcpyDeviceToHost, st));
-    }
+    const size_t n = (size_t)p.desc[i].d_out * p.desc[i].d_in;
+    const size_t ng = D->quant_group > 0 ? (size_t)p.desc[i].d_in / D->quant_group : 1;
+    const size_t ns = (size_t)p.desc[i].d_out * ng;
+    TB_CUDA_CHECK(cudaMemcpyAsync(io->codes[i], p.codes[i], n, cudaMemcpyDeviceToHost, st));
+    TB_CUDA_CHECK(cudaMemcpyAsync(io->scales[i], p.scales[i], ns * sizeof(float), cudaMemcpyDeviceToHost, st));
+    TB_CUDA_CHECK(cudaMemcpyAsync(io->zeros[i], p.zeros[i], ns * sizeof(int), cudaMemcpyDeviceToHost, st));
+    if (io->W_hat[i])
+      TB_CUDA_CHECK(cudaMemcpyAsync(io->W_hat[i], p.What[i], n * sizeof(float), cudaMemcpyDeviceToHost, st));
+    if (io->loss[i])
+      TB_CUDA_CHECK(cudaMemcpyAsync(io->loss[i], p.loss[i], sizeof(double) * (size_t)p.desc[i].n_heads,
+                                    cudaMemcpyDeviceToHost, st));
+    return TB_OK;
+  };
+  if (!value_last) {
+    // the two large projections first: their launches then fill the GPU while the small ones run beside them
+    const tb_projection_job order[4] = {jobs[0], jobs[3], jobs[1], jobs[2]};
+    TB_TRY(tb_quantize_block(order, 4, p.concurrent ? 1 : 0, st));
+    for (int i = 0; i < 4; ++i) TB_TRY(results_home(i));
+  } else {
+    // q, o and k while the value heads' activations are still crossing; then the value projection
+    const tb_projection_job first[3] = {jobs[0], jobs[3], jobs[1]};
+    TB_TRY(tb_quantize_block(first, 3, p.concurrent ? 1 : 0, st));
+    TB_TRY(results_home(0));
+    TB_TRY(results_home(3));
+    TB_TRY(results_home(1));
+    TB_TRY(value_side());
+    TB_TRY(tb_quantize_block(&jobs[2], 1, 0, st));
+    TB_TRY(results_home(2));
   }
+
   if (io->info) {
     TB_CUDA_CHECK(cudaMemcpyAsync(io->info, p.info, sizeof(int) * (size_t)p.info_count,
                                   p.on_host ? cudaMemcpyDeviceToHost : cudaMemcpyDeviceToDevice, st));
