@@ -383,10 +383,15 @@ typedef struct {
  * output projection runs with H_out = NULL (all rows at once, GPTAQ if X_o_fp
  * is given).  The workspace query only looks at which optional pointers of io
  * are non-NULL.  With on_host = 1 the activations cross to the device in pieces
- * of 16384 tokens on a copy stream while the Hessian of the pieces already there
- * accumulates (the Hessian's sums do not depend on the pieces; the deviation
- * correlation adds its two bf16 pieces per call, so its float sums differ from a
- * single call's in the last bits), results are copied back, and the call returns TB_ERR_NOT_SPD /
+ * of 16384 tokens on a copy stream (eight staging slots in the workspace) while
+ * the Hessian of the pieces already there accumulates on a stream of its own
+ * (the Hessian's sums do not depend on the pieces; the deviation correlation
+ * adds its two bf16 pieces per call, so its float sums differ from a single
+ * call's in the last bits).  The inputs cross in the order X, X_o, then the
+ * value heads of X_v; factors and quantizer calls follow each finished Hessian
+ * on the caller's stream (q, o and k are quantized while the value heads still
+ * cross, each value head is factored alone, with the batched factor's numbers),
+ * every projection's results are copied back as soon as it is done, and the call returns TB_ERR_NOT_SPD /
  * TB_ERR_TIMEOUT like tb_quantize_from_host; with on_host = 0 it only enqueues
  * and the caller reads `info`.  Helper streams as for tb_quantize_block. */
 int tb_attention_layer_info_count(const tb_attention_desc* desc, int per_head_v);
