@@ -409,14 +409,23 @@ tb_status layer_enqueue(const tb_attention_desc* D, const tb_attention_io* io, L
     TB_CUDA_CHECK(cudaEventRecord(bs->join[0], hs0));
     TB_CUDA_CHECK(cudaEventRecord(bs->join[1], hs1));
   }
+  // Side by side, device-resident, with per-head value inputs: the factor of the attention input's Hessian
+  // (one matrix: much of it waits on its own panel chain) runs on a helper stream beside the value heads'
+  // Hessians and is joined before the next factor, which shares its scratch.
+  cudaStream_t fs = (p.concurrent && !p.on_host && p.per_head_v) ? bs->helper[2] : st;
+  if (fs != st) {
+    TB_CUDA_CHECK(cudaEventRecord(bs->dep[N_HELPERS + 2], st));
+    TB_CUDA_CHECK(cudaStreamWaitEvent(fs, bs->dep[N_HELPERS + 2], 0));
+  }
   {
-    PhaseScope ph(PH_FACTOR, st);
-    TB_TRY(tb_factor(p.attn.H, 1, p.d, p.attn.U, nullptr, info_attn, p.ws_factor, p.factor_bytes, st));
+    PhaseScope ph(PH_FACTOR, fs);
+    TB_TRY(tb_factor(p.attn.H, 1, p.d, p.attn.U, nullptr, info_attn, p.ws_factor, p.factor_bytes, fs));
   }
   if (p.with_r) {
-    PhaseScope ph(PH_PREP, st);
-    TB_TRY(tb_prepare_correction(p.attn.R, p.attn.U, 1, p.d, p.attn.P, p.attn.C, p.ws_prep, p.prep_bytes, st));
+    PhaseScope ph(PH_PREP, fs);
+    TB_TRY(tb_prepare_correction(p.attn.R, p.attn.U, 1, p.d, p.attn.P, p.attn.C, p.ws_prep, p.prep_bytes, fs));
   }
+  if (fs != st) TB_CUDA_CHECK(cudaEventRecord(bs->dep[N_HELPERS + 3], fs));
 
   // ---- the value projection's own input Hessians, one per key/value head (Table 1, W_V row) ----
   auto value_side = [&]() -> tb_status {
@@ -433,6 +442,7 @@ tb_status layer_enqueue(const tb_attention_desc* D, const tb_attention_io* io, L
       }
     }
     if (in != st) return TB_OK;
+    if (fs != st) TB_CUDA_CHECK(cudaStreamWaitEvent(st, bs->dep[N_HELPERS + 3], 0));  // the attention input's factor is done
     PhaseScope ph(PH_FACTOR, st);
     return tb_factor(p.vhead.H, p.hkv, p.d, p.vhead.U, nullptr, info_v, p.ws_factor, p.factor_bytes, st);
   };
